@@ -1,0 +1,430 @@
+#!/usr/bin/env python
+"""Benchmark of the AASD draft-and-verify path on B200.
+
+One step = one pass of the whole path over one batch of the serving workload (256
+sequences, vocabulary 152064, bf16 logits): alignment sampling over the prefill logits of
+the sequences that arrive in that step (4 x 1024 rows), then one decoding step of all 256
+sequences: drafting, conditional verification of 256 x 2 x 8 = 4096 target rows, choice of
+the longest passing candidate and history append.  Over the configuration's 64 steps this
+is exactly its 256 x 1024 prefill rows and 64 x 4096 verification rows.
+
+The logits of every step are resident in HBM before the timed region (8 rotating buffers
+of 1.25 GB each for prefill and for verification rows: far larger than L2).  The decoding
+state is replayed: the logits of step j were drawn for the candidates the drafter emits at
+state j, and the state is restored every 8 steps by a small device copy inside the timed
+region.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload i]
+
+prints one JSON line.  `--impl reference` times the CPU oracle on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2505_13204_b200 import synth  # noqa: E402
+
+METRIC = "verified draft positions/sec"
+UNIT = "positions/s"
+ALPHA = float(np.float32(0.1))
+BETA = float(np.float32(0.1))
+K_EXTRA = 2
+N_BUF = 8
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(
+                ["nvidia-smi", "-i", str(index), "--query-gpu=" + self.Q,
+                 "--format=csv,noheader,nounits", "-lms", "50"], stdout=self.f,
+                stderr=subprocess.DEVNULL)
+        except OSError:
+            pass
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.f.read().splitlines():
+            t = [c.strip() for c in line.split(",")]
+            if len(t) < 7:
+                continue
+            try:
+                sm.append(float(t[0]))
+                mx.append(float(t[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, t[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        self.f.close()
+        os.unlink(self.f.name)
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), samples=len(sm),
+                       reasons=sorted(reasons))
+        return out
+
+
+# --------------------------------------------------------------------------------------
+# our arm
+# --------------------------------------------------------------------------------------
+class Bench:
+    def __init__(self, w: synth.Workload, device, rank: int):
+        from paper_2505_13204_b200 import binding
+        self.binding = binding
+        self.w = w
+        self.dev = device
+        self.ctx = binding.Context()
+        self.seqs_per_step = max(1, w.batch // w.steps)          # arriving sequences per step
+        self.pre_rows = self.seqs_per_step * w.prompt_len
+        self.R = w.rows_per_step
+        seed0 = w.seed + 1000 * rank
+        t0 = time.time()
+        self.prompts = [synth.prompt_ids(synth.scaled(w, seed=seed0), b) for b in range(w.batch)]
+        ids_all = torch.cat(self.prompts).to(device)
+        self.ids_all = ids_all
+        L = w.prompt_len
+        self.bank = synth.NoiseBank(max(self.pre_rows, self.R), w.vocab, seed0 + 7, device)
+        # alignment table of every sequence (set-up), keeping the first N_BUF prefill blocks
+        self.table = dict(
+            align_ids=torch.empty((w.batch * L, K_EXTRA), dtype=torch.int32, device=device),
+            n_extra=torch.empty(w.batch * L, dtype=torch.int32, device=device))
+        self.pre_bufs, self.pre_ids, self.pre_offs, self.pre_out = [], [], [], []
+        n_blocks = (w.batch + self.seqs_per_step - 1) // self.seqs_per_step
+        offs = torch.arange(0, self.pre_rows + 1, L, dtype=torch.int32, device=device)
+        scratch = None
+        for k in range(n_blocks):
+            lo = k * self.pre_rows
+            ids = ids_all[lo:lo + self.pre_rows]
+            hints = torch.cat([synth.next_token_hints(ids[i * L:(i + 1) * L])
+                               for i in range(self.seqs_per_step)])
+            keep = k < N_BUF
+            buf = None if not keep else torch.empty((self.pre_rows, w.vocab), dtype=w.torch_dtype,
+                                                     device=device)
+            if not keep and scratch is None:
+                scratch = torch.empty((self.pre_rows, w.vocab), dtype=w.torch_dtype, device=device)
+            x = synth.logits(self.pre_rows, w.vocab, w.torch_dtype, w.recipe, hints, seed0 + 31 * k,
+                             device=device, out=buf if keep else scratch,
+                             noise=self.bank.block(k), chunk_rows=1024)
+            out = self._align_out(lo)
+            self.ctx.align_sample(x, ids, offs, k_extra=K_EXTRA, outputs=out)
+            if keep:
+                self.pre_bufs.append(x)
+                self.pre_ids.append(ids)
+                self.pre_offs.append(offs)
+                self.pre_out.append(out)
+        del scratch
+        torch.cuda.synchronize()
+        # decoding state and the replayed verification logits
+        align = dict(align_ids=self.table["align_ids"], n_extra=self.table["n_extra"])
+        self.state = binding.DecodeState(self.ctx, self.prompts, N_BUF * (w.draft_len + 1) + 8, w.ngram,
+                                         w.draft_len, w.max_cands, w.vocab, w.torch_dtype, align=align,
+                                         alpha=ALPHA, beta=BETA)
+        self.hist0 = self.state.hist_ids.clone()
+        self.len0 = self.state.hist_len.clone()
+        self.ver_bufs = []
+        for j in range(N_BUF):
+            d = self.state.run_draft()["draft_ids"].reshape(-1).to(torch.int64)
+            x = synth.logits(self.R, w.vocab, w.torch_dtype, w.recipe, d, seed0 + 977 * (j + 1),
+                             device=device, noise=self.bank.block(100 + j), chunk_rows=1024)
+            self.ver_bufs.append(x)
+            self.state.step(x, j)
+        torch.cuda.synchronize()
+        self.accepted_per_cycle = int((self.state.hist_len - self.len0).sum().item())
+        self.restore()
+        self.ev_align = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+        self.setup_s = time.time() - t0
+        del self.bank
+
+    def _align_out(self, lo):
+        n = self.pre_rows
+        return dict(align_ids=self.table["align_ids"][lo:lo + n], n_extra=self.table["n_extra"][lo:lo + n],
+                    align_p=None, p_next=None, top1=None, entropy=None, pmax=None, aligned=None)
+
+    def restore(self):
+        self.state.hist_ids.copy_(self.hist0)
+        self.state.hist_len.copy_(self.len0)
+
+    def step(self, s: int, events=None):
+        j = s % N_BUF
+        if j == 0 and s > 0:
+            self.restore()
+        if events is not None:
+            events[0].record()
+        self.ctx.align_sample(self.pre_bufs[j], self.pre_ids[j], self.pre_offs[j], k_extra=K_EXTRA,
+                              outputs=self.pre_out[j])
+        if events is not None:
+            events[1].record()
+        self.state.step(self.ver_bufs[j], j)
+        if events is not None:
+            events[2].record()
+
+
+def run_ours(args, rank, world, local_rank):
+    import torch.distributed as dist
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    w = synth.workload(args.workload)
+    bench = Bench(w, dev, rank)
+    K, W = args.steps, max(args.warmup, 3)
+    for s in range(W):
+        bench.step(s)
+    torch.cuda.synchronize()
+    bench.restore()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    launches0 = bench.ctx.launch_count()
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
+    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    clocks = ClockSampler(local_rank)
+    time.sleep(0.2)
+    t_begin.record()
+    for s in range(K):
+        bench.step(s, evs[s])
+    t_end.record()
+    barrier()
+    clk = clocks.stop()
+    ms = t_begin.elapsed_time(t_end)
+    launches = bench.ctx.launch_count() - launches0
+    align_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in evs]))
+    decode_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in evs]))
+    if world > 1:
+        t = torch.tensor([ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+
+    # end to end: the same step fed from pinned host memory through the C ABI
+    e2e = run_e2e(bench, dev, min(K, 4))
+    if world > 1:
+        t = torch.tensor([e2e["ms_per_step"]], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e["ms_per_step"] = float(t.item())
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    esize = 2 if w.dtype == "bf16" else 4
+    peak, peak_src = measured_peaks()
+    row_bytes = w.vocab * esize
+    # the decode part is draft + verify + select + append; verification is all but a few us
+    ver_gbs = bench.R * row_bytes / (decode_ms * 1e-3) / 1e9
+    ali_gbs = bench.pre_rows * row_bytes / (align_ms * 1e-3) / 1e9
+    value = world * bench.R * K / (ms * 1e-3)
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "sequences_per_gpu": w.batch, "vocab": w.vocab,
+                   "logits_dtype": w.dtype, "verify_rows_per_step": bench.R,
+                   "prefill_rows_per_step": bench.pre_rows, "ngram": w.ngram, "k_extra": K_EXTRA,
+                   "alpha": ALPHA, "beta": BETA, "parallelism": "replicas x%d (sequences sharded, no collective)" % world,
+                   "l2": "inputs larger than L2: %d rotating buffers of %.2f GB" % (2 * N_BUF, bench.R * row_bytes / 1e9),
+                   "noise": "one bank of normals re-used under cyclic shifts",
+                   "setup_s": round(bench.setup_s, 1)},
+        "clocks": {"sm_mhz": clk["sm_mhz"], "sm_max_mhz": clk["sm_max_mhz"], "reasons": clk["reasons"],
+                   "samples": clk["samples"]},
+        "e2e": {"value": world * bench.R / (e2e["ms_per_step"] * 1e-3), "unit": UNIT,
+                "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
+                "ms_per_step": e2e["ms_per_step"]},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "hbm", "kernel": "verify_kernel<bf16> (timed with draft/select/append, <1% of it)",
+                     "achieved": ver_gbs, "peak": peak, "unit": "GB/s", "frac": ver_gbs / peak,
+                     "peak_source": peak_src + ", sustained copy figure", "traffic": None,
+                     "ms_per_launch": decode_ms, "bytes_per_launch": bench.R * row_bytes},
+        "roofline_align": {"bound": "hbm", "kernel": "align_kernel<bf16,2>", "achieved": ali_gbs, "peak": peak,
+                           "unit": "GB/s", "frac": ali_gbs / peak, "ms_per_launch": align_ms,
+                           "bytes_per_launch": bench.pre_rows * row_bytes},
+        "logits_gbs": (bench.R + bench.pre_rows) * row_bytes * K / (ms * 1e-3) / 1e9,
+        "accepted_tokens_per_s": world * bench.accepted_per_cycle / N_BUF * K / (ms * 1e-3),
+        "mean_tokens_per_seq_step": bench.accepted_per_cycle / N_BUF / w.batch,
+        "counters": bench.ctx.counters(),
+    }
+    if not args.no_cpu_baseline and world == 1:
+        line["cpu_baseline"] = cpu_baseline(w, seconds=args.cpu_seconds)
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_e2e(bench: Bench, dev, steps: int):
+    """The step with HOST inputs: per step the logits of that step travel from pinned host
+    memory to the device and the step's results travel back, all inside the timed region."""
+    w = bench.w
+    host_pre = bench.pre_bufs[0].cpu().pin_memory()
+    host_ver = bench.ver_bufs[0].cpu().pin_memory()
+    dpre, dver = bench.pre_bufs[0], bench.ver_bufs[0]
+    st = bench.state
+    res_emit = torch.empty(st.emit_ids.shape, dtype=torch.int32).pin_memory()
+    res_n = torch.empty(st.n_emit.shape, dtype=torch.int32).pin_memory()
+    res_tab = torch.empty(bench.pre_out[0]["align_ids"].shape, dtype=torch.int32).pin_memory()
+    h2d = host_pre.numel() * host_pre.element_size() + host_ver.numel() * host_ver.element_size()
+    d2h = (res_emit.numel() + res_n.numel() + res_tab.numel()) * 4
+    bench.restore()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    t0.record()
+    for s in range(steps):
+        bench.restore()
+        dpre.copy_(host_pre, non_blocking=True)
+        dver.copy_(host_ver, non_blocking=True)
+        bench.ctx.align_sample(dpre, bench.pre_ids[0], bench.pre_offs[0], k_extra=K_EXTRA,
+                               outputs=bench.pre_out[0])
+        st.step(dver, 0)
+        res_emit.copy_(st.emit_ids, non_blocking=True)
+        res_n.copy_(st.n_emit, non_blocking=True)
+        res_tab.copy_(bench.pre_out[0]["align_ids"], non_blocking=True)
+    t1.record()
+    torch.cuda.synchronize()
+    bench.restore()
+    return {"ms_per_step": t0.elapsed_time(t1) / steps, "h2d": int(h2d), "d2h": int(d2h)}
+
+
+# --------------------------------------------------------------------------------------
+# CPU legs: the oracle as it stands, on a bounded sample of the same workload
+# --------------------------------------------------------------------------------------
+def oracle_sample(w: synth.Workload, rows: int, threads: int):
+    """Times the oracle on `rows` prefill rows + `rows` verification rows of workload w.
+    Returns seconds."""
+    import oracle
+    L = min(w.prompt_len, rows)
+    n_seq = max(1, rows // L)
+    rows = n_seq * L
+    prompts = [synth.prompt_ids(w, b)[:L] for b in range(n_seq)]
+    ids = torch.cat(prompts)
+    hints = torch.cat([synth.next_token_hints(p) for p in prompts])
+    x = synth.logits(rows, w.vocab, w.torch_dtype, w.recipe, hints, w.seed, chunk_rows=64)
+    d = torch.randint(0, w.vocab, (rows,), generator=synth.generator(w.seed + 5), dtype=torch.int32)
+    xv = synth.logits(rows, w.vocab, w.torch_dtype, w.recipe, d.to(torch.int64), w.seed + 1, chunk_rows=64)
+    xn = xv.view(torch.int16).numpy().view(np.uint16) if w.dtype == "bf16" else xv.numpy()
+    pn = x.view(torch.int16).numpy().view(np.uint16) if w.dtype == "bf16" else x.numpy()
+    offs = np.arange(0, rows + 1, L, dtype=np.int32)
+    coffs = np.arange(0, rows + 1, w.draft_len, dtype=np.int32)
+    if coffs[-1] != rows:
+        coffs = np.append(coffs, rows).astype(np.int32)
+    t0 = time.perf_counter()
+    oracle.align_sample(pn, ids.numpy(), offs, k_extra=K_EXTRA, threads=threads)
+    oracle.verify(xn, d.numpy(), coffs, alpha=ALPHA, beta=BETA, threads=threads)
+    return time.perf_counter() - t0, rows
+
+
+def cpu_baseline(w: synth.Workload, seconds: float = 12.0):
+    import oracle
+    oracle.build()
+    cores = os.cpu_count() or 1
+    t_small, rows_small = oracle_sample(w, 2 * cores, cores)
+    rate = rows_small / t_small
+    rows = int(max(2 * cores, min(4096, rate * seconds)))
+    rows = max(cores, rows // cores * cores)
+    t, rows = oracle_sample(w, rows, cores)
+    return {"value": rows / t, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": "%d prefill rows (alignment sampling) + %d verification rows of %s, "
+                      "OpenMP over rows, %.1f s" % (rows, rows, w.name, t)}
+
+
+def run_reference(args, rank, world):
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    w = synth.workload(args.workload)
+    cores = os.cpu_count() or 1
+    rows = 2 * cores
+    K, W = args.steps, max(args.warmup, 1)
+    budget = 150.0
+    t_probe, rows = oracle_sample(w, rows, cores)
+    # keep the whole run within a few minutes
+    per_step_rows = rows
+    est = t_probe * (K + W)
+    if est > budget:
+        K = max(1, int(budget / t_probe) - W)
+    for _ in range(W):
+        oracle_sample(w, per_step_rows, cores)
+    t0 = time.perf_counter()
+    done = 0
+    for _ in range(K):
+        _, r = oracle_sample(w, per_step_rows, cores)
+        done += r
+    dt = time.perf_counter() - t0
+    value = done / dt
+    sample = ("each step = %d prefill rows + %d verification rows of %s through the oracle "
+              "(input drawing included in the step time)" % (per_step_rows, per_step_rows, w.name))
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world,
+            "steps": K, "warmup": W, "ms_per_step": dt / K * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "vocab": w.vocab, "logits_dtype": w.dtype},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=64)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", type=int, default=4, help="0-based index of the configuration")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (sm_100): there is no CPU fallback; "
+                         "use --impl reference for the CPU oracle")
+    run_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

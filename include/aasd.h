@@ -1,0 +1,290 @@
+/*
+ * aasd.h - C ABI of the B200 draft-and-verify path of Alignment-Augmented Speculative
+ * Decoding (AASD).
+ *
+ * The library covers what surrounds the target model in one decoding step of the method
+ * (Algorithm 1): alignment sampling over the prefill distributions (Sec. 2.3, Sec. 3.2,
+ * Fig. 2), context-aware drafting by longest-suffix lookup (Sec. 3.1), conditional
+ * verification with the entropy-adaptive threshold (Sec. 3.3, Eq. 3-6) including the
+ * prefix rule (Sec. 2.1), and the choice of the longest passing candidate.  The model's
+ * logits are an input.
+ *
+ * Conventions
+ *  - Every tensor pointer is a DEVICE pointer owned by the caller unless a comment says
+ *    HOST.  The library keeps no pointer after the work it enqueued has run.  Output
+ *    pointers inside the *_out structs may be NULL to skip that output.
+ *  - Calls enqueue work on the context's stream and return without synchronising, except
+ *    aasd_poll_status / aasd_get_counters, which synchronise that stream.
+ *  - The return value is an aasd_status.  Errors that the host can see (NULL required
+ *    pointer, bad size, unsupported mode, workspace too small) are returned before
+ *    anything is launched.  Anomalies seen on the device (token id outside the
+ *    vocabulary, NaN or +inf logit, history overflow) set bits in a device status word
+ *    that aasd_poll_status returns and clears; the kernels never trap.
+ *  - Logits are row-major [rows x vocab] with a row stride given in elements; dtype is
+ *    AASD_F32 or AASD_BF16.  Rows whose start is 16-byte aligned take the vectorised path;
+ *    other layouts are handled by a slower scalar path with identical results.
+ *  - Token ids are int32, AASD_NONE (-1) means "no token".  Offsets arrays are CSR.
+ *  - Scratch memory comes from the caller: a workspace of aasd_workspace_bytes() bytes
+ *    that was registered once with aasd_workspace_init().  A workspace must not be shared
+ *    by calls that may overlap on the device.
+ *  - There is no CPU fallback: aasd_create fails with AASD_ERR_NOT_SM100 on a device
+ *    whose compute capability is not 10.x.
+ */
+#ifndef AASD_H
+#define AASD_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define AASD_NONE (-1)
+#define AASD_MAX_EXTRA 4   /* upper bound of k_extra */
+#define AASD_MAX_NGRAM 16  /* upper bound of the key length n */
+
+typedef enum aasd_status {
+    AASD_OK = 0,
+    AASD_ERR_INVALID_ARG = 1,
+    AASD_ERR_BAD_SHAPE = 2,
+    AASD_ERR_BAD_DTYPE = 3,
+    AASD_ERR_WORKSPACE_TOO_SMALL = 4,
+    AASD_ERR_CUDA = 5,
+    AASD_ERR_NOT_SM100 = 6,
+    AASD_ERR_UNSUPPORTED = 7
+} aasd_status;
+
+typedef enum aasd_dtype { AASD_F32 = 0, AASD_BF16 = 1 } aasd_dtype;
+
+/* How the extra tokens of a misaligned position are chosen. */
+typedef enum aasd_align_mode {
+    AASD_ALIGN_TOPK = 0,   /* the tokens ranked above the prompt token (Fig. 2) */
+    AASD_ALIGN_GUMBEL = 1  /* k_extra keyed Gumbel-max draws from the distribution */
+} aasd_align_mode;
+
+typedef enum aasd_verify_mode {
+    AASD_VERIFY_CONDITIONAL = 0,   /* Eq. 4-6 for eligible tokens, strict for the others */
+    AASD_VERIFY_STRICT_GREEDY = 1, /* accept iff draft == argmax (Sec. 2.1) */
+    AASD_VERIFY_STRICT_SAMPLED = 2 /* accept iff draft == the row's keyed sample (Eq. 1) */
+} aasd_verify_mode;
+
+/* Bits of the device status word. */
+#define AASD_STATUS_BAD_ROW 1u        /* a logits row held NaN/+inf or only -inf */
+#define AASD_STATUS_ID_RANGE 2u       /* a token id outside [0, vocab) was ignored */
+#define AASD_STATUS_HIST_OVERFLOW 4u  /* aasd_append dropped tokens: history full */
+#define AASD_STATUS_BAD_OFFSETS 8u    /* a CSR array was not monotone / inconsistent */
+
+/* Bits of a draft token's flag byte (Sec. 3.3, last paragraph). */
+#define AASD_FLAG_CONDITIONAL 1u /* from the input context or alignment sampling */
+#define AASD_FLAG_EXTRA 2u       /* an alignment-sampled alternative */
+
+/* aasd_draft_params.flags */
+#define AASD_DRAFT_MATCH_ALIGN 1u /* the last key token may also match an extra */
+
+typedef struct aasd_ctx aasd_ctx;
+
+typedef struct aasd_counters {
+    uint64_t rows;            /* logits rows processed */
+    uint64_t bad_rows;        /* rows flagged AASD_STATUS_BAD_ROW */
+    uint64_t redo_rows;       /* rows that needed the second, max-referenced pass */
+    uint64_t near_threshold;  /* conditional decisions with |p - (alpha*H+beta)| <= 1e-6 */
+    uint64_t accepted;        /* accepted draft rows (before the prefix rule) */
+    uint64_t sampler_recheck; /* sampled rows whose leading groups were re-scored in fp64 */
+    uint64_t sampler_exact;   /* sampled rows that took the exhaustive fp64 path */
+    uint64_t reserved;
+} aasd_counters;
+
+/* ---- context ------------------------------------------------------------------- */
+
+/* Creates a context on CUDA device `device` whose work goes to `stream` (a cudaStream_t,
+ * NULL = the legacy default stream).  Allocates a small device block for the status word
+ * and counters.  AASD_ERR_NOT_SM100 unless the device is compute capability 10.x. */
+int aasd_create(aasd_ctx** out, int device, void* stream);
+int aasd_destroy(aasd_ctx* ctx);
+int aasd_set_stream(aasd_ctx* ctx, void* stream);
+/* Static string for a status code. */
+const char* aasd_status_str(int status);
+/* Synchronises the stream, returns the device status bits in *bits and clears them. */
+int aasd_poll_status(aasd_ctx* ctx, uint32_t* bits);
+/* Synchronises the stream and copies the running counters to *out (HOST). */
+int aasd_get_counters(aasd_ctx* ctx, aasd_counters* out);
+int aasd_reset_counters(aasd_ctx* ctx);
+/* Number of kernels the context has launched so far (host-side count). */
+uint64_t aasd_launch_count(const aasd_ctx* ctx);
+
+/* Bytes of scratch needed by aasd_align_sample / aasd_verify / aasd_step for at most
+ * max_rows logits rows and max_cands candidates per call. */
+int aasd_workspace_bytes(int64_t max_rows, int64_t max_cands, size_t* bytes);
+/* Registers a 256-byte aligned device buffer of at least aasd_workspace_bytes(max_rows,
+ * max_cands) bytes with the context and clears it (asynchronous).  Required once before
+ * the buffer's first use; the context remembers its layout by address. */
+int aasd_workspace_init(aasd_ctx* ctx, void* workspace, size_t bytes, int64_t max_rows,
+                        int64_t max_cands);
+/* Forgets a registered workspace (the caller frees the memory). */
+int aasd_workspace_release(aasd_ctx* ctx, void* workspace);
+
+/* ---- alignment sampling (Sec. 2.3, Sec. 3.2, Fig. 2) ----------------------------- */
+
+typedef struct aasd_align_params {
+    int32_t vocab;
+    int32_t dtype;          /* aasd_dtype of prefill_logits */
+    int64_t row_stride;     /* elements between consecutive rows, >= vocab */
+    float inv_temperature;  /* logits are multiplied by this before the softmax; > 0 */
+    int32_t k_extra;        /* at most this many extras per position (paper: 2), 0..4 */
+    int32_t mode;           /* aasd_align_mode */
+    uint32_t stream_tag;    /* distinguishes random streams of calls sharing a seed */
+    uint64_t seed;          /* key of the counter-based generator (GUMBEL mode) */
+} aasd_align_params;
+
+typedef struct aasd_align_out {
+    int32_t* align_ids;  /* [n_rows x k_extra] extras of the position after row t, NONE padded */
+    float* align_p;      /* [n_rows x k_extra] their probabilities, 0 padded */
+    int32_t* n_extra;    /* [n_rows] number of extras */
+    float* p_next;       /* [n_rows] probability of the prompt's own next token (0 if none) */
+    int32_t* top1;       /* [n_rows] greedy token of the row (ties: lowest id) */
+    float* entropy;      /* [n_rows] entropy in nats */
+    float* pmax;         /* [n_rows] largest probability */
+    uint8_t* aligned;    /* [n_rows] 1 iff the next prompt token equals top1 (Sec. 2.3) */
+} aasd_align_out;
+
+/* Row t of sequence b (seq_offsets[b] <= t < seq_offsets[b+1], global row index) holds the
+ * distribution of the token after prompt_ids[t]; its "next token" is prompt_ids[t+1], or
+ * NONE on the last row of a sequence.  TOPK mode: the extras are those of the row's
+ * k_extra best tokens (logit descending, ties by lower id) that rank above the next token;
+ * all k_extra of them when there is no next token.  GUMBEL mode: aligned rows get none,
+ * other rows k_extra keyed draws, keeping distinct tokens different from the next token.
+ * n_rows must equal seq_offsets[n_seqs].  A bad row gets NONE/0 everywhere. */
+int aasd_align_sample(aasd_ctx* ctx, const void* prefill_logits, const int32_t* prompt_ids,
+                      const int32_t* seq_offsets, int32_t n_seqs, int64_t n_rows,
+                      const aasd_align_params* params, void* workspace, size_t workspace_bytes,
+                      const aasd_align_out* out);
+
+/* ---- drafting (Sec. 3.1, Algorithm 1) --------------------------------------------- */
+
+typedef struct aasd_draft_params {
+    int32_t n_seqs;
+    int32_t n;          /* longest key (suffix) length, 1..AASD_MAX_NGRAM (paper: 6) */
+    int32_t draft_len;  /* tokens per candidate */
+    int32_t max_cands;  /* candidates per sequence */
+    int32_t k_extra;    /* row width of align_ids (0 = no alignment table) */
+    uint32_t flags;     /* AASD_DRAFT_* */
+} aasd_draft_params;
+
+typedef struct aasd_draft_in {
+    const int32_t* hist_ids;      /* token buffers of all sequences (prompt + generated) */
+    const int32_t* hist_offsets;  /* [n_seqs+1] start of each buffer; the gap is its capacity */
+    const int32_t* hist_len;      /* [n_seqs] tokens currently held */
+    const int32_t* prompt_len;    /* [n_seqs] how many of them are the input context */
+    const int32_t* align_ids;     /* [rows x k_extra] table from aasd_align_sample, or NULL */
+    const int32_t* align_n;       /* [rows] extras per table row */
+    const int32_t* align_row_offsets; /* [n_seqs] table row of each sequence's first position */
+    const int32_t* recent_ids;    /* [n_seqs x n] key tokens, the last recent_len[b] ... */
+    const int32_t* recent_len;    /* ... of which end the current sequence (0..n) */
+} aasd_draft_in;
+
+typedef struct aasd_draft_out {
+    int32_t* draft_ids;    /* [n_seqs x max_cands x draft_len], NONE padded */
+    uint8_t* draft_flags;  /* same shape, AASD_FLAG_* */
+    int32_t* cand_len;     /* [n_seqs x max_cands] */
+    int32_t* cand_pos;     /* [n_seqs x max_cands] match position of the candidate's main */
+    int32_t* n_cands;      /* [n_seqs] */
+    int32_t* match_len;    /* [n_seqs] length of the matched key, 0 = no match */
+} aasd_draft_out;
+
+/* For every sequence: the longest k <= min(n, recent_len) such that the last k key tokens
+ * occur in the history at a place that has a continuation; the places (index right after
+ * the occurrence) in descending order, at most max_cands, each continued by up to
+ * draft_len history tokens; then, while slots remain, alternatives in (main, depth i,
+ * extra slot) order made of the main's first i tokens plus one alignment extra of position
+ * p+i (extras of prompt position q are table row align_row_offsets[b] + q - 1).  All
+ * outputs are required. */
+int aasd_draft(aasd_ctx* ctx, const aasd_draft_in* in, const aasd_draft_params* params,
+               const aasd_draft_out* out);
+
+/* ---- conditional verification (Sec. 3.3, Eq. 3-6; prefix rule Sec. 2.1) ----------- */
+
+typedef struct aasd_verify_params {
+    int32_t vocab;
+    int32_t dtype;
+    int64_t row_stride;
+    float alpha;            /* entropy factor of Eq. 5 (paper: 0.1 / 0.2) */
+    float beta;             /* base threshold of Eq. 5 (paper: 0.1) */
+    float inv_temperature;
+    int32_t mode;           /* aasd_verify_mode */
+    int32_t rows_per_cand;  /* used when cand_offsets == NULL: every candidate has this many rows */
+    uint32_t step;          /* decoding step, part of the sampler's counter */
+    uint64_t seed;
+} aasd_verify_params;
+
+typedef struct aasd_verify_out {
+    float* p_draft;       /* [n_rows] probability of the draft token (0 for NONE) */
+    float* entropy;       /* [n_rows] H of Eq. 5, nats */
+    float* pmax;          /* [n_rows] Delta of Eq. 6 */
+    int32_t* argmax;      /* [n_rows] */
+    float* threshold;     /* [n_rows] delta = min(alpha*H + beta, Delta) */
+    uint8_t* accept;      /* [n_rows] accept bit of the row on its own */
+    int32_t* sampled;     /* [n_rows] the row's keyed sample (STRICT_SAMPLED), else NONE */
+    int32_t* accept_len;  /* [n_cands] leading accepted rows */
+    int32_t* next_token;  /* [n_cands] target's own token at the first rejected row, or NONE */
+} aasd_verify_out;
+
+/* Row r holds the target distribution that judges draft_ids[r].  draft_flags may be NULL
+ * (every row conditional-eligible).  A row is accepted when: CONDITIONAL mode and its flag
+ * has AASD_FLAG_CONDITIONAL: p_draft >= min(alpha*H + beta, Delta), where a draft logit
+ * equal to the row maximum always passes; otherwise draft == the target's own token
+ * (argmax, or the keyed sample in STRICT_SAMPLED).  NONE never passes.  Candidates are CSR
+ * row ranges (cand_offsets[n_cands+1], or regular when NULL); accept_len counts the leading
+ * accepted rows and next_token is the target's own token of row accept_len if the
+ * candidate has such a row.  n_rows must equal the last offset. */
+int aasd_verify(aasd_ctx* ctx, const void* target_logits, const int32_t* draft_ids,
+                const uint8_t* draft_flags, const int32_t* cand_offsets, int32_t n_cands,
+                int64_t n_rows, const aasd_verify_params* params, void* workspace,
+                size_t workspace_bytes, const aasd_verify_out* out);
+
+/* ---- longest passing candidate (Sec. 3.3) and history update (Algorithm 1) -------- */
+
+/* Per sequence, the candidate with the largest accept_len (ties: lowest index); emits its
+ * accepted draft ids followed by its next_token when that is not NONE.  Candidates of
+ * sequence b are seq_cand_offsets[b] .. seq_cand_offsets[b+1] (or cands_per_seq each when
+ * the pointer is NULL); candidate c's draft ids start at cand_offsets[c] (or
+ * c * rows_per_cand when NULL).  emit_ids is [n_seqs x emit_stride], NONE padded. */
+int aasd_select(aasd_ctx* ctx, const int32_t* accept_len, const int32_t* next_token,
+                const int32_t* draft_ids, const int32_t* cand_offsets, int32_t rows_per_cand,
+                const int32_t* seq_cand_offsets, int32_t cands_per_seq, int32_t n_seqs,
+                int32_t emit_stride, int32_t* best_cand, int32_t* n_emit, int32_t* emit_ids);
+
+/* Appends the emitted tokens to each history in place (q <- q + y).  Tokens that do not
+ * fit the buffer (hist_offsets[b+1] - hist_offsets[b]) are dropped and
+ * AASD_STATUS_HIST_OVERFLOW is raised. */
+int aasd_append(aasd_ctx* ctx, int32_t* hist_ids, const int32_t* hist_offsets,
+                int32_t* hist_len, const int32_t* emit_ids, const int32_t* n_emit,
+                int32_t n_seqs, int32_t emit_stride);
+
+/* ---- one decoding step of the batched driver (Algorithm 1, loop body) ------------- */
+
+typedef struct aasd_step_args {
+    aasd_draft_in draft_in;        /* recent_ids == NULL: the key is the history's own tail */
+    aasd_draft_params draft;
+    aasd_draft_out draft_out;
+    const void* target_logits;     /* [n_seqs*max_cands*draft_len x vocab], row = (b, c, i) */
+    aasd_verify_params verify;     /* rows_per_cand is set to draft_len by the call */
+    aasd_verify_out verify_out;
+    int32_t* hist_ids;             /* the same buffer as draft_in.hist_ids, writable */
+    int32_t* hist_len;             /* the same array as draft_in.hist_len, writable */
+    int32_t* best_cand;            /* [n_seqs] */
+    int32_t* n_emit;               /* [n_seqs] */
+    int32_t* emit_ids;             /* [n_seqs x (draft_len+1)] */
+} aasd_step_args;
+
+/* draft -> verify -> select -> append on the context's stream.  The target logits of the
+ * step must already be resident: row (b, c, i) judges token i of candidate c of sequence
+ * b, so the caller's model runs on the candidates of the previous aasd_draft of the same
+ * state (the benchmark replays logits drawn for exactly those candidates). */
+int aasd_step(aasd_ctx* ctx, const aasd_step_args* args, void* workspace,
+              size_t workspace_bytes);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AASD_H */

@@ -307,6 +307,9 @@ int oracle_align_sample(const void* logits, int dtype, const int32_t* prompt_ids
                             for (int q = 0; q < k; ++q) taken |= (best[q] == (int32_t)i);
                             if (taken) continue;
                             double y = X.at(t, i) * invT;
+                            // a masked token (probability 0) cannot be drawn from the
+                            // distribution, so it is never an extra
+                            if (y == -std::numeric_limits<double>::infinity()) continue;
                             if (pick < 0 || ahead(y, i, py, pick)) {
                                 pick = i;
                                 py = y;

@@ -1,0 +1,392 @@
+// Host side of the C ABI declared in include/aasd.h: argument checks, workspace layout,
+// launch geometry.  Every step of the path runs in the kernels of aasd_rows.cuh and
+// aasd_tokens.cuh; nothing here computes on the host.
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <new>
+
+#include "../../include/aasd.h"
+#include "aasd_rows.cuh"
+#include "aasd_tokens.cuh"
+
+using namespace aasd;
+
+namespace {
+
+struct WorkspaceLayout {
+    size_t bytes;
+    int64_t max_rows, max_cands;
+    size_t off_partials, off_row_tickets, off_cand_tickets, off_row_accept, off_row_own, off_next;
+};
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+WorkspaceLayout make_layout(int64_t max_rows, int64_t max_cands) {
+    WorkspaceLayout L{};
+    L.max_rows = max_rows;
+    L.max_cands = max_cands;
+    size_t o = 0;
+    L.off_partials = o;
+    o = align_up(o + sizeof(RowPartial) * (size_t)kPartialSlots, 256);
+    L.off_row_tickets = o;
+    o = align_up(o + 4 * (size_t)max_rows, 256);
+    L.off_cand_tickets = o;
+    o = align_up(o + 4 * (size_t)max_cands, 256);
+    L.off_row_accept = o;
+    o = align_up(o + (size_t)max_rows, 256);
+    L.off_row_own = o;
+    o = align_up(o + 4 * (size_t)max_rows, 256);
+    L.off_next = o;
+    o = align_up(o + 4 * (size_t)max_rows, 256);
+    L.bytes = o;
+    return L;
+}
+
+}  // namespace
+
+struct aasd_ctx {
+    int device;
+    cudaStream_t stream;
+    int sm_count;
+    DeviceState* state;
+    uint64_t launches;
+    std::map<void*, WorkspaceLayout> workspaces;
+};
+
+namespace {
+
+#define AASD_CUDA(call)                                   \
+    do {                                                  \
+        cudaError_t e__ = (call);                         \
+        if (e__ != cudaSuccess) return AASD_ERR_CUDA;     \
+    } while (0)
+
+int after_launch(aasd_ctx* ctx, int n) {
+    ctx->launches += (uint64_t)n;
+    return cudaGetLastError() == cudaSuccess ? AASD_OK : AASD_ERR_CUDA;
+}
+
+const WorkspaceLayout* find_workspace(aasd_ctx* ctx, void* ws, size_t bytes, int64_t rows, int64_t cands,
+                                      int* err) {
+    auto it = ctx->workspaces.find(ws);
+    if (ws == nullptr || it == ctx->workspaces.end()) {
+        *err = AASD_ERR_INVALID_ARG;
+        return nullptr;
+    }
+    const WorkspaceLayout& L = it->second;
+    if (bytes < L.bytes || rows > L.max_rows || cands > L.max_cands) {
+        *err = AASD_ERR_WORKSPACE_TOO_SMALL;
+        return nullptr;
+    }
+    return &L;
+}
+
+// Geometry of a streaming launch: how many CTAs share a row and which path the rows take.
+int plan_rows(aasd_ctx* ctx, RowJob& job, const void* logits, int dtype, int vocab, int64_t row_stride,
+              int64_t n_rows, float inv_temperature, char* ws, const WorkspaceLayout& L) {
+    if (dtype != AASD_F32 && dtype != AASD_BF16) return AASD_ERR_BAD_DTYPE;
+    if (vocab <= 0 || row_stride < vocab || n_rows < 0) return AASD_ERR_BAD_SHAPE;
+    if (!(inv_temperature > 0.f) || !(inv_temperature <= 3.0e38f)) return AASD_ERR_INVALID_ARG;
+    if (n_rows > 0 && logits == nullptr) return AASD_ERR_INVALID_ARG;
+    const int esize = dtype == AASD_F32 ? 4 : 2;
+    const int vec = 16 / esize;
+    if (((uintptr_t)logits % esize) != 0) return AASD_ERR_INVALID_ARG;
+    job.logits = logits;
+    job.row_stride = row_stride;
+    job.n_rows = n_rows;
+    job.vocab = vocab;
+    job.vector_ok = ((uintptr_t)logits % 16 == 0) && ((row_stride * esize) % 16 == 0);
+    job.nvec = job.vector_ok ? vocab / vec : 0;
+    job.c1 = inv_temperature * kLog2e;
+    // Fill the machine: aim at eight CTAs per SM, but keep at least one sweep of the CTA
+    // per chunk and stay within the partial-record slots of the workspace.
+    int chunks = 1;
+    if (n_rows > 0) {
+        const int64_t target = (int64_t)ctx->sm_count * 8;
+        const int64_t units = job.vector_ok ? job.nvec : vocab;
+        int64_t c = target / n_rows;
+        c = c < 1 ? 1 : c;
+        c = c > kMaxSplit ? kMaxSplit : c;
+        int64_t by_size = units / (2 * kThreads);
+        c = c > by_size ? (by_size < 1 ? 1 : by_size) : c;
+        while (c > 1 && c * n_rows > kPartialSlots) --c;
+        chunks = (int)c;
+    }
+    job.chunks = chunks;
+    int per = (job.nvec + chunks - 1) / chunks;
+    per = (per + 7) / 8 * 8;
+    job.vec_per_chunk = per;
+    job.partials = reinterpret_cast<RowPartial*>(ws + L.off_partials);
+    job.row_tickets = reinterpret_cast<unsigned int*>(ws + L.off_row_tickets);
+    job.state = ctx->state;
+    return AASD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* aasd_status_str(int status) {
+    switch (status) {
+        case AASD_OK: return "ok";
+        case AASD_ERR_INVALID_ARG: return "invalid argument";
+        case AASD_ERR_BAD_SHAPE: return "bad shape";
+        case AASD_ERR_BAD_DTYPE: return "bad dtype";
+        case AASD_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case AASD_ERR_CUDA: return "CUDA error";
+        case AASD_ERR_NOT_SM100: return "device is not compute capability 10.x";
+        case AASD_ERR_UNSUPPORTED: return "unsupported mode";
+        default: return "unknown status";
+    }
+}
+
+int aasd_create(aasd_ctx** out, int device, void* stream) {
+    if (out == nullptr) return AASD_ERR_INVALID_ARG;
+    *out = nullptr;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) return AASD_ERR_CUDA;
+    cudaDeviceProp prop;
+    AASD_CUDA(cudaGetDeviceProperties(&prop, device));
+    if (prop.major != 10) return AASD_ERR_NOT_SM100;
+    AASD_CUDA(cudaSetDevice(device));
+    aasd_ctx* ctx = new (std::nothrow) aasd_ctx();
+    if (ctx == nullptr) return AASD_ERR_CUDA;
+    ctx->device = device;
+    ctx->stream = static_cast<cudaStream_t>(stream);
+    ctx->sm_count = prop.multiProcessorCount;
+    ctx->launches = 0;
+    if (cudaMalloc(&ctx->state, sizeof(DeviceState)) != cudaSuccess) {
+        delete ctx;
+        return AASD_ERR_CUDA;
+    }
+    if (cudaMemset(ctx->state, 0, sizeof(DeviceState)) != cudaSuccess) {
+        cudaFree(ctx->state);
+        delete ctx;
+        return AASD_ERR_CUDA;
+    }
+    *out = ctx;
+    return AASD_OK;
+}
+
+int aasd_destroy(aasd_ctx* ctx) {
+    if (ctx == nullptr) return AASD_OK;
+    cudaStreamSynchronize(ctx->stream);
+    cudaFree(ctx->state);
+    delete ctx;
+    return AASD_OK;
+}
+
+int aasd_set_stream(aasd_ctx* ctx, void* stream) {
+    if (ctx == nullptr) return AASD_ERR_INVALID_ARG;
+    ctx->stream = static_cast<cudaStream_t>(stream);
+    return AASD_OK;
+}
+
+int aasd_poll_status(aasd_ctx* ctx, uint32_t* bits) {
+    if (ctx == nullptr || bits == nullptr) return AASD_ERR_INVALID_ARG;
+    unsigned int v = 0;
+    AASD_CUDA(cudaMemcpyAsync(&v, &ctx->state->status, 4, cudaMemcpyDeviceToHost, ctx->stream));
+    AASD_CUDA(cudaMemsetAsync(&ctx->state->status, 0, 4, ctx->stream));
+    AASD_CUDA(cudaStreamSynchronize(ctx->stream));
+    *bits = v;
+    return AASD_OK;
+}
+
+int aasd_get_counters(aasd_ctx* ctx, aasd_counters* out) {
+    if (ctx == nullptr || out == nullptr) return AASD_ERR_INVALID_ARG;
+    static_assert(sizeof(aasd_counters) == 64, "counter block layout");
+    AASD_CUDA(cudaMemcpyAsync(out, ctx->state->counters, 64, cudaMemcpyDeviceToHost, ctx->stream));
+    AASD_CUDA(cudaStreamSynchronize(ctx->stream));
+    return AASD_OK;
+}
+
+int aasd_reset_counters(aasd_ctx* ctx) {
+    if (ctx == nullptr) return AASD_ERR_INVALID_ARG;
+    AASD_CUDA(cudaMemsetAsync(ctx->state->counters, 0, 64, ctx->stream));
+    return AASD_OK;
+}
+
+uint64_t aasd_launch_count(const aasd_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int aasd_workspace_bytes(int64_t max_rows, int64_t max_cands, size_t* bytes) {
+    if (bytes == nullptr || max_rows < 0 || max_cands < 0) return AASD_ERR_INVALID_ARG;
+    *bytes = make_layout(max_rows, max_cands).bytes;
+    return AASD_OK;
+}
+
+int aasd_workspace_init(aasd_ctx* ctx, void* workspace, size_t bytes, int64_t max_rows, int64_t max_cands) {
+    if (ctx == nullptr || workspace == nullptr || max_rows < 0 || max_cands < 0) return AASD_ERR_INVALID_ARG;
+    if ((uintptr_t)workspace % 256 != 0) return AASD_ERR_INVALID_ARG;
+    WorkspaceLayout L = make_layout(max_rows, max_cands);
+    if (bytes < L.bytes) return AASD_ERR_WORKSPACE_TOO_SMALL;
+    AASD_CUDA(cudaMemsetAsync(workspace, 0, L.bytes, ctx->stream));
+    ctx->workspaces[workspace] = L;
+    return AASD_OK;
+}
+
+int aasd_workspace_release(aasd_ctx* ctx, void* workspace) {
+    if (ctx == nullptr) return AASD_ERR_INVALID_ARG;
+    ctx->workspaces.erase(workspace);
+    return AASD_OK;
+}
+
+int aasd_align_sample(aasd_ctx* ctx, const void* prefill_logits, const int32_t* prompt_ids,
+                      const int32_t* seq_offsets, int32_t n_seqs, int64_t n_rows,
+                      const aasd_align_params* p, void* workspace, size_t workspace_bytes,
+                      const aasd_align_out* out) {
+    if (ctx == nullptr || p == nullptr || out == nullptr) return AASD_ERR_INVALID_ARG;
+    if (n_seqs < 0 || n_rows < 0) return AASD_ERR_BAD_SHAPE;
+    if (p->k_extra < 0 || p->k_extra > AASD_MAX_EXTRA) return AASD_ERR_INVALID_ARG;
+    if (p->mode != AASD_ALIGN_TOPK && p->mode != AASD_ALIGN_GUMBEL) return AASD_ERR_INVALID_ARG;
+    if (p->mode == AASD_ALIGN_GUMBEL) return AASD_ERR_UNSUPPORTED;
+    if (n_rows > 0 && (prompt_ids == nullptr || seq_offsets == nullptr || n_seqs == 0)) return AASD_ERR_INVALID_ARG;
+    int err = AASD_OK;
+    const WorkspaceLayout* L = find_workspace(ctx, workspace, workspace_bytes, n_rows, 0, &err);
+    if (L == nullptr) return err;
+    char* ws = static_cast<char*>(workspace);
+    AlignArgs a{};
+    err = plan_rows(ctx, a.job, prefill_logits, p->dtype, p->vocab, p->row_stride, n_rows, p->inv_temperature, ws, *L);
+    if (err != AASD_OK) return err;
+    if (n_rows == 0) return AASD_OK;
+    if (n_rows * (int64_t)a.job.chunks > 0x7FFFFFFFLL) return AASD_ERR_BAD_SHAPE;
+    a.prompt_ids = prompt_ids;
+    a.seq_offsets = seq_offsets;
+    a.n_seqs = n_seqs;
+    a.k_extra = p->k_extra;
+    a.mode = p->mode;
+    a.next_ids = reinterpret_cast<int32_t*>(ws + L->off_next);
+    a.out = *out;
+    AASD_CUDA(cudaSetDevice(ctx->device));
+    align_next_kernel<<<(unsigned int)((n_rows + 255) / 256), 256, 0, ctx->stream>>>(a);
+    const unsigned int grid = (unsigned int)(n_rows * a.job.chunks);
+    const int K = p->k_extra <= 1 ? 1 : (p->k_extra == 2 ? 2 : 4);
+    if (p->dtype == AASD_F32) {
+        if (K == 1) align_kernel<AASD_F32, 1><<<grid, kThreads, 0, ctx->stream>>>(a);
+        else if (K == 2) align_kernel<AASD_F32, 2><<<grid, kThreads, 0, ctx->stream>>>(a);
+        else align_kernel<AASD_F32, 4><<<grid, kThreads, 0, ctx->stream>>>(a);
+    } else {
+        if (K == 1) align_kernel<AASD_BF16, 1><<<grid, kThreads, 0, ctx->stream>>>(a);
+        else if (K == 2) align_kernel<AASD_BF16, 2><<<grid, kThreads, 0, ctx->stream>>>(a);
+        else align_kernel<AASD_BF16, 4><<<grid, kThreads, 0, ctx->stream>>>(a);
+    }
+    return after_launch(ctx, 2);
+}
+
+int aasd_draft(aasd_ctx* ctx, const aasd_draft_in* in, const aasd_draft_params* p, const aasd_draft_out* out) {
+    if (ctx == nullptr || in == nullptr || p == nullptr || out == nullptr) return AASD_ERR_INVALID_ARG;
+    if (p->n_seqs < 0) return AASD_ERR_BAD_SHAPE;
+    if (p->n < 1 || p->n > AASD_MAX_NGRAM || p->draft_len < 1 || p->max_cands < 1 || p->max_cands > kMaxCands)
+        return AASD_ERR_INVALID_ARG;
+    if (p->k_extra < 0 || p->k_extra > AASD_MAX_EXTRA) return AASD_ERR_INVALID_ARG;
+    if (p->n_seqs == 0) return AASD_OK;
+    if (!in->hist_ids || !in->hist_offsets || !in->hist_len || !in->prompt_len) return AASD_ERR_INVALID_ARG;
+    if (in->recent_ids && !in->recent_len) return AASD_ERR_INVALID_ARG;
+    if (in->align_ids && p->k_extra > 0 && (!in->align_n || !in->align_row_offsets)) return AASD_ERR_INVALID_ARG;
+    if (!out->draft_ids || !out->draft_flags || !out->cand_len || !out->cand_pos || !out->n_cands || !out->match_len)
+        return AASD_ERR_INVALID_ARG;
+    DraftArgs a{*in, *p, *out, ctx->state};
+    AASD_CUDA(cudaSetDevice(ctx->device));
+    draft_kernel<<<(unsigned int)p->n_seqs, kThreads, 0, ctx->stream>>>(a);
+    return after_launch(ctx, 1);
+}
+
+int aasd_verify(aasd_ctx* ctx, const void* target_logits, const int32_t* draft_ids,
+                const uint8_t* draft_flags, const int32_t* cand_offsets, int32_t n_cands,
+                int64_t n_rows, const aasd_verify_params* p, void* workspace, size_t workspace_bytes,
+                const aasd_verify_out* out) {
+    if (ctx == nullptr || p == nullptr || out == nullptr) return AASD_ERR_INVALID_ARG;
+    if (n_cands < 0 || n_rows < 0) return AASD_ERR_BAD_SHAPE;
+    if (p->mode < AASD_VERIFY_CONDITIONAL || p->mode > AASD_VERIFY_STRICT_SAMPLED) return AASD_ERR_INVALID_ARG;
+    if (p->mode == AASD_VERIFY_STRICT_SAMPLED) return AASD_ERR_UNSUPPORTED;
+    if (!(p->alpha >= 0.f) || !(p->beta >= 0.f)) return AASD_ERR_INVALID_ARG;
+    if (cand_offsets == nullptr) {
+        if (p->rows_per_cand < 1 || (int64_t)n_cands * p->rows_per_cand != n_rows) return AASD_ERR_BAD_SHAPE;
+    }
+    if (n_rows > 0 && (draft_ids == nullptr || n_cands == 0)) return AASD_ERR_INVALID_ARG;
+    int err = AASD_OK;
+    const WorkspaceLayout* L = find_workspace(ctx, workspace, workspace_bytes, n_rows, n_cands, &err);
+    if (L == nullptr) return err;
+    char* ws = static_cast<char*>(workspace);
+    VerifyArgs a{};
+    err = plan_rows(ctx, a.job, target_logits, p->dtype, p->vocab, p->row_stride, n_rows, p->inv_temperature, ws, *L);
+    if (err != AASD_OK) return err;
+    if (n_rows * (int64_t)a.job.chunks > 0x7FFFFFFFLL) return AASD_ERR_BAD_SHAPE;
+    a.draft_ids = draft_ids;
+    a.draft_flags = draft_flags;
+    a.cand_offsets = cand_offsets;
+    a.n_cands = n_cands;
+    a.rows_per_cand = p->rows_per_cand;
+    a.alpha = p->alpha;
+    a.beta = p->beta;
+    a.mode = p->mode;
+    a.cand_tickets = reinterpret_cast<unsigned int*>(ws + L->off_cand_tickets);
+    a.row_accept = reinterpret_cast<uint8_t*>(ws + L->off_row_accept);
+    a.row_own = reinterpret_cast<int32_t*>(ws + L->off_row_own);
+    a.out = *out;
+    AASD_CUDA(cudaSetDevice(ctx->device));
+    if (n_rows == 0) {
+        if (n_cands == 0) return AASD_OK;
+        verify_empty_kernel<<<(unsigned int)((n_cands + 255) / 256), 256, 0, ctx->stream>>>(a);
+        return after_launch(ctx, 1);
+    }
+    const unsigned int grid = (unsigned int)(n_rows * a.job.chunks);
+    if (p->dtype == AASD_F32) verify_kernel<AASD_F32><<<grid, kThreads, 0, ctx->stream>>>(a);
+    else verify_kernel<AASD_BF16><<<grid, kThreads, 0, ctx->stream>>>(a);
+    return after_launch(ctx, 1);
+}
+
+int aasd_select(aasd_ctx* ctx, const int32_t* accept_len, const int32_t* next_token,
+                const int32_t* draft_ids, const int32_t* cand_offsets, int32_t rows_per_cand,
+                const int32_t* seq_cand_offsets, int32_t cands_per_seq, int32_t n_seqs,
+                int32_t emit_stride, int32_t* best_cand, int32_t* n_emit, int32_t* emit_ids) {
+    if (ctx == nullptr) return AASD_ERR_INVALID_ARG;
+    if (n_seqs < 0 || emit_stride < 1) return AASD_ERR_BAD_SHAPE;
+    if (n_seqs == 0) return AASD_OK;
+    if (!accept_len || !next_token || !draft_ids || !best_cand || !n_emit || !emit_ids) return AASD_ERR_INVALID_ARG;
+    if (!cand_offsets && rows_per_cand < 1) return AASD_ERR_BAD_SHAPE;
+    if (!seq_cand_offsets && cands_per_seq < 0) return AASD_ERR_BAD_SHAPE;
+    SelectArgs a{accept_len, next_token, draft_ids, cand_offsets, rows_per_cand, seq_cand_offsets,
+                 cands_per_seq, n_seqs, emit_stride, best_cand, n_emit, emit_ids};
+    AASD_CUDA(cudaSetDevice(ctx->device));
+    select_kernel<<<(unsigned int)((n_seqs + 127) / 128), 128, 0, ctx->stream>>>(a);
+    return after_launch(ctx, 1);
+}
+
+int aasd_append(aasd_ctx* ctx, int32_t* hist_ids, const int32_t* hist_offsets, int32_t* hist_len,
+                const int32_t* emit_ids, const int32_t* n_emit, int32_t n_seqs, int32_t emit_stride) {
+    if (ctx == nullptr) return AASD_ERR_INVALID_ARG;
+    if (n_seqs < 0 || emit_stride < 1) return AASD_ERR_BAD_SHAPE;
+    if (n_seqs == 0) return AASD_OK;
+    if (!hist_ids || !hist_offsets || !hist_len || !emit_ids || !n_emit) return AASD_ERR_INVALID_ARG;
+    AppendArgs a{hist_ids, hist_offsets, hist_len, emit_ids, n_emit, n_seqs, emit_stride, ctx->state};
+    AASD_CUDA(cudaSetDevice(ctx->device));
+    append_kernel<<<(unsigned int)((n_seqs + 127) / 128), 128, 0, ctx->stream>>>(a);
+    return after_launch(ctx, 1);
+}
+
+int aasd_step(aasd_ctx* ctx, const aasd_step_args* s, void* workspace, size_t workspace_bytes) {
+    if (ctx == nullptr || s == nullptr) return AASD_ERR_INVALID_ARG;
+    const aasd_draft_params& dp = s->draft;
+    if (!s->hist_ids || !s->hist_len || !s->best_cand || !s->n_emit || !s->emit_ids) return AASD_ERR_INVALID_ARG;
+    if (!s->verify_out.accept_len || !s->verify_out.next_token) return AASD_ERR_INVALID_ARG;
+    int err = aasd_draft(ctx, &s->draft_in, &dp, &s->draft_out);
+    if (err != AASD_OK) return err;
+    aasd_verify_params vp = s->verify;
+    vp.rows_per_cand = dp.draft_len;
+    const int32_t n_cands = dp.n_seqs * dp.max_cands;
+    const int64_t n_rows = (int64_t)n_cands * dp.draft_len;
+    err = aasd_verify(ctx, s->target_logits, s->draft_out.draft_ids, s->draft_out.draft_flags, nullptr, n_cands,
+                      n_rows, &vp, workspace, workspace_bytes, &s->verify_out);
+    if (err != AASD_OK) return err;
+    err = aasd_select(ctx, s->verify_out.accept_len, s->verify_out.next_token, s->draft_out.draft_ids, nullptr,
+                      dp.draft_len, nullptr, dp.max_cands, dp.n_seqs, dp.draft_len + 1, s->best_cand, s->n_emit,
+                      s->emit_ids);
+    if (err != AASD_OK) return err;
+    return aasd_append(ctx, s->hist_ids, s->draft_in.hist_offsets, s->hist_len, s->emit_ids, s->n_emit, dp.n_seqs,
+                       dp.draft_len + 1);
+}
+
+}  // extern "C"

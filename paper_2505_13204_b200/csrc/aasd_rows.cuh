@@ -1,0 +1,494 @@
+// Streaming kernels over logits rows: alignment sampling and conditional verification.
+#pragma once
+
+#include "aasd_device.cuh"
+
+namespace aasd {
+
+// What every row kernel needs to know about the logits block and the scratch memory.
+struct RowJob {
+    const void* logits;
+    int64_t row_stride;     // elements
+    int64_t n_rows;
+    int vocab;
+    int vector_ok;          // rows are 16-byte aligned: take the vector path
+    int nvec;               // whole vectors per row (vector path)
+    int chunks;             // CTAs per row
+    int vec_per_chunk;      // vectors per chunk (multiple of 8)
+    float c1;               // inv_temperature * log2(e)
+    RowPartial* partials;   // [n_rows x chunks] when chunks > 1
+    unsigned int* row_tickets;
+    DeviceState* state;
+};
+
+struct BlockScratch {
+    double S[kWarps];
+    double A[kWarps];
+    u64 keys[kWarps][kMaxK];
+    RowPartial merged;
+    int flag;
+};
+
+template <int DT>
+__device__ __forceinline__ const char* row_pointer(const RowJob& job, int64_t row) {
+    return static_cast<const char*>(job.logits) + row * job.row_stride * (int64_t)Elt<DT>::kSize;
+}
+
+// Provisional reference of a row: the hinted token's logit (the draft token / the prompt's
+// next token, very often the row maximum) and the first few entries.  Any finite value is
+// valid; a good one keeps the exponents small.
+template <int DT>
+__device__ __forceinline__ float provisional_ref(const char* row, int vocab, int hint) {
+    float r = -CUDART_INF_F;
+    const int n = vocab < 4 ? vocab : 4;
+    for (int i = 0; i < n; ++i) r = fmaxf(r, Elt<DT>::load(row, i));
+    if (hint >= 0) r = fmaxf(r, Elt<DT>::load(row, hint));
+    if (!(fabsf(r) <= 3.0e38f)) r = 0.f;   // NaN, +-inf
+    return r;
+}
+
+// Streams vectors [vbeg, vend) of a row plus scalar elements [sbeg, send) and leaves the
+// CTA-wide result in sc.merged (valid for every thread after the closing barrier).
+template <int DT, int K, bool SAFE>
+__device__ void block_row_pass(const char* row, int vbeg, int vend, int sbeg, int send, float c1,
+                               float neg_refc, BlockScratch& sc) {
+    constexpr int kVec = Elt<DT>::kVec;
+    const int tid = threadIdx.x;
+    const int lane = tid & 31, warp = tid >> 5;
+    RowAccumulator<DT, K, SAFE> acc;
+    acc.init();
+
+    const uint4* vrow = reinterpret_cast<const uint4*>(row);
+    int v = vbeg + tid;
+    for (; v + 3 * kThreads < vend; v += 4 * kThreads) {
+        uint4 q0 = load_stream16(vrow + v);
+        uint4 q1 = load_stream16(vrow + v + kThreads);
+        uint4 q2 = load_stream16(vrow + v + 2 * kThreads);
+        uint4 q3 = load_stream16(vrow + v + 3 * kThreads);
+        acc.add_vector(q0, v, c1, neg_refc);
+        acc.add_vector(q1, v + kThreads, c1, neg_refc);
+        acc.add_vector(q2, v + 2 * kThreads, c1, neg_refc);
+        acc.add_vector(q3, v + 3 * kThreads, c1, neg_refc);
+    }
+    for (; v < vend; v += kThreads) {
+        uint4 q = load_stream16(vrow + v);
+        acc.add_vector(q, v, c1, neg_refc);
+    }
+
+    // the thread's best tokens: they lie inside its K best vectors
+    u64 ek[K];
+#pragma unroll
+    for (int j = 0; j < K; ++j) ek[j] = 0;
+#pragma unroll
+    for (int j = 0; j < K; ++j) {
+        if (acc.best_vec[j] >= 0) {
+            uint4 q = __ldg(vrow + acc.best_vec[j]);
+            float x[kVec];
+            Elt<DT>::unpack(q, x);
+#pragma unroll
+            for (int i = 0; i < kVec; ++i)
+                if (x[i] > -CUDART_INF_F) key_insert<K>(ek, make_key(x[i], acc.best_vec[j] * kVec + i));
+        }
+    }
+    double S, A;
+    acc.totals(S, A);
+    // scalar part: the ragged tail of a vectorised row, or a whole unaligned row
+    {
+        float s = 0.f, a = 0.f;
+        for (int i = sbeg + tid; i < send; i += kThreads) {
+            float xv = Elt<DT>::load(row, i);
+            acc.add_scalar(xv, c1, neg_refc, s, a);
+            if (xv > -CUDART_INF_F) key_insert<K>(ek, make_key(xv, i));
+        }
+        S += (double)s;
+        A += (double)a;
+    }
+
+    S = warp_sum_f64(S);
+    A = warp_sum_f64(A);
+#pragma unroll
+    for (int r = 0; r < K; ++r) {
+        u64 m = warp_max_u64(ek[0]);
+        if (lane == 0) sc.keys[warp][r] = m;
+        if (m != 0 && ek[0] == m) {
+#pragma unroll
+            for (int j = 0; j + 1 < K; ++j) ek[j] = ek[j + 1];
+            ek[K - 1] = 0;
+        }
+    }
+    if (lane == 0) {
+        sc.S[warp] = S;
+        sc.A[warp] = A;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        double s = lane < kWarps ? sc.S[lane] : 0.0;
+        double a = lane < kWarps ? sc.A[lane] : 0.0;
+        s = warp_sum_f64(s);
+        a = warp_sum_f64(a);
+        u64 k = 0;
+        if (lane < kWarps * K) k = sc.keys[lane / K][lane % K];
+#pragma unroll
+        for (int r = 0; r < K; ++r) {
+            u64 m = warp_max_u64(k);
+            if (lane == 0) sc.merged.key[r] = m;
+            if (m != 0 && k == m) k = 0;
+        }
+        if (lane == 0) {
+            sc.merged.S = s;
+            sc.merged.A = a;
+#pragma unroll
+            for (int r = K; r < kMaxK; ++r) sc.merged.key[r] = 0;
+        }
+    }
+    __syncthreads();
+}
+
+// Whole-row driver used by both kernels.  Returns true in the one CTA that holds the
+// finished row (every CTA when chunks == 1); sc.merged then holds the row's sums and best
+// tokens.  The exponents behind the sums are fma(x, c1, neg_refc) when `centered` is false
+// and (x - max) * c1 (with neg_refc = -max) when the second pass ran.
+template <int DT, int K>
+__device__ bool row_reduce(const RowJob& job, int64_t row, int chunk, int hint, const char* rowp,
+                           float& neg_refc, bool& centered, BlockScratch& sc) {
+    centered = false;
+    constexpr int kVec = Elt<DT>::kVec;
+    const int tid = threadIdx.x;
+    const int V = job.vocab;
+    const float c1 = job.c1;
+    neg_refc = -(provisional_ref<DT>(rowp, V, hint) * c1);
+
+    int vbeg = 0, vend = 0, sbeg = 0, send = 0;
+    if (job.vector_ok) {
+        vbeg = chunk * job.vec_per_chunk;
+        vend = min(job.nvec, vbeg + job.vec_per_chunk);
+        if (vbeg > vend) vbeg = vend;
+        if (chunk == 0) {
+            sbeg = job.nvec * kVec;
+            send = V;
+        }
+    } else {
+        // unaligned layout: split the elements themselves
+        int per = (V + job.chunks - 1) / job.chunks;
+        sbeg = min(V, chunk * per);
+        send = min(V, sbeg + per);
+    }
+    block_row_pass<DT, K, false>(rowp, vbeg, vend, sbeg, send, c1, neg_refc, sc);
+
+    if (job.chunks > 1) {
+        RowPartial* slots = job.partials + row * job.chunks;
+        if (tid == 0) {
+            slots[chunk] = sc.merged;
+            __threadfence();
+            unsigned int t = atomicAdd(&job.row_tickets[row], 1u);
+            sc.flag = (t == (unsigned int)job.chunks - 1);
+        }
+        __syncthreads();
+        if (!sc.flag) return false;
+        __threadfence();
+        if (tid < 32) {
+            double s = 0.0, a = 0.0;
+            u64 k[K];
+#pragma unroll
+            for (int j = 0; j < K; ++j) k[j] = 0;
+            if (tid < job.chunks) {
+                const RowPartial* p = slots + tid;
+                s = __ldcg(&p->S);
+                a = __ldcg(&p->A);
+#pragma unroll
+                for (int j = 0; j < K; ++j) k[j] = __ldcg(&p->key[j]);
+            }
+            s = warp_sum_f64(s);
+            a = warp_sum_f64(a);
+#pragma unroll
+            for (int r = 0; r < K; ++r) {
+                u64 m = warp_max_u64(k[0]);
+                if (tid == 0) sc.merged.key[r] = m;
+                if (m != 0 && k[0] == m) {
+#pragma unroll
+                    for (int j = 0; j + 1 < K; ++j) k[j] = k[j + 1];
+                    k[K - 1] = 0;
+                }
+            }
+            if (tid == 0) {
+                sc.merged.S = s;
+                sc.merged.A = a;
+                job.row_tickets[row] = 0;   // ready for the next call
+            }
+        }
+        __syncthreads();
+    }
+
+    // Second pass when the provisional reference was too far from the maximum for the
+    // fp32 sums to be trusted (overflow, underflow to zero, -inf entries, large shift).
+    const u64 k0 = sc.merged.key[0];
+    const float m = key_value(k0);
+    bool redo = false;
+    if (k0 != 0 && fabsf(m) <= 3.0e38f) {
+        const double S = sc.merged.S, A = sc.merged.A;
+        const float shift = fmaf(m, c1, neg_refc);
+        redo = !(S > 0.0) || !(S <= 1.0e300) || !(fabs(A) <= 1.0e300) || !(fabsf(shift) <= kRedoShift);
+    }
+    __syncthreads();   // everyone has read sc.merged
+    if (redo) {
+        neg_refc = -m;
+        centered = true;
+        int vb = 0, ve = 0, sb = 0, se = V;
+        if (job.vector_ok) {
+            ve = job.nvec;
+            sb = job.nvec * kVec;
+        }
+        block_row_pass<DT, K, true>(rowp, vb, ve, sb, se, c1, neg_refc, sc);
+        if (tid == 0) atomicAdd(&job.state->counters[kCntRedo], 1ull);
+    }
+    return true;
+}
+
+// Scalars of a finished row (Eq. 5-6), evaluated in double by one thread.
+struct RowFinal {
+    bool bad;
+    float m;        // raw logit of the best token
+    int top1;
+    double S;       // relative to the reference
+    double H;       // nats
+    double pmax;
+    double c1;
+    double neg_refc;
+    bool centered;
+    // probability of a token from its raw logit, with the exponent the streaming pass used
+    __device__ double prob(float x) const {
+        const double t = centered ? ((double)x + neg_refc) * c1 : (double)x * c1 + neg_refc;
+        return exp2(t) / S;
+    }
+};
+
+__device__ inline RowFinal finish_row(const RowPartial& p, float c1, float neg_refc, bool centered) {
+    RowFinal f;
+    f.c1 = (double)c1;
+    f.neg_refc = (double)neg_refc;
+    f.centered = centered;
+    f.m = key_value(p.key[0]);
+    f.top1 = key_id(p.key[0]);
+    f.S = p.S;
+    f.bad = (p.key[0] == 0) || !(fabsf(f.m) <= 3.0e38f) || !(p.S > 0.0) || !(p.S <= 1.0e300) ||
+            !(fabs(p.A) <= 1.0e300);
+    if (f.bad) {
+        f.top1 = AASD_NONE;
+        f.H = 0.0;
+        f.pmax = 0.0;
+        f.S = 1.0;
+        return f;
+    }
+    f.H = log(p.S) - kLn2 * (p.A / p.S);
+    f.pmax = f.prob(f.m);
+    return f;
+}
+
+// ---- conditional verification -----------------------------------------------------------------
+
+struct VerifyArgs {
+    RowJob job;
+    const int32_t* draft_ids;
+    const uint8_t* draft_flags;
+    const int32_t* cand_offsets;   // NULL: regular candidates of rows_per_cand rows
+    int n_cands;
+    int rows_per_cand;
+    float alpha, beta;
+    int mode;
+    unsigned int* cand_tickets;
+    uint8_t* row_accept;           // scratch [n_rows]
+    int32_t* row_own;              // scratch [n_rows]
+    aasd_verify_out out;
+};
+
+// Candidate that owns row r: the last c with cand_offsets[c] <= r.
+__device__ inline int find_segment(const int32_t* offsets, int n, int64_t r) {
+    int lo = 0, hi = n;   // invariant: offsets[lo] <= r < offsets[hi]
+    while (hi - lo > 1) {
+        int mid = (lo + hi) >> 1;
+        if ((int64_t)__ldg(offsets + mid) <= r) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+__device__ inline void write_empty_candidate(const VerifyArgs& a, int c) {
+    if (a.out.accept_len) a.out.accept_len[c] = 0;
+    if (a.out.next_token) a.out.next_token[c] = AASD_NONE;
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kThreads) verify_kernel(const VerifyArgs a) {
+    __shared__ BlockScratch sc;
+    const RowJob& job = a.job;
+    const int64_t row = blockIdx.x / job.chunks;
+    const int chunk = blockIdx.x % job.chunks;
+    const char* rowp = row_pointer<DT>(job, row);
+    int d = __ldg(a.draft_ids + row);
+    const bool d_ok = d >= 0 && d < job.vocab;
+    float neg_refc;
+    bool centered;
+    if (!row_reduce<DT, 1>(job, row, chunk, d_ok ? d : -1, rowp, neg_refc, centered, sc)) return;
+    if (threadIdx.x != 0) return;
+
+    const RowFinal f = finish_row(sc.merged, job.c1, neg_refc, centered);
+    const unsigned int flag = a.draft_flags ? a.draft_flags[row] : AASD_FLAG_CONDITIONAL;
+    const double lin = (double)a.alpha * f.H + (double)a.beta;
+    const double thr = f.bad ? 0.0 : fmin(lin, f.pmax);
+    const int own = f.top1;   // NONE on a bad row
+    double pd = 0.0;
+    bool acc = false, near = false;
+    unsigned int status = 0;
+    if (f.bad) status |= AASD_STATUS_BAD_ROW;
+    if (!d_ok && d != AASD_NONE) status |= AASD_STATUS_ID_RANGE;
+    if (d_ok && !f.bad) {
+        const float xd = Elt<DT>::load(rowp, d);
+        pd = f.prob(xd);
+        if (a.mode == AASD_VERIFY_CONDITIONAL && (flag & AASD_FLAG_CONDITIONAL)) {
+            const bool at_max = (xd == f.m);
+            acc = at_max || (pd >= lin);
+            near = !at_max && fabs(pd - lin) <= 1.0e-6;
+        } else {
+            acc = (d == own);
+        }
+    }
+    if (a.out.p_draft) a.out.p_draft[row] = (float)pd;
+    if (a.out.entropy) a.out.entropy[row] = (float)f.H;
+    if (a.out.pmax) a.out.pmax[row] = (float)f.pmax;
+    if (a.out.argmax) a.out.argmax[row] = f.top1;
+    if (a.out.threshold) a.out.threshold[row] = (float)thr;
+    if (a.out.accept) a.out.accept[row] = acc ? 1 : 0;
+    if (a.out.sampled) a.out.sampled[row] = AASD_NONE;
+    a.row_accept[row] = acc ? 1 : 0;
+    a.row_own[row] = own;
+    atomicAdd(&job.state->counters[kCntRows], 1ull);
+    if (f.bad) atomicAdd(&job.state->counters[kCntBad], 1ull);
+    if (near) atomicAdd(&job.state->counters[kCntNear], 1ull);
+    if (acc) atomicAdd(&job.state->counters[kCntAccepted], 1ull);
+    if (status) atomicOr(&job.state->status, status);
+
+    // The CTA that finishes the last row of a candidate applies the prefix rule.
+    int c;
+    int64_t lo, hi;
+    if (a.cand_offsets) {
+        c = find_segment(a.cand_offsets, a.n_cands, row);
+        lo = a.cand_offsets[c];
+        hi = a.cand_offsets[c + 1];
+        // empty candidates own no row: their neighbours write their (empty) result
+        if (row == lo)
+            for (int e = c - 1; e >= 0 && a.cand_offsets[e] == a.cand_offsets[e + 1]; --e)
+                write_empty_candidate(a, e);
+        if (row == job.n_rows - 1)
+            for (int e = c + 1; e < a.n_cands; ++e) write_empty_candidate(a, e);
+    } else {
+        c = (int)(row / a.rows_per_cand);
+        lo = (int64_t)c * a.rows_per_cand;
+        hi = lo + a.rows_per_cand;
+    }
+    __threadfence();
+    const unsigned int t = atomicAdd(&a.cand_tickets[c], 1u);
+    if (t != (unsigned int)(hi - lo) - 1u) return;
+    __threadfence();
+    a.cand_tickets[c] = 0;
+    int n = 0;
+    while (lo + n < hi && __ldcg(a.row_accept + lo + n)) ++n;
+    if (a.out.accept_len) a.out.accept_len[c] = n;
+    if (a.out.next_token) a.out.next_token[c] = (lo + n < hi) ? __ldcg(a.row_own + lo + n) : AASD_NONE;
+}
+
+// Candidates of a call without rows.
+__global__ void verify_empty_kernel(const VerifyArgs a) {
+    int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c < a.n_cands) write_empty_candidate(a, c);
+}
+
+// ---- alignment sampling ---------------------------------------------------------------------------
+
+struct AlignArgs {
+    RowJob job;
+    const int32_t* prompt_ids;
+    const int32_t* seq_offsets;
+    int n_seqs;
+    int k_extra;
+    int mode;
+    int32_t* next_ids;   // scratch [n_rows]: the prompt's next token of every row
+    aasd_align_out out;
+};
+
+// next_ids[t] = prompt_ids[t+1] unless t is the last row of its sequence.
+__global__ void align_next_kernel(const AlignArgs a) {
+    int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= a.job.n_rows) return;
+    int b = find_segment(a.seq_offsets, a.n_seqs, t);
+    int nxt = AASD_NONE;
+    if (t + 1 < (int64_t)a.seq_offsets[b + 1]) {
+        nxt = a.prompt_ids[t + 1];
+        if (nxt < 0 || nxt >= a.job.vocab) {
+            nxt = AASD_NONE;
+            atomicOr(&a.job.state->status, AASD_STATUS_ID_RANGE);
+        }
+    }
+    a.next_ids[t] = nxt;
+}
+
+template <int DT, int K>
+__global__ void __launch_bounds__(kThreads) align_kernel(const AlignArgs a) {
+    __shared__ BlockScratch sc;
+    const RowJob& job = a.job;
+    const int64_t row = blockIdx.x / job.chunks;
+    const int chunk = blockIdx.x % job.chunks;
+    const char* rowp = row_pointer<DT>(job, row);
+    const int next = __ldg(a.next_ids + row);
+    float neg_refc;
+    bool centered;
+    if (!row_reduce<DT, K>(job, row, chunk, next, rowp, neg_refc, centered, sc)) return;
+    if (threadIdx.x != 0) return;
+
+    const RowFinal f = finish_row(sc.merged, job.c1, neg_refc, centered);
+    const int KE = a.k_extra;
+    int ids[kMaxK];
+    float ps[kMaxK];
+    int n = 0;
+    for (int j = 0; j < kMaxK; ++j) {
+        ids[j] = AASD_NONE;
+        ps[j] = 0.f;
+    }
+    double pn = 0.0;
+    bool aligned = false;
+    if (!f.bad) {
+        float xn = 0.f;
+        if (next != AASD_NONE) {
+            xn = Elt<DT>::load(rowp, next);
+            pn = f.prob(xn);
+            aligned = (next == f.top1);
+        }
+        // the listed tokens that rank above the next token (Fig. 2)
+        for (int j = 0; j < KE && j < K; ++j) {
+            const u64 k = sc.merged.key[j];
+            if (k == 0) break;
+            const float xv = key_value(k);
+            const int id = key_id(k);
+            if (next == AASD_NONE || xv > xn || (xv == xn && id < next)) {
+                ids[n] = id;
+                ps[n] = (float)f.prob(xv);
+                ++n;
+            }
+        }
+    }
+    for (int j = 0; j < KE; ++j) {
+        if (a.out.align_ids) a.out.align_ids[row * KE + j] = ids[j];
+        if (a.out.align_p) a.out.align_p[row * KE + j] = ps[j];
+    }
+    if (a.out.n_extra) a.out.n_extra[row] = n;
+    if (a.out.p_next) a.out.p_next[row] = (float)pn;
+    if (a.out.top1) a.out.top1[row] = f.top1;
+    if (a.out.entropy) a.out.entropy[row] = (float)f.H;
+    if (a.out.pmax) a.out.pmax[row] = (float)f.pmax;
+    if (a.out.aligned) a.out.aligned[row] = aligned ? 1 : 0;
+    atomicAdd(&job.state->counters[kCntRows], 1ull);
+    if (f.bad) {
+        atomicAdd(&job.state->counters[kCntBad], 1ull);
+        atomicOr(&job.state->status, AASD_STATUS_BAD_ROW);
+    }
+}
+
+}  // namespace aasd

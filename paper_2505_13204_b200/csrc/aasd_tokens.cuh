@@ -1,0 +1,229 @@
+// Integer kernels on token buffers: suffix-match drafting, candidate selection, append.
+#pragma once
+
+#include "aasd_device.cuh"
+
+namespace aasd {
+
+constexpr int kMaxCands = 64;   // candidates per sequence a draft call can emit
+
+struct DraftArgs {
+    aasd_draft_in in;
+    aasd_draft_params p;
+    aasd_draft_out out;
+    DeviceState* state;
+};
+
+// One CTA per sequence.  Every history position p (the index right after a possible key
+// occurrence) is scored by the length of the common suffix of hist[..p) and the key; the
+// positions that reach the best length are the lookup result of Algorithm 1's dictionary
+// for the longest key that has one (Sec. 3.1: longer keys first).  Warp ballots compact the
+// hits in descending position order.
+__global__ void __launch_bounds__(kThreads) draft_kernel(const DraftArgs a) {
+    __shared__ int s_rec[AASD_MAX_NGRAM];
+    __shared__ int s_pos[kMaxCands];
+    __shared__ int s_warp[kWarps];
+    __shared__ int s_count;
+    __shared__ int s_kstar;
+
+    const int b = blockIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int n = a.p.n, draft_len = a.p.draft_len, max_cands = a.p.max_cands, K = a.p.k_extra;
+    const int32_t* h = a.in.hist_ids + a.in.hist_offsets[b];
+    const int len = a.in.hist_len[b];
+    const int plen = min(a.in.prompt_len[b], len);
+    const bool have_align = a.in.align_ids != nullptr && a.in.align_n != nullptr && K > 0;
+    const bool match_align = have_align && (a.p.flags & AASD_DRAFT_MATCH_ALIGN);
+    const int64_t arow0 = have_align ? (int64_t)a.in.align_row_offsets[b] : 0;
+
+    int rl;
+    if (a.in.recent_ids) {
+        rl = max(0, min(n, a.in.recent_len[b]));
+        if (tid < rl) s_rec[tid] = a.in.recent_ids[(int64_t)b * n + tid];
+    } else {
+        rl = min(n, len);
+        if (tid < rl) s_rec[tid] = h[len - rl + tid];
+    }
+    if (tid == 0) {
+        s_count = 0;
+        s_kstar = 0;
+    }
+    __syncthreads();
+
+    auto n_ext = [&](int q) -> int {
+        if (!have_align || q < 1 || q >= plen) return 0;
+        return min(K, max(0, a.in.align_n[arow0 + q - 1]));
+    };
+    auto ext = [&](int q, int s) -> int { return a.in.align_ids[(arow0 + q - 1) * K + s]; };
+    auto match_len_at = [&](int p) -> int {
+        const int lim = min(min(n, p), rl);
+        int m = 0;
+        for (int j = 1; j <= lim; ++j) {
+            const int q = p - j, want = s_rec[rl - j];
+            bool ok = (h[q] == want);
+            if (!ok && j == 1 && match_align) {
+                const int ne = n_ext(q);
+                for (int s = 0; s < ne; ++s) ok |= (ext(q, s) == want);
+            }
+            if (!ok) break;
+            m = j;
+        }
+        return m;
+    };
+
+    // pass 1: the longest key that occurs at a place with a continuation (p < len)
+    int best = 0;
+    for (int p = 1 + tid; p < len; p += kThreads) best = max(best, match_len_at(p));
+    best = __reduce_max_sync(0xFFFFFFFFu, best);
+    if (lane == 0 && best > 0) atomicMax(&s_kstar, best);
+    __syncthreads();
+    const int kstar = s_kstar;
+
+    // pass 2: its places, most recent first
+    if (kstar > 0) {
+        for (int base = len - 1; base >= 1; base -= kThreads) {
+            const int p = base - tid;
+            const bool hit = p >= 1 && match_len_at(p) == kstar;
+            const unsigned int bal = __ballot_sync(0xFFFFFFFFu, hit);
+            if (lane == 0) s_warp[warp] = __popc(bal);
+            __syncthreads();
+            int before = s_count;
+            for (int w = 0; w < warp; ++w) before += s_warp[w];
+            const int rank = before + __popc(bal & ((1u << lane) - 1u));
+            if (hit && rank < max_cands) s_pos[rank] = p;
+            __syncthreads();
+            if (tid == 0) {
+                int tot = s_count;
+                for (int w = 0; w < kWarps; ++w) tot += s_warp[w];
+                s_count = tot;
+            }
+            __syncthreads();
+            if (s_count >= max_cands) break;
+        }
+    }
+    const int n_main = min(s_count, max_cands);
+
+    int32_t* d_ids = a.out.draft_ids + (int64_t)b * max_cands * draft_len;
+    uint8_t* d_fl = a.out.draft_flags + (int64_t)b * max_cands * draft_len;
+    int32_t* c_len = a.out.cand_len + (int64_t)b * max_cands;
+    int32_t* c_pos = a.out.cand_pos + (int64_t)b * max_cands;
+    for (int i = tid; i < max_cands * draft_len; i += kThreads) {
+        const int c = i / draft_len, j = i % draft_len;
+        int tok = AASD_NONE;
+        unsigned int fl = 0;
+        if (c < n_main) {
+            const int q = s_pos[c] + j;
+            if (q < len) {
+                tok = h[q];
+                fl = (q < plen) ? AASD_FLAG_CONDITIONAL : 0u;
+            }
+        }
+        d_ids[i] = tok;
+        d_fl[i] = (uint8_t)fl;
+    }
+    for (int c = tid; c < max_cands; c += kThreads) {
+        c_len[c] = c < n_main ? min(draft_len, len - s_pos[c]) : 0;
+        c_pos[c] = c < n_main ? s_pos[c] : AASD_NONE;
+    }
+    __syncthreads();
+
+    // alternatives: a main's prefix plus one alignment-sampled token (Sec. 3.2), in
+    // (main, depth, extra slot) order while slots remain
+    if (tid == 0) {
+        int total = n_main;
+        for (int c = 0; c < n_main && total < max_cands; ++c) {
+            const int p = s_pos[c];
+            const int L = min(draft_len, len - p);
+            for (int i = 0; i < L && total < max_cands; ++i) {
+                const int ne = n_ext(p + i);
+                for (int s = 0; s < ne && total < max_cands; ++s) {
+                    const int slot = total++;
+                    for (int q = 0; q < i; ++q) {
+                        d_ids[slot * draft_len + q] = d_ids[c * draft_len + q];
+                        d_fl[slot * draft_len + q] = d_fl[c * draft_len + q];
+                    }
+                    d_ids[slot * draft_len + i] = ext(p + i, s);
+                    d_fl[slot * draft_len + i] = AASD_FLAG_CONDITIONAL | AASD_FLAG_EXTRA;
+                    c_len[slot] = i + 1;
+                    c_pos[slot] = p;
+                }
+            }
+        }
+        a.out.n_cands[b] = total;
+        a.out.match_len[b] = kstar;
+    }
+}
+
+struct SelectArgs {
+    const int32_t* accept_len;
+    const int32_t* next_token;
+    const int32_t* draft_ids;
+    const int32_t* cand_offsets;
+    int rows_per_cand;
+    const int32_t* seq_cand_offsets;
+    int cands_per_seq;
+    int n_seqs;
+    int emit_stride;
+    int32_t* best_cand;
+    int32_t* n_emit;
+    int32_t* emit_ids;
+};
+
+// Longest passing candidate per sequence (Sec. 3.3), ties to the lowest index.
+__global__ void select_kernel(const SelectArgs a) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= a.n_seqs) return;
+    const int lo = a.seq_cand_offsets ? a.seq_cand_offsets[b] : b * a.cands_per_seq;
+    const int hi = a.seq_cand_offsets ? a.seq_cand_offsets[b + 1] : lo + a.cands_per_seq;
+    int best = AASD_NONE, best_a = -1;
+    for (int c = lo; c < hi; ++c) {
+        const int v = a.accept_len[c];
+        if (v > best_a) {
+            best_a = v;
+            best = c;
+        }
+    }
+    int32_t* e = a.emit_ids + (int64_t)b * a.emit_stride;
+    int ne = 0;
+    if (best != AASD_NONE) {
+        const int64_t d0 = a.cand_offsets ? (int64_t)a.cand_offsets[best] : (int64_t)best * a.rows_per_cand;
+        for (int i = 0; i < best_a && ne < a.emit_stride; ++i) e[ne++] = a.draft_ids[d0 + i];
+        const int nt = a.next_token[best];
+        if (nt != AASD_NONE && ne < a.emit_stride) e[ne++] = nt;
+    }
+    for (int i = ne; i < a.emit_stride; ++i) e[i] = AASD_NONE;
+    a.best_cand[b] = best;
+    a.n_emit[b] = ne;
+}
+
+struct AppendArgs {
+    int32_t* hist_ids;
+    const int32_t* hist_offsets;
+    int32_t* hist_len;
+    const int32_t* emit_ids;
+    const int32_t* n_emit;
+    int n_seqs;
+    int emit_stride;
+    DeviceState* state;
+};
+
+// q <- q + y (Algorithm 1), in place, clipped at the buffer's capacity.
+__global__ void append_kernel(const AppendArgs a) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= a.n_seqs) return;
+    const int off = a.hist_offsets[b];
+    const int cap = a.hist_offsets[b + 1] - off;
+    int len = a.hist_len[b];
+    const int ne = min(a.n_emit[b], a.emit_stride);
+    for (int i = 0; i < ne; ++i) {
+        if (len >= cap) {
+            atomicOr(&a.state->status, AASD_STATUS_HIST_OVERFLOW);
+            break;
+        }
+        a.hist_ids[off + len] = a.emit_ids[(int64_t)b * a.emit_stride + i];
+        ++len;
+    }
+    a.hist_len[b] = len;
+}
+
+}  // namespace aasd

@@ -119,12 +119,14 @@ def prompt_ids(w: Workload, seq: int, device="cpu") -> torch.Tensor:
 
 
 def logits(rows: int, vocab: int, dtype: torch.dtype, recipe: LogitRecipe, hint_ids,
-           seed: int, device="cpu", chunk_rows: int = 2048, out=None) -> torch.Tensor:
+           seed: int, device="cpu", chunk_rows: int = 2048, out=None, noise=None) -> torch.Tensor:
     """[rows x vocab] logits drawn by ``recipe``.
 
     ``hint_ids`` (int tensor [rows], or None) names the token that takes the row's spike;
     rows whose hint is negative take it on a random token.  The generator lives on
     ``device``, so CPU and CUDA draws differ; a test draws once and copies.
+    ``noise(lo, n)`` may supply the standard-normal block of rows lo..lo+n (fp32) instead
+    of fresh draws (see NoiseBank).
     """
     g = generator(seed, device)
     if out is None:
@@ -135,7 +137,10 @@ def logits(rows: int, vocab: int, dtype: torch.dtype, recipe: LogitRecipe, hint_
     r = recipe
     for lo in range(0, rows, chunk_rows):
         n = min(chunk_rows, rows - lo)
-        x = torch.randn((n, vocab), generator=g, device=device, dtype=torch.float32)
+        if noise is None:
+            x = torch.randn((n, vocab), generator=g, device=device, dtype=torch.float32)
+        else:
+            x = noise(lo, n)
         x.mul_(r.sigma)
         u_kind = torch.rand((n,), generator=g, device=device)
         u_spike = torch.rand((n,), generator=g, device=device)
@@ -179,3 +184,32 @@ def recent_window(ids: torch.Tensor, n: int, seed: int) -> torch.Tensor:
     L = ids.numel()
     s = int(torch.randint(0, max(1, L - n), (), generator=g).item())
     return ids[s:s + n].clone()
+
+
+class NoiseBank:
+    """A block of standard-normal noise drawn once and re-used under cyclic shifts.
+
+    Drawing tens of billions of normals dominates the set-up of the large workloads, so
+    the benchmark draws ``rows x vocab`` of them once and gives block ``k`` the bank rolled
+    by a block-dependent offset along both axes.  Every row of every block is still an
+    i.i.d. standard-normal vector; rows of different blocks are shifted copies of one
+    another, which no step of the method can notice (rows are processed independently).
+    """
+
+    def __init__(self, rows: int, vocab: int, seed: int, device):
+        g = generator(seed, device)
+        self.rows, self.vocab = rows, vocab
+        self.bank = torch.empty((rows, vocab), dtype=torch.bfloat16, device=device)
+        for lo in range(0, rows, 1024):
+            n = min(1024, rows - lo)
+            self.bank[lo:lo + n] = torch.randn((n, vocab), generator=g, device=device,
+                                               dtype=torch.float32).to(torch.bfloat16)
+
+    def block(self, k: int):
+        """noise callable of block ``k`` for ``logits(..., noise=...)``."""
+        dr, dv = (k * 977) % self.rows, (k * 7919 + 13) % self.vocab
+
+        def fn(lo, n):
+            idx = (torch.arange(lo, lo + n, device=self.bank.device) + dr) % self.rows
+            return torch.roll(self.bank[idx], shifts=dv, dims=1).float()
+        return fn

@@ -1,0 +1,216 @@
+"""GPU parity of the streaming kernels (aasd_verify, aasd_align_sample) with the oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2505_13204_b200 import binding, synth
+from parity import F32, check_align, check_verify, cpu, to_oracle
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = binding.Context()
+    yield c
+    c.close()
+
+
+def _make_logits(rows, V, dtype, seed, hints, recipe=None, stride=None):
+    recipe = recipe or synth.LogitRecipe(sigma=2.5, p_hint=0.6, p_random=0.2, spike_lo=4, spike_hi=12)
+    x = synth.logits(rows, V, dtype, recipe, hints, seed, device="cpu")
+    if stride is not None and stride != V:
+        buf = torch.zeros((rows, stride), dtype=dtype)
+        buf[:, :V] = x
+        x = buf[:, :V]
+    return x
+
+
+def _random_csr(rng, rows, with_empty=True):
+    offs = [0]
+    while offs[-1] < rows:
+        step = int(rng.integers(0 if with_empty else 1, 9))
+        offs.append(min(rows, offs[-1] + step))
+    if with_empty:
+        offs += [rows, rows]
+    return np.asarray(offs, np.int32)
+
+
+def _to_dev(x):
+    """Copies a (possibly strided) CPU tensor to the GPU keeping its row stride."""
+    base = x._base if x._base is not None else x
+    d = base.cuda()
+    return d[:, :x.shape[1]] if d.shape != x.shape else d
+
+
+CASES = [
+    # (V, dtype, stride, rows): aligned vector path, ragged tail, unaligned scalar path,
+    # several sweeps and several chunks per row
+    (1000, torch.float32, None, 70),
+    (1003, torch.float32, 1004, 40),       # 16-byte aligned rows with a 3-element tail
+    (1003, torch.float32, None, 40),       # odd stride: scalar path
+    (1000, torch.bfloat16, None, 70),
+    (1001, torch.bfloat16, 1008, 40),
+    (1001, torch.bfloat16, None, 40),
+    (32000, torch.float32, None, 24),
+    (128256, torch.bfloat16, None, 20),
+    (152064, torch.bfloat16, None, 12),
+    (40, torch.float32, None, 30),
+    (5, torch.bfloat16, None, 9),
+]
+
+
+@pytest.mark.parametrize("V,dtype,stride,rows", CASES)
+@pytest.mark.parametrize("mode", [binding.VERIFY_CONDITIONAL, binding.VERIFY_STRICT_GREEDY])
+def test_verify_parity(ctx, V, dtype, stride, rows, mode):
+    rng = np.random.default_rng(V + rows)
+    d = rng.integers(0, V, rows).astype(np.int32)
+    x = _make_logits(rows, V, dtype, 100 + V, torch.as_tensor(d, dtype=torch.int64), stride=stride)
+    # a third of the drafts are the true argmax, some are sentinels or out of range
+    top = np.argmax(x.float().numpy(), axis=1)
+    pick = rng.random(rows)
+    d = np.where(pick < 0.35, top, d).astype(np.int32)
+    d[pick > 0.95] = -1
+    if rows > 10:
+        d[3] = V + 5
+    flags = rng.integers(0, 4, rows).astype(np.uint8)
+    offs = _random_csr(rng, rows)
+    alpha, beta = F32(0.1), F32(0.05)
+    ref = oracle.verify(to_oracle(x), d, offs, draft_flags=flags, alpha=alpha, beta=beta, mode=mode)
+    xd = _to_dev(x)
+    got = ctx.verify(xd, torch.as_tensor(d).cuda(), torch.as_tensor(offs).cuda(),
+                     draft_flags=torch.as_tensor(flags).cuda(), alpha=alpha, beta=beta, mode=mode)
+    got["sampled"] = None
+    check_verify(got, ref, offs, dtype)
+    st = ctx.poll_status()
+    assert bool(st & binding.STATUS_ID_RANGE) == (rows > 10)
+    assert not (st & binding.STATUS_BAD_ROW)
+    # a second run on the same workspace gives the same bytes (tickets reset themselves)
+    again = ctx.verify(xd, torch.as_tensor(d).cuda(), torch.as_tensor(offs).cuda(),
+                       draft_flags=torch.as_tensor(flags).cuda(), alpha=alpha, beta=beta, mode=mode)
+    for k in ("accept", "accept_len", "next_token", "argmax", "p_draft", "entropy"):
+        assert torch.equal(got[k], again[k]), k
+    ctx.poll_status()
+
+
+@pytest.mark.parametrize("V,dtype,stride,rows", CASES)
+@pytest.mark.parametrize("K", [0, 1, 2, 3, 4])
+def test_align_parity(ctx, V, dtype, stride, rows, K):
+    if V > 40000 and K in (0, 3):
+        pytest.skip("large vocabularies run K = 1, 2, 4")
+    rng = np.random.default_rng(7 * V + rows + K)
+    prompt = rng.integers(0, V, rows).astype(np.int32)
+    cut = sorted(set([0, rows] + [int(c) for c in rng.integers(1, rows, 2)]))
+    hints = synth.next_token_hints(torch.as_tensor(prompt))
+    x = _make_logits(rows, V, dtype, 200 + V, hints, stride=stride)
+    if dtype == torch.bfloat16 and V >= 1000:
+        # force exact ties at the top of some rows
+        for r in range(0, rows, 5):
+            a, b = rng.integers(0, V, 2)
+            x[r, a] = x[r, b] = 30.0
+    ref = oracle.align_sample(to_oracle(x), prompt, cut, k_extra=K)
+    got = ctx.align_sample(_to_dev(x), torch.as_tensor(prompt).cuda(), cut, k_extra=K)
+    check_align(got, ref, dtype)
+    assert ctx.poll_status() == 0
+
+
+def test_rows_with_masked_entries_far_maxima_and_bad_rows(ctx):
+    V, rows = 4096, 12
+    rng = np.random.default_rng(3)
+    for dtype in (torch.float32, torch.bfloat16):
+        x = torch.as_tensor(rng.standard_normal((rows, V)) * 2, dtype=torch.float32)
+        x[0, 100:3000] = -float("inf")            # masked vocabulary
+        x[1, :] = -float("inf"); x[1, 77] = 1.0   # a single live token
+        x[2, :] += -3.0e4; x[2, 4000] = 5.0       # maximum far above the first entries
+        x[3, :] *= 30.0                           # wide spread: exponents far below the max
+        x[4, 9] = float("nan")
+        x[5, 9] = float("inf")
+        x[6, :] = -float("inf")
+        x[7, :] = 1.0e30 if dtype == torch.float32 else 1.0e30
+        x[8, :] = -1.0e30
+        x = x.to(dtype)
+        d = np.asarray([5, 77, 1, 1, 9, 9, 0, 3, 3, 2, 2, 2], np.int32)
+        offs = np.arange(rows + 1, dtype=np.int32)
+        ref = oracle.verify(to_oracle(x), d, offs, alpha=F32(0.1), beta=F32(0.1))
+        got = ctx.verify(x.cuda(), torch.as_tensor(d).cuda(), torch.as_tensor(offs).cuda(),
+                         alpha=F32(0.1), beta=F32(0.1))
+        got["sampled"] = None
+        check_verify(got, ref, offs, dtype)
+        assert list(ref["bad"][:9]) == [0, 0, 0, 0, 1, 1, 1, 0, 0]
+        assert ctx.poll_status() & binding.STATUS_BAD_ROW
+        prompt = rng.integers(0, V, rows).astype(np.int32)
+        prompt[2] = 77
+        refa = oracle.align_sample(to_oracle(x), prompt, [0, rows], k_extra=2)
+        gota = ctx.align_sample(x.cuda(), torch.as_tensor(prompt).cuda(), [0, rows], k_extra=2)
+        check_align(gota, refa, dtype)
+        assert ctx.poll_status() & binding.STATUS_BAD_ROW
+    assert ctx.counters()["redo_rows"] > 0
+
+
+def test_temperature_and_thresholds(ctx):
+    V, rows = 2048, 64
+    rng = np.random.default_rng(11)
+    recipe = synth.LogitRecipe(sigma=3.0, p_hint=0.8, spike_lo=2, spike_hi=9)
+    d = rng.integers(0, V, rows).astype(np.int32)
+    x = synth.logits(rows, V, torch.bfloat16, recipe, torch.as_tensor(d, dtype=torch.int64), 5)
+    offs = np.arange(0, rows + 1, 8, dtype=np.int32)
+    for alpha, beta, invT in ((0.0, 0.1, 1.0), (0.2, 0.1, 1 / 1.5), (0.1, 0.0, 2.0), (0.05, 1.0, 0.7)):
+        alpha, beta, invT = F32(alpha), F32(beta), F32(invT)
+        ref = oracle.verify(to_oracle(x), d, offs, alpha=alpha, beta=beta, inv_temperature=invT)
+        got = ctx.verify(x.cuda(), torch.as_tensor(d).cuda(), torch.as_tensor(offs).cuda(),
+                         alpha=alpha, beta=beta, inv_temperature=invT)
+        got["sampled"] = None
+        check_verify(got, ref, offs, torch.bfloat16)
+        gr = ctx.verify(x.cuda(), torch.as_tensor(d).cuda(), None, alpha=alpha, beta=beta,
+                        inv_temperature=invT, rows_per_cand=8)
+        assert torch.equal(gr["accept_len"], got["accept_len"])
+        assert torch.equal(gr["next_token"], got["next_token"])
+    ctx.poll_status()
+
+
+def test_empty_and_degenerate_calls(ctx):
+    V = 64
+    x = torch.zeros((0, V), dtype=torch.float32, device="cuda")
+    offs = torch.zeros(4, dtype=torch.int32, device="cuda")
+    got = ctx.verify(x, torch.zeros(0, dtype=torch.int32, device="cuda"), offs)
+    assert cpu(got["accept_len"]).tolist() == [0, 0, 0]
+    assert cpu(got["next_token"]).tolist() == [-1, -1, -1]
+    out = ctx.align_sample(x, torch.zeros(0, dtype=torch.int32, device="cuda"), [0], k_extra=2)
+    assert out["top1"].numel() == 0
+    # one row, one token
+    x1 = torch.tensor([[2.5]], dtype=torch.float32, device="cuda")
+    got = ctx.verify(x1, torch.zeros(1, dtype=torch.int32, device="cuda"), [0, 1])
+    assert cpu(got["accept"]).tolist() == [1] and cpu(got["pmax"])[0] == pytest.approx(1.0)
+    assert cpu(got["entropy"])[0] == pytest.approx(0.0, abs=1e-7)
+    assert ctx.poll_status() == 0
+
+
+def test_host_side_errors(ctx):
+    x = torch.zeros((4, 64), dtype=torch.float16, device="cuda")
+    d = torch.zeros(4, dtype=torch.int32, device="cuda")
+    with pytest.raises(binding.AasdError) as e:
+        ctx.verify(x, d, [0, 4])
+    assert e.value.code == 3
+    xf = torch.zeros((4, 64), dtype=torch.float32, device="cuda")
+    with pytest.raises(binding.AasdError) as e:
+        ctx.verify(xf, d, [0, 4], alpha=-1.0)
+    assert e.value.code == 1
+    with pytest.raises(binding.AasdError) as e:
+        ctx.verify(xf, d, None, rows_per_cand=3)
+    assert e.value.code == 2
+    with pytest.raises(binding.AasdError) as e:
+        ctx.verify(xf, d, [0, 4], inv_temperature=0.0)
+    assert e.value.code == 1
+    with pytest.raises(binding.AasdError) as e:
+        ctx.align_sample(xf, d, [0, 4], k_extra=5)
+    assert e.value.code == 1
+    # an unregistered workspace is refused before anything is launched
+    import ctypes as C
+    prm = binding.VerifyParams(64, 0, 64, 0.1, 0.1, 1.0, 0, 0, 0, 0)
+    out = binding.VerifyOut()
+    junk = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
+    rc = ctx.lib.aasd_verify(ctx._h, xf.data_ptr(), d.data_ptr(), None,
+                             torch.tensor([0, 4], dtype=torch.int32, device="cuda").data_ptr(), 1, 4,
+                             C.byref(prm), junk.data_ptr(), junk.numel(), C.byref(out))
+    assert rc == 1
