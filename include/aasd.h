@@ -74,6 +74,9 @@ typedef enum aasd_verify_mode {
 #define AASD_STATUS_ID_RANGE 2u       /* a token id outside [0, vocab) was ignored */
 #define AASD_STATUS_HIST_OVERFLOW 4u  /* aasd_append dropped tokens: history full */
 #define AASD_STATUS_BAD_OFFSETS 8u    /* a CSR array was not monotone / inconsistent */
+#define AASD_STATUS_TIMEOUT 16u       /* a bounded wait inside a kernel ran out: the results of
+                                         that call are invalid and the workspace must be
+                                         registered again before its next use */
 
 /* Bits of a draft token's flag byte (Sec. 3.3, last paragraph). */
 #define AASD_FLAG_CONDITIONAL 1u /* from the input context or alignment sampling */

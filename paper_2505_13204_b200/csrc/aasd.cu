@@ -4,12 +4,14 @@
 #include <cuda_runtime.h>
 
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <map>
 #include <new>
 
 #include "../../include/aasd.h"
 #include "aasd_rows.cuh"
+#include "aasd_stream.cuh"
 #include "aasd_tokens.cuh"
 
 using namespace aasd;
@@ -122,6 +124,59 @@ int plan_rows(aasd_ctx* ctx, RowJob& job, const void* logits, int dtype, int voc
     job.partials = reinterpret_cast<RowPartial*>(ws + L.off_partials);
     job.row_tickets = reinterpret_cast<unsigned int*>(ws + L.off_row_tickets);
     job.state = ctx->state;
+    return AASD_OK;
+}
+
+// Geometry of the persistent streaming launch over 16-byte aligned rows.  Work items are
+// (row, piece) pairs handed out round-robin to a grid of two CTAs per SM; rows are cut into
+// pieces (at tile boundaries) only while there are too few rows to keep every CTA busy for
+// several items.
+void plan_stream(aasd_ctx* ctx, StreamJob& sj, const RowJob& job, const int32_t* hint_ids, unsigned int* grid) {
+    sj.row = job;
+    sj.hint_ids = hint_ids;
+    const int64_t row_bytes = (int64_t)job.nvec * 16;
+    const int tiles = (int)((row_bytes + kTileBytes - 1) / kTileBytes);
+    const int64_t slots = (int64_t)ctx->sm_count * 2;
+    int64_t chunks = (6 * slots + job.n_rows - 1) / job.n_rows;
+    if (chunks > kMaxSplit) chunks = kMaxSplit;
+    if (chunks > tiles) chunks = tiles;
+    if (chunks < 1) chunks = 1;
+    if (const char* e = getenv("AASD_STREAM_CHUNKS")) {   // tuning override
+        const long v = atol(e);
+        if (v >= 1) chunks = v > tiles ? tiles : v;
+    }
+    while (chunks > 1 && chunks * job.n_rows > kPartialSlots) --chunks;
+    int per = (int)((tiles + chunks - 1) / chunks);
+    if (per < 1) per = 1;
+    chunks = tiles > 0 ? (tiles + per - 1) / per : 1;
+    sj.tiles_per_row = tiles;
+    sj.tiles_per_chunk = per;
+    sj.row.chunks = (int)chunks;
+    sj.n_items = job.n_rows * chunks;
+    *grid = (unsigned int)(sj.n_items < slots ? sj.n_items : slots);
+}
+
+template <class Kernel>
+int enable_stream_smem(Kernel kernel) {
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStreamSmemBytes) ==
+                   cudaSuccess
+               ? AASD_OK
+               : AASD_ERR_CUDA;
+}
+
+template <int DT, int K>
+int launch_align_stream(aasd_ctx* ctx, const StreamJob& sj, const AlignArgs& a, unsigned int grid) {
+    auto kernel = stream_kernel<DT, K, AlignEpilogue<DT>>;
+    if (enable_stream_smem(kernel) != AASD_OK) return AASD_ERR_CUDA;
+    kernel<<<grid, kStreamThreads, kStreamSmemBytes, ctx->stream>>>(sj, a);
+    return AASD_OK;
+}
+
+template <int DT>
+int launch_verify_stream(aasd_ctx* ctx, const StreamJob& sj, const VerifyArgs& a, unsigned int grid) {
+    auto kernel = stream_kernel<DT, 1, VerifyEpilogue<DT>>;
+    if (enable_stream_smem(kernel) != AASD_OK) return AASD_ERR_CUDA;
+    kernel<<<grid, kStreamThreads, kStreamSmemBytes, ctx->stream>>>(sj, a);
     return AASD_OK;
 }
 
@@ -261,8 +316,26 @@ int aasd_align_sample(aasd_ctx* ctx, const void* prefill_logits, const int32_t* 
     a.out = *out;
     AASD_CUDA(cudaSetDevice(ctx->device));
     align_next_kernel<<<(unsigned int)((n_rows + 255) / 256), 256, 0, ctx->stream>>>(a);
-    const unsigned int grid = (unsigned int)(n_rows * a.job.chunks);
     const int K = p->k_extra <= 1 ? 1 : (p->k_extra == 2 ? 2 : 4);
+    if (a.job.vector_ok && a.job.nvec > 0) {
+        // 16-byte aligned rows: persistent TMA-fed streaming kernel
+        StreamJob sj{};
+        unsigned int grid = 0;
+        plan_stream(ctx, sj, a.job, a.next_ids, &grid);
+        a.job = sj.row;
+        int rc;
+        if (p->dtype == AASD_F32)
+            rc = K == 1 ? launch_align_stream<AASD_F32, 1>(ctx, sj, a, grid)
+                        : (K == 2 ? launch_align_stream<AASD_F32, 2>(ctx, sj, a, grid)
+                                  : launch_align_stream<AASD_F32, 4>(ctx, sj, a, grid));
+        else
+            rc = K == 1 ? launch_align_stream<AASD_BF16, 1>(ctx, sj, a, grid)
+                        : (K == 2 ? launch_align_stream<AASD_BF16, 2>(ctx, sj, a, grid)
+                                  : launch_align_stream<AASD_BF16, 4>(ctx, sj, a, grid));
+        if (rc != AASD_OK) return rc;
+        return after_launch(ctx, 2);
+    }
+    const unsigned int grid = (unsigned int)(n_rows * a.job.chunks);
     if (p->dtype == AASD_F32) {
         if (K == 1) align_kernel<AASD_F32, 1><<<grid, kThreads, 0, ctx->stream>>>(a);
         else if (K == 2) align_kernel<AASD_F32, 2><<<grid, kThreads, 0, ctx->stream>>>(a);
@@ -330,6 +403,16 @@ int aasd_verify(aasd_ctx* ctx, const void* target_logits, const int32_t* draft_i
     if (n_rows == 0) {
         if (n_cands == 0) return AASD_OK;
         verify_empty_kernel<<<(unsigned int)((n_cands + 255) / 256), 256, 0, ctx->stream>>>(a);
+        return after_launch(ctx, 1);
+    }
+    if (a.job.vector_ok && a.job.nvec > 0) {
+        StreamJob sj{};
+        unsigned int sgrid = 0;
+        plan_stream(ctx, sj, a.job, draft_ids, &sgrid);
+        a.job = sj.row;
+        const int rc = p->dtype == AASD_F32 ? launch_verify_stream<AASD_F32>(ctx, sj, a, sgrid)
+                                            : launch_verify_stream<AASD_BF16>(ctx, sj, a, sgrid);
+        if (rc != AASD_OK) return rc;
         return after_launch(ctx, 1);
     }
     const unsigned int grid = (unsigned int)(n_rows * a.job.chunks);

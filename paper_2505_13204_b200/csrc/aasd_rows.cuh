@@ -316,21 +316,14 @@ __device__ inline void write_empty_candidate(const VerifyArgs& a, int c) {
     if (a.out.next_token) a.out.next_token[c] = AASD_NONE;
 }
 
+// Row epilogue of verification, run by one thread once the row's sums and best token are
+// known: Eq. 4-6 for the row, then, in the thread that completes a candidate, the prefix rule.
 template <int DT>
-__global__ void __launch_bounds__(kThreads) verify_kernel(const VerifyArgs a) {
-    __shared__ BlockScratch sc;
-    const RowJob& job = a.job;
-    const int64_t row = blockIdx.x / job.chunks;
-    const int chunk = blockIdx.x % job.chunks;
-    const char* rowp = row_pointer<DT>(job, row);
-    int d = __ldg(a.draft_ids + row);
+__device__ void verify_finish(const VerifyArgs& a, const RowJob& job, int64_t row, const char* rowp,
+                              const RowPartial& merged, float neg_refc, bool centered) {
+    const int d = __ldg(a.draft_ids + row);
     const bool d_ok = d >= 0 && d < job.vocab;
-    float neg_refc;
-    bool centered;
-    if (!row_reduce<DT, 1>(job, row, chunk, d_ok ? d : -1, rowp, neg_refc, centered, sc)) return;
-    if (threadIdx.x != 0) return;
-
-    const RowFinal f = finish_row(sc.merged, job.c1, neg_refc, centered);
+    const RowFinal f = finish_row(merged, job.c1, neg_refc, centered);
     const unsigned int flag = a.draft_flags ? a.draft_flags[row] : AASD_FLAG_CONDITIONAL;
     const double lin = (double)a.alpha * f.H + (double)a.beta;
     const double thr = f.bad ? 0.0 : fmin(lin, f.pmax);
@@ -366,7 +359,7 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(const VerifyArgs a) {
     if (acc) atomicAdd(&job.state->counters[kCntAccepted], 1ull);
     if (status) atomicOr(&job.state->status, status);
 
-    // The CTA that finishes the last row of a candidate applies the prefix rule.
+    // The thread that finishes the last row of a candidate applies the prefix rule.
     int c;
     int64_t lo, hi;
     if (a.cand_offsets) {
@@ -393,6 +386,24 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(const VerifyArgs a) {
     while (lo + n < hi && __ldcg(a.row_accept + lo + n)) ++n;
     if (a.out.accept_len) a.out.accept_len[c] = n;
     if (a.out.next_token) a.out.next_token[c] = (lo + n < hi) ? __ldcg(a.row_own + lo + n) : AASD_NONE;
+}
+
+// One CTA (or `chunks` CTAs) per row with plain vector / scalar loads: the path for logits
+// whose rows are not 16-byte aligned.
+template <int DT>
+__global__ void __launch_bounds__(kThreads) verify_kernel(const VerifyArgs a) {
+    __shared__ BlockScratch sc;
+    const RowJob& job = a.job;
+    const int64_t row = blockIdx.x / job.chunks;
+    const int chunk = blockIdx.x % job.chunks;
+    const char* rowp = row_pointer<DT>(job, row);
+    const int d = __ldg(a.draft_ids + row);
+    const bool d_ok = d >= 0 && d < job.vocab;
+    float neg_refc;
+    bool centered;
+    if (!row_reduce<DT, 1>(job, row, chunk, d_ok ? d : -1, rowp, neg_refc, centered, sc)) return;
+    if (threadIdx.x != 0) return;
+    verify_finish<DT>(a, job, row, rowp, sc.merged, neg_refc, centered);
 }
 
 // Candidates of a call without rows.
@@ -430,20 +441,12 @@ __global__ void align_next_kernel(const AlignArgs a) {
     a.next_ids[t] = nxt;
 }
 
-template <int DT, int K>
-__global__ void __launch_bounds__(kThreads) align_kernel(const AlignArgs a) {
-    __shared__ BlockScratch sc;
-    const RowJob& job = a.job;
-    const int64_t row = blockIdx.x / job.chunks;
-    const int chunk = blockIdx.x % job.chunks;
-    const char* rowp = row_pointer<DT>(job, row);
+// Row epilogue of alignment sampling (Sec. 2.3 alignment test, Fig. 2 extras), one thread.
+template <int DT>
+__device__ void align_finish(const AlignArgs& a, const RowJob& job, int64_t row, const char* rowp,
+                             const RowPartial& merged, float neg_refc, bool centered) {
     const int next = __ldg(a.next_ids + row);
-    float neg_refc;
-    bool centered;
-    if (!row_reduce<DT, K>(job, row, chunk, next, rowp, neg_refc, centered, sc)) return;
-    if (threadIdx.x != 0) return;
-
-    const RowFinal f = finish_row(sc.merged, job.c1, neg_refc, centered);
+    const RowFinal f = finish_row(merged, job.c1, neg_refc, centered);
     const int KE = a.k_extra;
     int ids[kMaxK];
     float ps[kMaxK];
@@ -462,8 +465,8 @@ __global__ void __launch_bounds__(kThreads) align_kernel(const AlignArgs a) {
             aligned = (next == f.top1);
         }
         // the listed tokens that rank above the next token (Fig. 2)
-        for (int j = 0; j < KE && j < K; ++j) {
-            const u64 k = sc.merged.key[j];
+        for (int j = 0; j < KE; ++j) {
+            const u64 k = merged.key[j];
             if (k == 0) break;
             const float xv = key_value(k);
             const int id = key_id(k);
@@ -489,6 +492,21 @@ __global__ void __launch_bounds__(kThreads) align_kernel(const AlignArgs a) {
         atomicAdd(&job.state->counters[kCntBad], 1ull);
         atomicOr(&job.state->status, AASD_STATUS_BAD_ROW);
     }
+}
+
+template <int DT, int K>
+__global__ void __launch_bounds__(kThreads) align_kernel(const AlignArgs a) {
+    __shared__ BlockScratch sc;
+    const RowJob& job = a.job;
+    const int64_t row = blockIdx.x / job.chunks;
+    const int chunk = blockIdx.x % job.chunks;
+    const char* rowp = row_pointer<DT>(job, row);
+    const int next = __ldg(a.next_ids + row);
+    float neg_refc;
+    bool centered;
+    if (!row_reduce<DT, K>(job, row, chunk, next, rowp, neg_refc, centered, sc)) return;
+    if (threadIdx.x != 0) return;
+    align_finish<DT>(a, job, row, rowp, sc.merged, neg_refc, centered);
 }
 
 }  // namespace aasd

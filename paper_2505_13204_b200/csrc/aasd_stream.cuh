@@ -1,0 +1,561 @@
+// Persistent, warp-specialised streaming of logits rows (sm_100a).
+//
+// One CTA per SM slot runs for the whole launch.  A producer warp moves 16 KB tiles of the
+// rows from HBM into a ring of shared-memory stages with bulk asynchronous copies (TMA,
+// cp.async.bulk, completion signalled on an mbarrier); eight consumer warps turn each tile
+// into running sums and best-token candidates; a finisher warp merges what the consumers
+// leave per work item, combines the pieces of rows that were split over several CTAs and
+// evaluates the row (entropy, probabilities, threshold test, accept scan).  The three roles
+// only meet at mbarriers, so the copies of the next rows are in flight while the current
+// row is being reduced and finished.
+//
+// Every wait is bounded: a role that gives up raises AASD_STATUS_TIMEOUT, tells the other
+// roles through a shared flag and leaves; the producer first waits (bounded again) for the
+// copies it still has in flight.
+#pragma once
+
+#include "aasd_rows.cuh"
+
+namespace aasd {
+
+constexpr int kTileBytes = 16384;
+constexpr int kStages = 6;
+constexpr int kConsumerWarps = 8;
+constexpr int kConsumers = kConsumerWarps * 32;
+constexpr int kStreamThreads = kConsumers + 64;   // + producer warp + finisher warp
+constexpr int kRing = 16;
+constexpr unsigned int kWaitLimit = 1u << 24;     // polls of try_wait before giving up
+
+// ---- mbarrier / bulk copy primitives ---------------------------------------------------
+__device__ __forceinline__ unsigned int smem_u32(const void* p) {
+    return (unsigned int)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(u64* bar, unsigned int count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(u64* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(u64* bar, unsigned int bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(u64* bar, unsigned int parity) {
+    unsigned int ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false when the limit ran out or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(u64* bar, unsigned int parity, volatile int* abort_flag) {
+    for (unsigned int it = 0; it < kWaitLimit; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 255u) == 255u && *abort_flag) return false;
+    }
+    return false;
+}
+__device__ __forceinline__ void give_up(volatile int* abort_flag, DeviceState* state) {
+    *abort_flag = 1;
+    atomicOr(&state->status, AASD_STATUS_TIMEOUT);
+}
+__device__ __forceinline__ void bulk_copy_g2s(void* dst_smem, const void* src_gmem, unsigned int bytes, u64* bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+            smem_u32(dst_smem)),
+        "l"(src_gmem), "r"(bytes), "r"(smem_u32(bar))
+        : "memory");
+}
+__device__ __forceinline__ uint4 lds16(const void* p) {
+    uint4 q;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(q.x), "=r"(q.y), "=r"(q.z), "=r"(q.w)
+                 : "r"(smem_u32(p)));
+    return q;
+}
+
+// ---- shared state of a streaming CTA -----------------------------------------------------
+struct ItemInfo {
+    float neg_refc;   // -(reference * c1) of the item's row
+    int hint;         // hinted token of the row (validated), or NONE
+};
+struct WarpPartial {
+    double S, A;
+    u64 key[kMaxK];   // vector-level: (ordered vector maximum << 32) | ~vector index
+};
+struct StreamShared {
+    u64 full[kStages];
+    u64 empty[kStages];
+    u64 done[2];
+    u64 freeb[2];
+    ItemInfo ring[kRing];
+    WarpPartial wp[2][kConsumerWarps];
+    int abort_flag;
+};
+constexpr size_t kStreamSmemBytes = (size_t)kStages * kTileBytes + sizeof(StreamShared) + 128;
+
+struct StreamJob {
+    RowJob row;               // logits, geometry, scratch (chunks = pieces per row)
+    const int32_t* hint_ids;  // [n_rows] token whose logit seeds the row's reference
+    int tiles_per_row;
+    int tiles_per_chunk;
+    long long n_items;        // n_rows * chunks
+};
+
+__device__ __forceinline__ u64 make_vec_key(float vmax, int vec) {
+    return ((u64)ordered_bits(vmax) << 32) | (u64)(0xFFFFFFFFu - (unsigned int)vec);
+}
+
+// NaN-propagating lower clamp of the logits that feed the exponentials: a -inf entry (a
+// masked token) becomes a huge negative finite number, so that its weight is exactly zero
+// without 0 * inf, while NaN still reaches the sums and marks the row bad.  The candidates
+// for the maximum are taken from the unclamped values.
+template <int DT> struct Clamp;
+template <> struct Clamp<AASD_F32> {
+    static __device__ __forceinline__ unsigned int one(unsigned int w) {
+        float r;
+        const float lo = -1.0e30f;
+        asm("max.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(__uint_as_float(w)), "f"(lo));
+        return __float_as_uint(r);
+    }
+    static __device__ __forceinline__ uint4 apply(const uint4& q) {
+        return make_uint4(one(q.x), one(q.y), one(q.z), one(q.w));
+    }
+    static __device__ __forceinline__ float vector_max(const uint4& q) {
+        return fmaxf(fmaxf(__uint_as_float(q.x), __uint_as_float(q.y)),
+                     fmaxf(__uint_as_float(q.z), __uint_as_float(q.w)));
+    }
+};
+template <> struct Clamp<AASD_BF16> {
+    static constexpr unsigned int kLo2 = 0xF149F149u;   // bf16 pair (-1.0e30, -1.0e30)
+    static __device__ __forceinline__ uint4 apply(const uint4& q) {
+        uint4 r;
+        asm("max.NaN.bf16x2 %0, %1, %2;" : "=r"(r.x) : "r"(q.x), "r"(kLo2));
+        asm("max.NaN.bf16x2 %0, %1, %2;" : "=r"(r.y) : "r"(q.y), "r"(kLo2));
+        asm("max.NaN.bf16x2 %0, %1, %2;" : "=r"(r.z) : "r"(q.z), "r"(kLo2));
+        asm("max.NaN.bf16x2 %0, %1, %2;" : "=r"(r.w) : "r"(q.w), "r"(kLo2));
+        return r;
+    }
+    static __device__ __forceinline__ float vector_max(const uint4& q) {
+        unsigned int a, b, c;
+        asm("max.bf16x2 %0, %1, %2;" : "=r"(a) : "r"(q.x), "r"(q.y));
+        asm("max.bf16x2 %0, %1, %2;" : "=r"(b) : "r"(q.z), "r"(q.w));
+        asm("max.bf16x2 %0, %1, %2;" : "=r"(c) : "r"(a), "r"(b));
+        return fmaxf(__uint_as_float(c << 16), __uint_as_float(c & 0xFFFF0000u));
+    }
+};
+
+// Per-thread state of a consumer: packed fp32 sums and the K best vectors.
+template <int DT, int K>
+struct TileAccumulator {
+    static constexpr int kVec = Elt<DT>::kVec;
+    static constexpr int kAcc = kVec / 2;
+    float2 S2[kAcc];
+    float2 A2[kAcc];
+    float best[K];
+    int best_vec[K];
+
+    __device__ __forceinline__ void init() {
+#pragma unroll
+        for (int i = 0; i < kAcc; ++i) {
+            S2[i] = make_float2(0.f, 0.f);
+            A2[i] = make_float2(0.f, 0.f);
+        }
+#pragma unroll
+        for (int j = 0; j < K; ++j) {
+            best[j] = -CUDART_INF_F;
+            best_vec[j] = -1;
+        }
+    }
+    __device__ __forceinline__ void add(const uint4& raw, int vec_index, float c1, float neg_refc) {
+        float x[kVec];
+        Elt<DT>::unpack(Clamp<DT>::apply(raw), x);
+        const float2 cc = make_float2(c1, c1);
+        const float2 rr = make_float2(neg_refc, neg_refc);
+#pragma unroll
+        for (int i = 0; i < kAcc; ++i) {
+            float2 t = __ffma2_rn(make_float2(x[2 * i], x[2 * i + 1]), cc, rr);
+            float2 e = make_float2(ex2_approx(t.x), ex2_approx(t.y));
+            S2[i] = __fadd2_rn(S2[i], e);
+            A2[i] = __ffma2_rn(e, t, A2[i]);
+        }
+        float vmax = Clamp<DT>::vector_max(raw);
+        int vi = vec_index;
+#pragma unroll
+        for (int j = 0; j < K; ++j) {
+            // strict '>' keeps the earlier (lower id) vector ahead among equals
+            const bool up = vmax > best[j];
+            const float hi = fmaxf(best[j], vmax);
+            const float lo = fminf(best[j], vmax);
+            const int hi_i = up ? vi : best_vec[j];
+            const int lo_i = up ? best_vec[j] : vi;
+            best[j] = hi;
+            best_vec[j] = hi_i;
+            vmax = lo;
+            vi = lo_i;
+        }
+    }
+};
+
+// exponent and weight of one raw logit exactly as the consumers form them
+__device__ __forceinline__ void scalar_term(float x, float c1, float neg_refc, float& e, float& t) {
+    float xc;
+    const float lo = -1.0e30f;
+    asm("max.NaN.f32 %0, %1, %2;" : "=f"(xc) : "f"(x), "f"(lo));
+    t = fmaf(xc, c1, neg_refc);
+    e = ex2_approx(t);
+}
+
+// Second, max-centred evaluation of a whole row by one warp: only for rows whose maximum
+// lies so far above the provisional reference that the fp32 sums cannot be trusted.
+template <int DT>
+__device__ void warp_row_centered(const char* rowp, int V, float m, float c1, double& S, double& A) {
+    const int lane = threadIdx.x & 31;
+    double s = 0.0, a = 0.0;
+    for (int i = lane; i < V; i += 32) {
+        const float x = Elt<DT>::load(rowp, i);
+        float t = (x - m) * c1;
+        t = (t < -3.0e38f) ? -3.0e38f : t;   // NaN stays NaN
+        const float e = ex2_approx(t);
+        s += (double)e;
+        a += (double)e * (double)t;
+    }
+    S = warp_sum_f64(s);
+    A = warp_sum_f64(a);
+}
+
+// What the finisher hands to the kernel-specific epilogue.
+struct FinishedRow {
+    RowPartial merged;   // S, A and element-level keys (best tokens)
+    float neg_refc;
+    bool centered;
+};
+
+// Epilogue interface (static functions of a policy type E):
+//   E::finish(args, job, row, rowp, FinishedRow&)  - called by lane 0 of the finisher warp
+template <int DT, int K, class E>
+__global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJob job, const typename E::Args args) {
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* tiles = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
+    StreamShared& sh = *reinterpret_cast<StreamShared*>(tiles + (size_t)kStages * kTileBytes);
+    constexpr int kVec = Elt<DT>::kVec;
+    constexpr int kTileVecs = kTileBytes / 16;
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5, lane = tid & 31;
+    const RowJob& rj = job.row;
+    const int chunks = rj.chunks;
+    const float c1 = rj.c1;
+    volatile int* abort_flag = &sh.abort_flag;
+
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&sh.full[s], 1);
+            mbar_init(&sh.empty[s], kConsumerWarps);
+        }
+        for (int p = 0; p < 2; ++p) {
+            mbar_init(&sh.done[p], kConsumerWarps);
+            mbar_init(&sh.freeb[p], 1);
+        }
+        sh.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    if (warp < kConsumerWarps) {
+        // ------------------------------------------------------------------ consumers
+        unsigned int it = 0, seq = 0;
+        for (long long item = blockIdx.x; item < job.n_items; item += gridDim.x, ++seq) {
+            const int chunk = (int)(item % chunks);
+            const int tb = chunk * job.tiles_per_chunk;
+            const int te = min(job.tiles_per_row, tb + job.tiles_per_chunk);
+            TileAccumulator<DT, K> acc;
+            acc.init();
+            float neg_refc = 0.f;
+            bool alive = true;
+            for (int t = tb; t < te; ++t, ++it) {
+                const int s = it % kStages;
+                if (!mbar_wait(&sh.full[s], (it / kStages) & 1u, abort_flag)) {
+                    if (lane == 0) give_up(abort_flag, rj.state);
+                    alive = false;
+                    break;
+                }
+                if (t == tb) neg_refc = sh.ring[seq % kRing].neg_refc;
+                const unsigned char* base = tiles + (size_t)s * kTileBytes;
+                const int v0 = t * kTileVecs;
+                const int nv = min(kTileVecs, rj.nvec - v0);
+                if (nv == kTileVecs) {
+                    uint4 q[kTileVecs / kConsumers];
+#pragma unroll
+                    for (int k = 0; k < kTileVecs / kConsumers; ++k) q[k] = lds16(base + (size_t)(k * kConsumers + tid) * 16);
+#pragma unroll
+                    for (int k = 0; k < kTileVecs / kConsumers; ++k) acc.add(q[k], v0 + k * kConsumers + tid, c1, neg_refc);
+                } else {
+                    for (int v = tid; v < nv; v += kConsumers) acc.add(lds16(base + (size_t)v * 16), v0 + v, c1, neg_refc);
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sh.empty[s]);
+            }
+            if (!alive) break;
+            // warp-level result of the item
+            double S = 0.0, A = 0.0;
+#pragma unroll
+            for (int i = 0; i < TileAccumulator<DT, K>::kAcc; ++i) {
+                S += (double)acc.S2[i].x + (double)acc.S2[i].y;
+                A += (double)acc.A2[i].x + (double)acc.A2[i].y;
+            }
+            S = warp_sum_f64(S);
+            A = warp_sum_f64(A);
+            u64 vk[K];
+#pragma unroll
+            for (int j = 0; j < K; ++j) vk[j] = acc.best_vec[j] >= 0 ? make_vec_key(acc.best[j], acc.best_vec[j]) : 0ull;
+            u64 wk[K];
+#pragma unroll
+            for (int r = 0; r < K; ++r) {
+                const u64 m = warp_max_u64(vk[0]);
+                wk[r] = m;
+                if (m != 0 && vk[0] == m) {
+#pragma unroll
+                    for (int j = 0; j + 1 < K; ++j) vk[j] = vk[j + 1];
+                    vk[K - 1] = 0;
+                }
+            }
+            const int p = seq & 1;
+            if (!mbar_wait(&sh.freeb[p], ((seq >> 1) & 1u) ^ 1u, abort_flag)) {
+                if (lane == 0) give_up(abort_flag, rj.state);
+                break;
+            }
+            if (lane == 0) {
+                WarpPartial& w = sh.wp[p][warp];
+                w.S = S;
+                w.A = A;
+#pragma unroll
+                for (int j = 0; j < K; ++j) w.key[j] = wk[j];
+                mbar_arrive(&sh.done[p]);
+            }
+        }
+        return;
+    }
+
+    if (warp == kConsumerWarps) {
+        // ------------------------------------------------------------------- producer
+        unsigned int it = 0, seq = 0;
+        unsigned int armed = 0;   // bit s: a copy into stage s was issued in the current use
+        bool alive = true;
+        for (long long item = blockIdx.x; item < job.n_items && alive; item += gridDim.x, ++seq) {
+            const long long row = item / chunks;
+            const int chunk = (int)(item % chunks);
+            const char* rowp = row_pointer<DT>(rj, row);
+            // reference of the row: its hinted logit and its first entries
+            int hint = __ldg(job.hint_ids + row);
+            if (hint < 0 || hint >= rj.vocab) hint = AASD_NONE;
+            float r = -CUDART_INF_F;
+            if (lane < 4 && lane < rj.vocab) r = Elt<DT>::load(rowp, lane);
+            if (lane == 4 && hint >= 0) r = Elt<DT>::load(rowp, hint);
+#pragma unroll
+            for (int o = 4; o > 0; o >>= 1) r = fmaxf(r, __shfl_xor_sync(0xFFFFFFFFu, r, o));
+            r = __shfl_sync(0xFFFFFFFFu, r, 0);
+            if (!(fabsf(r) <= 3.0e38f)) r = 0.f;
+            if (lane == 0) {
+                ItemInfo& info = sh.ring[seq % kRing];
+                info.neg_refc = -(r * c1);
+                info.hint = hint;
+                const int tb = chunk * job.tiles_per_chunk;
+                const int te = min(job.tiles_per_row, tb + job.tiles_per_chunk);
+                for (int t = tb; t < te; ++t, ++it) {
+                    const int s = it % kStages;
+                    if (!mbar_wait(&sh.empty[s], ((it / kStages) & 1u) ^ 1u, abort_flag)) {
+                        alive = false;
+                        break;
+                    }
+                    const long long off = (long long)t * kTileBytes;
+                    const long long left = (long long)rj.nvec * 16 - off;
+                    const unsigned int bytes = (unsigned int)(left < kTileBytes ? left : kTileBytes);
+                    mbar_arrive_expect_tx(&sh.full[s], bytes);
+                    bulk_copy_g2s(tiles + (size_t)s * kTileBytes, rowp + off, bytes, &sh.full[s]);
+                    armed |= 1u << s;
+                }
+            }
+            alive = __shfl_sync(0xFFFFFFFFu, alive ? 1 : 0, 0) != 0;
+        }
+        if (!alive && lane == 0) {
+            // give the copies still in flight a bounded time to land before the CTA leaves
+            give_up(abort_flag, rj.state);
+            for (int back = 1; back <= kStages && back <= (int)it; ++back) {
+                const unsigned int j = it - back;
+                const int s = j % kStages;
+                if (armed & (1u << s)) {
+                    for (unsigned int w = 0; w < kWaitLimit; ++w)
+                        if (mbar_try_wait(&sh.full[s], (j / kStages) & 1u)) break;
+                }
+            }
+        }
+        return;
+    }
+
+    // ------------------------------------------------------------------------- finisher
+    unsigned int seq = 0;
+    for (long long item = blockIdx.x; item < job.n_items; item += gridDim.x, ++seq) {
+        const long long row = item / chunks;
+        const int chunk = (int)(item % chunks);
+        const char* rowp = row_pointer<DT>(rj, row);
+        const int p = seq & 1;
+        if (!mbar_wait(&sh.done[p], (seq >> 1) & 1u, abort_flag)) {
+            if (lane == 0) give_up(abort_flag, rj.state);
+            return;
+        }
+        double S = 0.0, A = 0.0;
+        u64 vk[K];
+#pragma unroll
+        for (int j = 0; j < K; ++j) vk[j] = 0;
+        if (lane < kConsumerWarps) {
+            const WarpPartial& w = sh.wp[p][lane];
+            S = w.S;
+            A = w.A;
+#pragma unroll
+            for (int j = 0; j < K; ++j) vk[j] = w.key[j];
+        }
+        const ItemInfo info = sh.ring[seq % kRing];
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.freeb[p]);
+        S = warp_sum_f64(S);
+        A = warp_sum_f64(A);
+        u64 mk[K];   // merged vector keys, identical in every lane
+#pragma unroll
+        for (int r = 0; r < K; ++r) {
+            const u64 m = warp_max_u64(vk[0]);
+            mk[r] = m;
+            if (m != 0 && vk[0] == m) {
+#pragma unroll
+                for (int j = 0; j + 1 < K; ++j) vk[j] = vk[j + 1];
+                vk[K - 1] = 0;
+            }
+        }
+        if (chunks > 1) {
+            // pieces of a row meet in global memory; the last one to arrive carries on
+            RowPartial* slots = rj.partials + row * chunks;
+            int last = 0;
+            if (lane == 0) {
+                RowPartial mine;
+                mine.S = S;
+                mine.A = A;
+#pragma unroll
+                for (int j = 0; j < kMaxK; ++j) mine.key[j] = j < K ? mk[j] : 0ull;
+                slots[chunk] = mine;
+                __threadfence();
+                const unsigned int t = atomicAdd(&rj.row_tickets[row], 1u);
+                last = (t == (unsigned int)chunks - 1);
+                if (last) rj.row_tickets[row] = 0;
+            }
+            last = __shfl_sync(0xFFFFFFFFu, last, 0);
+            if (!last) continue;
+            __threadfence();
+            S = 0.0;
+            A = 0.0;
+#pragma unroll
+            for (int j = 0; j < K; ++j) vk[j] = 0;
+            for (int c = lane; c < chunks; c += 32) {
+                const RowPartial* q = slots + c;
+                S += __ldcg(&q->S);
+                A += __ldcg(&q->A);
+#pragma unroll
+                for (int j = 0; j < K; ++j) key_insert<K>(vk, __ldcg(&q->key[j]));
+            }
+            S = warp_sum_f64(S);
+            A = warp_sum_f64(A);
+#pragma unroll
+            for (int r = 0; r < K; ++r) {
+                const u64 m = warp_max_u64(vk[0]);
+                mk[r] = m;
+                if (m != 0 && vk[0] == m) {
+#pragma unroll
+                    for (int j = 0; j + 1 < K; ++j) vk[j] = vk[j + 1];
+                    vk[K - 1] = 0;
+                }
+            }
+        }
+        // Best tokens: they lie inside the K best vectors; plus the ragged tail of the row.
+        u64 ek[K];
+#pragma unroll
+        for (int j = 0; j < K; ++j) ek[j] = 0;
+        float ts = 0.f, ta = 0.f;
+        {
+            u64 mine = 0;
+#pragma unroll
+            for (int j = 0; j < K; ++j)
+                if (lane == j) mine = mk[j];
+            if (lane < K && mine != 0) {
+                const int vec = key_id(mine);
+                const uint4 q = __ldg(reinterpret_cast<const uint4*>(rowp) + vec);
+                float x[kVec];
+                Elt<DT>::unpack(q, x);
+#pragma unroll
+                for (int i = 0; i < kVec; ++i)
+                    if (x[i] > -CUDART_INF_F) key_insert<K>(ek, make_key(x[i], vec * kVec + i));
+            }
+            const int tail0 = rj.nvec * kVec;
+            const int i = tail0 + lane - K;
+            if (lane >= K && i < rj.vocab) {
+                const float x = Elt<DT>::load(rowp, i);
+                float e, t;
+                scalar_term(x, c1, info.neg_refc, e, t);
+                ts = e;
+                ta = e * t;
+                if (x > -CUDART_INF_F) key_insert<K>(ek, make_key(x, i));
+            }
+        }
+        S += warp_sum_f64((double)ts);
+        A += warp_sum_f64((double)ta);
+        FinishedRow fr;
+#pragma unroll
+        for (int r = 0; r < kMaxK; ++r) fr.merged.key[r] = 0;
+#pragma unroll
+        for (int r = 0; r < K; ++r) {
+            const u64 m = warp_max_u64(ek[0]);
+            fr.merged.key[r] = m;
+            if (m != 0 && ek[0] == m) {
+#pragma unroll
+                for (int j = 0; j + 1 < K; ++j) ek[j] = ek[j + 1];
+                ek[K - 1] = 0;
+            }
+        }
+        fr.neg_refc = info.neg_refc;
+        fr.centered = false;
+        const u64 k0 = fr.merged.key[0];
+        const float m = key_value(k0);
+        if (k0 != 0 && fabsf(m) <= 3.0e38f) {
+            const float shift = fmaf(m, c1, info.neg_refc);
+            if (!(S > 0.0) || !(S <= 1.0e300) || !(fabs(A) <= 1.0e300) || !(fabsf(shift) <= kRedoShift)) {
+                warp_row_centered<DT>(rowp, rj.vocab, m, c1, S, A);
+                fr.neg_refc = -m;
+                fr.centered = true;
+                if (lane == 0) atomicAdd(&rj.state->counters[kCntRedo], 1ull);
+            }
+        }
+        fr.merged.S = S;
+        fr.merged.A = A;
+        if (lane == 0) E::finish(args, rj, row, rowp, fr);
+    }
+}
+
+template <int DT>
+struct VerifyEpilogue {
+    using Args = VerifyArgs;
+    static __device__ void finish(const VerifyArgs& a, const RowJob& job, int64_t row, const char* rowp,
+                                  const FinishedRow& fr) {
+        verify_finish<DT>(a, job, row, rowp, fr.merged, fr.neg_refc, fr.centered);
+    }
+};
+template <int DT>
+struct AlignEpilogue {
+    using Args = AlignArgs;
+    static __device__ void finish(const AlignArgs& a, const RowJob& job, int64_t row, const char* rowp,
+                                  const FinishedRow& fr) {
+        align_finish<DT>(a, job, row, rowp, fr.merged, fr.neg_refc, fr.centered);
+    }
+};
+
+}  // namespace aasd
