@@ -129,16 +129,17 @@ int plan_rows(aasd_ctx* ctx, RowJob& job, const void* logits, int dtype, int voc
 
 // Geometry of the persistent streaming launch over 16-byte aligned rows.  Work items are
 // (row, piece) pairs handed out round-robin to a grid of two CTAs per SM; rows are cut into
-// pieces (at tile boundaries) only while there are too few rows to keep every CTA busy for
-// several items.
+// pieces (at tile boundaries) only when there are far fewer rows than CTA slots.
 void plan_stream(aasd_ctx* ctx, StreamJob& sj, const RowJob& job, const int32_t* hint_ids, unsigned int* grid) {
     sj.row = job;
     sj.hint_ids = hint_ids;
     const int64_t row_bytes = (int64_t)job.nvec * 16;
     const int tiles = (int)((row_bytes + kTileBytes - 1) / kTileBytes);
     const int64_t slots = (int64_t)ctx->sm_count * 2;
-    int64_t chunks = (6 * slots + job.n_rows - 1) / job.n_rows;
-    if (chunks > kMaxSplit) chunks = kMaxSplit;
+    // Cutting a row costs its pieces a trip through global memory (partial record, fence,
+    // ticket), which measured slower than the imbalance it removes unless rows are scarce.
+    int64_t chunks = slots / (4 * job.n_rows);
+    if (chunks > 8) chunks = 8;
     if (chunks > tiles) chunks = tiles;
     if (chunks < 1) chunks = 1;
     if (const char* e = getenv("AASD_STREAM_CHUNKS")) {   // tuning override
