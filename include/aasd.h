@@ -287,6 +287,45 @@ typedef struct aasd_step_args {
 int aasd_step(aasd_ctx* ctx, const aasd_step_args* args, void* workspace,
               size_t workspace_bytes);
 
+/* ---- verification for callers that cannot allocate ------------------------------- */
+
+#define AASD_STATIC_MAX_ROWS 8192   /* most logits rows per aasd_verify_static call */
+#define AASD_STATIC_MAX_CANDS 8192  /* most candidates per aasd_verify_static call */
+
+/* (No counterpart in the paper: this is a packaging variant of aasd_verify.)
+ *
+ * Some callers may not allocate device memory at the point where they verify: code that
+ * runs inside a region where cudaMalloc is forbidden or would synchronise the device (an
+ * inference server's steady-state loop that pre-allocated everything at start-up, a plugin
+ * that only owns the buffers its host hands it, a caller holding a memory-pool lock).
+ * aasd_verify needs a context (aasd_create allocates its status block) and a caller-made
+ * workspace; this entry point needs neither.  Its scratch - what the workspace and the
+ * context's status block would hold - lives in a fixed block of device memory that is part
+ * of the library image: about 0.5 MB on every GPU that loads the library, held until the
+ * process exits.  The call itself makes no cudaMalloc / cudaFree and calls nothing that
+ * allocates.
+ *
+ * Arguments are those of aasd_verify, with the device index and the stream (a
+ * cudaStream_t, NULL = legacy default stream) given directly, and results identical to
+ * aasd_verify's on the same inputs.  status_bits (DEVICE pointer, may be NULL) receives the
+ * AASD_STATUS_* bits this call raised, written on the stream after the kernel.
+ *
+ * Limits and rules:
+ *  - n_rows <= AASD_STATIC_MAX_ROWS and n_cands <= AASD_STATIC_MAX_CANDS, otherwise
+ *    AASD_ERR_WORKSPACE_TOO_SMALL is returned and nothing is launched.
+ *  - The first call on a device looks up the block's device address (once per device, with
+ *    that device made current) and so should be made before any stream capture begins.
+ *  - Every call on a device shares the one block.  Each call clears the parts that must
+ *    start at zero (on the stream, before its kernel), so the block's old contents never
+ *    leak into a result; but two calls that can overlap on the GPU (different streams
+ *    without an ordering between them) race on it and give undefined results.  Order them.
+ *  - The call makes `device` the current device of the calling thread. */
+int aasd_verify_static(int device, void* stream, const void* target_logits,
+                       const int32_t* draft_ids, const uint8_t* draft_flags,
+                       const int32_t* cand_offsets, int32_t n_cands, int64_t n_rows,
+                       const aasd_verify_params* params, const aasd_verify_out* out,
+                       uint32_t* status_bits);
+
 #ifdef __cplusplus
 }
 #endif

@@ -25,8 +25,9 @@ EXPORTS = [
     "aasd_create", "aasd_destroy", "aasd_set_stream", "aasd_status_str", "aasd_poll_status",
     "aasd_get_counters", "aasd_reset_counters", "aasd_launch_count", "aasd_workspace_bytes",
     "aasd_workspace_init", "aasd_workspace_release", "aasd_align_sample", "aasd_draft",
-    "aasd_verify", "aasd_select", "aasd_append", "aasd_step",
+    "aasd_verify", "aasd_select", "aasd_append", "aasd_step", "aasd_verify_static",
 ]
+STATIC_MAX_ROWS = STATIC_MAX_CANDS = 8192
 
 _vp = C.c_void_p
 
@@ -119,6 +120,8 @@ def load_library(path: str | None = None):
                                 C.c_int32, _vp, _vp, _vp]
     lib.aasd_append.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, C.c_int32, C.c_int32]
     lib.aasd_step.argtypes = [_vp, C.POINTER(StepArgs), _vp, C.c_size_t]
+    lib.aasd_verify_static.argtypes = [C.c_int, _vp, _vp, _vp, _vp, _vp, C.c_int32, C.c_int64,
+                                       C.POINTER(VerifyParams), C.POINTER(VerifyOut), _vp]
     if path == _build.LIB:
         _lib = lib
     return lib
@@ -155,6 +158,48 @@ def _dev_i32(x, device):
         assert x.dtype == torch.int32 and x.is_cuda and x.is_contiguous()
         return x
     return torch.as_tensor(x, dtype=torch.int32).to(device)
+
+
+def verify_static(target_logits, draft_ids, cand_offsets=None, draft_flags=None, alpha=0.1,
+                  beta=0.1, mode=VERIFY_CONDITIONAL, seed=0, step=0, inv_temperature=1.0,
+                  rows_per_cand=0, outputs=None, status_bits=None, stream=None):
+    """aasd_verify_static: verification for callers that cannot allocate device memory.
+
+    No context and no workspace: the library's own fixed scratch block is used, and the
+    call itself allocates nothing.  Every tensor (``outputs`` included, a dict like the one
+    ``Context.verify`` returns; ``status_bits``, one int32 on the device) must therefore be
+    passed in ready-made when the caller is in such a region; when ``outputs`` is None this
+    wrapper allocates it with torch for convenience.  At most STATIC_MAX_ROWS rows and
+    STATIC_MAX_CANDS candidates per call; calls on one device must not overlap.
+    """
+    lib = load_library()
+    x = target_logits
+    assert x.is_cuda and x.dim() == 2 and x.stride(1) == 1
+    R, V = x.shape
+    dev = x.device
+    d = draft_ids.reshape(-1)
+    offs = cand_offsets
+    assert offs is None or (offs.is_cuda and offs.dtype == torch.int32)
+    Cn = (offs.numel() - 1) if offs is not None else (R // rows_per_cand if rows_per_cand else 0)
+    o = outputs or dict(
+        p_draft=torch.empty(R, dtype=torch.float32, device=dev),
+        entropy=torch.empty(R, dtype=torch.float32, device=dev),
+        pmax=torch.empty(R, dtype=torch.float32, device=dev),
+        argmax=torch.empty(R, dtype=torch.int32, device=dev),
+        threshold=torch.empty(R, dtype=torch.float32, device=dev),
+        accept=torch.empty(R, dtype=torch.uint8, device=dev),
+        sampled=torch.empty(R, dtype=torch.int32, device=dev),
+        accept_len=torch.empty(Cn, dtype=torch.int32, device=dev),
+        next_token=torch.empty(Cn, dtype=torch.int32, device=dev))
+    prm = VerifyParams(V, _dtype_code(x), x.stride(0), float(alpha), float(beta),
+                       float(inv_temperature), int(mode), int(rows_per_cand), int(step), int(seed))
+    out = VerifyOut(*[_p(o.get(n)) for n, _ in VerifyOut._fields_])
+    fl = None if draft_flags is None else draft_flags.reshape(-1)
+    stream = stream or torch.cuda.current_stream(dev)
+    _check(lib.aasd_verify_static(dev.index, _vp(stream.cuda_stream), _p(x), _p(d), _p(fl), _p(offs),
+                                  Cn, R, C.byref(prm), C.byref(out), _p(status_bits)),
+           "aasd_verify_static")
+    return o
 
 
 class Context:

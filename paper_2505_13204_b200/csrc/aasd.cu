@@ -7,6 +7,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <map>
+#include <mutex>
 #include <new>
 
 #include "../../include/aasd.h"
@@ -474,3 +475,123 @@ int aasd_step(aasd_ctx* ctx, const aasd_step_args* s, void* workspace, size_t wo
 }
 
 }  // extern "C"
+
+// ---- verification without any allocation ---------------------------------------------------
+//
+// Scratch of aasd_verify_static: one block per GPU that loads the library, held until the
+// process exits.  Layout = the workspace layout for kStaticMaxRows rows and kStaticMaxCands
+// candidates, followed by the status word and counters that a context would own.
+namespace {
+
+constexpr int64_t kStaticMaxRows = AASD_STATIC_MAX_ROWS;
+constexpr int64_t kStaticMaxCands = AASD_STATIC_MAX_CANDS;
+constexpr size_t kStaticWorkspaceBytes =
+    ((sizeof(RowPartial) * (size_t)kPartialSlots + 255) / 256 * 256) +   // pieces of split rows
+    ((4 * (size_t)kStaticMaxRows + 255) / 256 * 256) +                   // row tickets
+    ((4 * (size_t)kStaticMaxCands + 255) / 256 * 256) +                  // candidate tickets
+    (((size_t)kStaticMaxRows + 255) / 256 * 256) +                       // accept bits
+    2 * ((4 * (size_t)kStaticMaxRows + 255) / 256 * 256);                // own tokens, next ids
+constexpr size_t kStaticBytes = kStaticWorkspaceBytes + 256;
+
+}  // namespace
+
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];
+
+namespace {
+
+constexpr int kStaticMaxDevices = 64;
+struct StaticSlot {
+    bool ready;
+    int sm_count;
+    char* scratch;   // device address of g_static_scratch on this device
+};
+StaticSlot g_static_slots[kStaticMaxDevices];
+std::mutex g_static_mutex;
+
+}  // namespace
+
+extern "C" int aasd_verify_static(int device, void* stream, const void* target_logits,
+                                  const int32_t* draft_ids, const uint8_t* draft_flags,
+                                  const int32_t* cand_offsets, int32_t n_cands, int64_t n_rows,
+                                  const aasd_verify_params* p, const aasd_verify_out* out,
+                                  uint32_t* status_bits) {
+    if (p == nullptr || out == nullptr) return AASD_ERR_INVALID_ARG;
+    if (device < 0 || device >= kStaticMaxDevices) return AASD_ERR_INVALID_ARG;
+    if (n_cands < 0 || n_rows < 0) return AASD_ERR_BAD_SHAPE;
+    if (n_rows > kStaticMaxRows || n_cands > kStaticMaxCands) return AASD_ERR_WORKSPACE_TOO_SMALL;
+    if (p->mode < AASD_VERIFY_CONDITIONAL || p->mode > AASD_VERIFY_STRICT_SAMPLED) return AASD_ERR_INVALID_ARG;
+    if (p->mode == AASD_VERIFY_STRICT_SAMPLED) return AASD_ERR_UNSUPPORTED;
+    if (!(p->alpha >= 0.f) || !(p->beta >= 0.f)) return AASD_ERR_INVALID_ARG;
+    if (cand_offsets == nullptr) {
+        if (p->rows_per_cand < 1 || (int64_t)n_cands * p->rows_per_cand != n_rows) return AASD_ERR_BAD_SHAPE;
+    }
+    if (n_rows > 0 && (draft_ids == nullptr || n_cands == 0)) return AASD_ERR_INVALID_ARG;
+    const WorkspaceLayout L = make_layout(kStaticMaxRows, kStaticMaxCands);
+    if (L.bytes != kStaticWorkspaceBytes) return AASD_ERR_WORKSPACE_TOO_SMALL;   // layouts out of step
+
+    std::lock_guard<std::mutex> guard(g_static_mutex);
+    AASD_CUDA(cudaSetDevice(device));
+    StaticSlot& slot = g_static_slots[device];
+    if (!slot.ready) {
+        // Set-up, once per device and with that device current.  In host code the array's
+        // name is only a handle: the address a kernel can use comes from the runtime.
+        int major = 0, sms = 0;
+        AASD_CUDA(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device));
+        if (major != 10) return AASD_ERR_NOT_SM100;
+        AASD_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || ptr == nullptr) return AASD_ERR_CUDA;
+        slot.scratch = static_cast<char*>(ptr);
+        slot.sm_count = sms;
+        slot.ready = true;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    char* ws = slot.scratch;
+    DeviceState* state = reinterpret_cast<DeviceState*>(ws + kStaticWorkspaceBytes);
+    // The block keeps what the last call left: the tickets and the status word must start
+    // at zero even if that call was cut short.
+    AASD_CUDA(cudaMemsetAsync(ws + L.off_row_tickets, 0, L.off_row_accept - L.off_row_tickets, s));
+    AASD_CUDA(cudaMemsetAsync(state, 0, sizeof(DeviceState), s));
+
+    aasd_ctx local{};   // launch geometry only: nothing of it outlives the call
+    local.device = device;
+    local.stream = s;
+    local.sm_count = slot.sm_count;
+    local.state = state;
+    VerifyArgs a{};
+    int err = plan_rows(&local, a.job, target_logits, p->dtype, p->vocab, p->row_stride, n_rows, p->inv_temperature,
+                        ws, L);
+    if (err != AASD_OK) return err;
+    if (n_rows * (int64_t)a.job.chunks > 0x7FFFFFFFLL) return AASD_ERR_BAD_SHAPE;
+    a.draft_ids = draft_ids;
+    a.draft_flags = draft_flags;
+    a.cand_offsets = cand_offsets;
+    a.n_cands = n_cands;
+    a.rows_per_cand = p->rows_per_cand;
+    a.alpha = p->alpha;
+    a.beta = p->beta;
+    a.mode = p->mode;
+    a.cand_tickets = reinterpret_cast<unsigned int*>(ws + L.off_cand_tickets);
+    a.row_accept = reinterpret_cast<uint8_t*>(ws + L.off_row_accept);
+    a.row_own = reinterpret_cast<int32_t*>(ws + L.off_row_own);
+    a.out = *out;
+    if (n_rows == 0) {
+        if (n_cands > 0) verify_empty_kernel<<<(unsigned int)((n_cands + 255) / 256), 256, 0, s>>>(a);
+    } else if (a.job.vector_ok && a.job.nvec > 0) {
+        StreamJob sj{};
+        unsigned int sgrid = 0;
+        plan_stream(&local, sj, a.job, draft_ids, &sgrid);
+        a.job = sj.row;
+        const int rc = p->dtype == AASD_F32 ? launch_verify_stream<AASD_F32>(&local, sj, a, sgrid)
+                                            : launch_verify_stream<AASD_BF16>(&local, sj, a, sgrid);
+        if (rc != AASD_OK) return rc;
+    } else {
+        const unsigned int grid = (unsigned int)(n_rows * a.job.chunks);
+        if (p->dtype == AASD_F32) verify_kernel<AASD_F32><<<grid, kThreads, 0, s>>>(a);
+        else verify_kernel<AASD_BF16><<<grid, kThreads, 0, s>>>(a);
+    }
+    if (cudaGetLastError() != cudaSuccess) return AASD_ERR_CUDA;
+    if (status_bits != nullptr)
+        AASD_CUDA(cudaMemcpyAsync(status_bits, &state->status, 4, cudaMemcpyDeviceToDevice, s));
+    return AASD_OK;
+}
