@@ -447,18 +447,40 @@ def run_micro(args):
         call(s % n_buf)
     torch.cuda.synchronize()
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    t0.record()
-    for s in range(args.steps):
-        call(s % n_buf)
-    t1.record()
-    torch.cuda.synchronize()
-    ms = t0.elapsed_time(t1) / args.steps
+    if args.graph:
+        # few rows: a launch from Python costs more than the kernel runs, so the launches
+        # are captured once (one per buffer) and the graph is replayed
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        ctx.set_stream(side)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            call(0)
+            with torch.cuda.graph(graph, stream=side):
+                for j in range(n_buf):
+                    call(j)
+            reps = max(1, args.steps // n_buf)
+            for _ in range(3):
+                graph.replay()
+            t0.record()
+            for _ in range(reps):
+                graph.replay()
+            t1.record()
+        torch.cuda.synchronize()
+        ms = t0.elapsed_time(t1) / (reps * n_buf)
+    else:
+        t0.record()
+        for s in range(args.steps):
+            call(s % n_buf)
+        t1.record()
+        torch.cuda.synchronize()
+        ms = t0.elapsed_time(t1) / args.steps
     esize = 2 if w.dtype == "bf16" else 4
     peak, src = measured_peaks()
     gbs = R * w.vocab * esize / (ms * 1e-3) / 1e9
     print(json.dumps({"micro": args.micro, "workload": w.name, "rows": R, "vocab": w.vocab, "us_per_launch": ms * 1e3,
                       "rows_per_s": R / (ms * 1e-3), "GBps": gbs, "frac_of_peak": gbs / peak, "peak": peak,
-                      "peak_source": src, "buffers": n_buf, "counters": ctx.counters()}))
+                      "peak_source": src, "buffers": n_buf, "graph": bool(args.graph), "counters": ctx.counters()}))
 
 
 def main():
@@ -466,6 +488,7 @@ def main():
     ap.add_argument("--micro", default=None, choices=["verify", "align"],
                     help="time one kernel alone on --rows rows of the workload")
     ap.add_argument("--rows", type=int, default=1024)
+    ap.add_argument("--graph", action="store_true", help="--micro: replay the launches from a CUDA graph")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=64)
     ap.add_argument("--warmup", type=int, default=8)

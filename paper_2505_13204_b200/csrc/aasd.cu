@@ -22,7 +22,7 @@ namespace {
 struct WorkspaceLayout {
     size_t bytes;
     int64_t max_rows, max_cands;
-    size_t off_partials, off_row_tickets, off_cand_tickets, off_row_accept, off_row_own, off_next;
+    size_t off_partials, off_row_tickets, off_cand_tickets, off_sched, off_row_accept, off_row_own, off_next;
 };
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -38,6 +38,8 @@ WorkspaceLayout make_layout(int64_t max_rows, int64_t max_cands) {
     o = align_up(o + 4 * (size_t)max_rows, 256);
     L.off_cand_tickets = o;
     o = align_up(o + 4 * (size_t)max_cands, 256);
+    L.off_sched = o;
+    o = align_up(o + 2 * sizeof(unsigned int), 256);
     L.off_row_accept = o;
     o = align_up(o + (size_t)max_rows, 256);
     L.off_row_own = o;
@@ -128,33 +130,41 @@ int plan_rows(aasd_ctx* ctx, RowJob& job, const void* logits, int dtype, int voc
     return AASD_OK;
 }
 
-// Geometry of the persistent streaming launch over 16-byte aligned rows.  Work items are
-// (row, piece) pairs handed out round-robin to a grid of two CTAs per SM; rows are cut into
-// pieces (at tile boundaries) only when there are far fewer rows than CTA slots.
-void plan_stream(aasd_ctx* ctx, StreamJob& sj, const RowJob& job, const int32_t* hint_ids, unsigned int* grid) {
+// Geometry of the persistent streaming launch over 16-byte aligned rows: a grid of two CTAs
+// per SM that claim work items from a counter.  An item is a whole row unless there are
+// fewer rows than CTA slots; then every row is cut into pieces at tile boundaries.
+void plan_stream(aasd_ctx* ctx, StreamJob& sj, const RowJob& job, const int32_t* hint_ids, char* ws,
+                 const WorkspaceLayout& L, unsigned int* grid) {
     sj.row = job;
     sj.hint_ids = hint_ids;
+    sj.sched = reinterpret_cast<unsigned int*>(ws + L.off_sched);
     const int64_t row_bytes = (int64_t)job.nvec * 16;
     const int tiles = (int)((row_bytes + kTileBytes - 1) / kTileBytes);
     const int64_t slots = (int64_t)ctx->sm_count * 2;
     // Cutting a row costs its pieces a trip through global memory (partial record, fence,
-    // ticket), which measured slower than the imbalance it removes unless rows are scarce.
-    int64_t chunks = slots / (4 * job.n_rows);
-    if (chunks > 8) chunks = 8;
-    if (chunks > tiles) chunks = tiles;
-    if (chunks < 1) chunks = 1;
-    if (const char* e = getenv("AASD_STREAM_CHUNKS")) {   // tuning override
-        const long v = atol(e);
-        if (v >= 1) chunks = v > tiles ? tiles : v;
+    // ticket) on the finisher's serial path; with many rows that measured slower than the
+    // idle time it removes at the end of the launch (dynamic claiming already evens out
+    // CTAs of different speed), so rows are cut only when they are scarce.
+    int64_t tail_rows = 0, chunks = 1;
+    if (job.n_rows < slots) {
+        tail_rows = job.n_rows;
+        chunks = slots / (2 * job.n_rows);
+        if (chunks > 8) chunks = 8;
+        if (const char* e = getenv("AASD_STREAM_CHUNKS")) {   // tuning override
+            const long v = atol(e);
+            if (v >= 1) chunks = v;
+        }
     }
-    while (chunks > 1 && chunks * job.n_rows > kPartialSlots) --chunks;
-    int per = (int)((tiles + chunks - 1) / chunks);
-    if (per < 1) per = 1;
-    chunks = tiles > 0 ? (tiles + per - 1) / per : 1;
+    if (chunks > tiles) chunks = tiles;
+    if (chunks <= 1) {
+        chunks = 1;
+        tail_rows = 0;
+    }
+    while (tail_rows * chunks > kPartialSlots) --tail_rows;
     sj.tiles_per_row = tiles;
-    sj.tiles_per_chunk = per;
-    sj.row.chunks = (int)chunks;
-    sj.n_items = job.n_rows * chunks;
+    sj.whole_rows = (int)(job.n_rows - tail_rows);
+    sj.tail_chunks = (int)chunks;
+    sj.n_items = (job.n_rows - tail_rows) + tail_rows * chunks;
     *grid = (unsigned int)(sj.n_items < slots ? sj.n_items : slots);
 }
 
@@ -323,8 +333,7 @@ int aasd_align_sample(aasd_ctx* ctx, const void* prefill_logits, const int32_t* 
         // 16-byte aligned rows: persistent TMA-fed streaming kernel
         StreamJob sj{};
         unsigned int grid = 0;
-        plan_stream(ctx, sj, a.job, a.next_ids, &grid);
-        a.job = sj.row;
+        plan_stream(ctx, sj, a.job, a.next_ids, ws, *L, &grid);
         int rc;
         if (p->dtype == AASD_F32)
             rc = K == 1 ? launch_align_stream<AASD_F32, 1>(ctx, sj, a, grid)
@@ -410,8 +419,7 @@ int aasd_verify(aasd_ctx* ctx, const void* target_logits, const int32_t* draft_i
     if (a.job.vector_ok && a.job.nvec > 0) {
         StreamJob sj{};
         unsigned int sgrid = 0;
-        plan_stream(ctx, sj, a.job, draft_ids, &sgrid);
-        a.job = sj.row;
+        plan_stream(ctx, sj, a.job, draft_ids, ws, *L, &sgrid);
         const int rc = p->dtype == AASD_F32 ? launch_verify_stream<AASD_F32>(ctx, sj, a, sgrid)
                                             : launch_verify_stream<AASD_BF16>(ctx, sj, a, sgrid);
         if (rc != AASD_OK) return rc;
@@ -489,6 +497,7 @@ constexpr size_t kStaticWorkspaceBytes =
     ((sizeof(RowPartial) * (size_t)kPartialSlots + 255) / 256 * 256) +   // pieces of split rows
     ((4 * (size_t)kStaticMaxRows + 255) / 256 * 256) +                   // row tickets
     ((4 * (size_t)kStaticMaxCands + 255) / 256 * 256) +                  // candidate tickets
+    256 +                                                                // work-item counters
     (((size_t)kStaticMaxRows + 255) / 256 * 256) +                       // accept bits
     2 * ((4 * (size_t)kStaticMaxRows + 255) / 256 * 256);                // own tokens, next ids
 constexpr size_t kStaticBytes = kStaticWorkspaceBytes + 256;
@@ -548,8 +557,8 @@ extern "C" int aasd_verify_static(int device, void* stream, const void* target_l
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     char* ws = slot.scratch;
     DeviceState* state = reinterpret_cast<DeviceState*>(ws + kStaticWorkspaceBytes);
-    // The block keeps what the last call left: the tickets and the status word must start
-    // at zero even if that call was cut short.
+    // The block keeps what the last call left: the tickets, the work-item counters and the status
+    // word must start at zero even if that call was cut short.
     AASD_CUDA(cudaMemsetAsync(ws + L.off_row_tickets, 0, L.off_row_accept - L.off_row_tickets, s));
     AASD_CUDA(cudaMemsetAsync(state, 0, sizeof(DeviceState), s));
 
@@ -580,8 +589,7 @@ extern "C" int aasd_verify_static(int device, void* stream, const void* target_l
     } else if (a.job.vector_ok && a.job.nvec > 0) {
         StreamJob sj{};
         unsigned int sgrid = 0;
-        plan_stream(&local, sj, a.job, draft_ids, &sgrid);
-        a.job = sj.row;
+        plan_stream(&local, sj, a.job, draft_ids, ws, L, &sgrid);
         const int rc = p->dtype == AASD_F32 ? launch_verify_stream<AASD_F32>(&local, sj, a, sgrid)
                                             : launch_verify_stream<AASD_BF16>(&local, sj, a, sgrid);
         if (rc != AASD_OK) return rc;

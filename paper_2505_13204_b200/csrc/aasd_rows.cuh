@@ -316,12 +316,27 @@ __device__ inline void write_empty_candidate(const VerifyArgs& a, int c) {
     if (a.out.next_token) a.out.next_token[c] = AASD_NONE;
 }
 
-// Row epilogue of verification, run by one thread once the row's sums and best token are
-// known: Eq. 4-6 for the row, then, in the thread that completes a candidate, the prefix rule.
+// What a finished row adds to the running counters and the status word.  The streaming
+// kernel keeps one per CTA in registers and flushes it when the CTA leaves.
+struct Tally {
+    unsigned int rows, bad, redo, near, accepted, status;
+    __device__ void clear() { rows = bad = redo = near = accepted = status = 0; }
+    __device__ void flush(DeviceState* st) const {
+        if (rows) atomicAdd(&st->counters[kCntRows], (u64)rows);
+        if (bad) atomicAdd(&st->counters[kCntBad], (u64)bad);
+        if (redo) atomicAdd(&st->counters[kCntRedo], (u64)redo);
+        if (near) atomicAdd(&st->counters[kCntNear], (u64)near);
+        if (accepted) atomicAdd(&st->counters[kCntAccepted], (u64)accepted);
+        if (status) atomicOr(&st->status, status);
+    }
+};
+
+// Eq. 4-6 for one row, by one thread, once the row's sums and best token are known: writes
+// the row's outputs and its accept bit / own token for the prefix rule.  d is the row's
+// draft id as given, xd its raw logit (read only when d lies inside the vocabulary).
 template <int DT>
-__device__ void verify_finish(const VerifyArgs& a, const RowJob& job, int64_t row, const char* rowp,
-                              const RowPartial& merged, float neg_refc, bool centered) {
-    const int d = __ldg(a.draft_ids + row);
+__device__ void verify_row(const VerifyArgs& a, const RowJob& job, int64_t row, const RowPartial& merged,
+                           float neg_refc, bool centered, int d, float xd, Tally& tally) {
     const bool d_ok = d >= 0 && d < job.vocab;
     const RowFinal f = finish_row(merged, job.c1, neg_refc, centered);
     const unsigned int flag = a.draft_flags ? a.draft_flags[row] : AASD_FLAG_CONDITIONAL;
@@ -330,11 +345,9 @@ __device__ void verify_finish(const VerifyArgs& a, const RowJob& job, int64_t ro
     const int own = f.top1;   // NONE on a bad row
     double pd = 0.0;
     bool acc = false, near = false;
-    unsigned int status = 0;
-    if (f.bad) status |= AASD_STATUS_BAD_ROW;
-    if (!d_ok && d != AASD_NONE) status |= AASD_STATUS_ID_RANGE;
+    if (f.bad) tally.status |= AASD_STATUS_BAD_ROW;
+    if (!d_ok && d != AASD_NONE) tally.status |= AASD_STATUS_ID_RANGE;
     if (d_ok && !f.bad) {
-        const float xd = Elt<DT>::load(rowp, d);
         pd = f.prob(xd);
         if (a.mode == AASD_VERIFY_CONDITIONAL && (flag & AASD_FLAG_CONDITIONAL)) {
             const bool at_max = (xd == f.m);
@@ -353,30 +366,46 @@ __device__ void verify_finish(const VerifyArgs& a, const RowJob& job, int64_t ro
     if (a.out.sampled) a.out.sampled[row] = AASD_NONE;
     a.row_accept[row] = acc ? 1 : 0;
     a.row_own[row] = own;
-    atomicAdd(&job.state->counters[kCntRows], 1ull);
-    if (f.bad) atomicAdd(&job.state->counters[kCntBad], 1ull);
-    if (near) atomicAdd(&job.state->counters[kCntNear], 1ull);
-    if (acc) atomicAdd(&job.state->counters[kCntAccepted], 1ull);
-    if (status) atomicOr(&job.state->status, status);
+    tally.rows += 1;
+    tally.bad += f.bad ? 1 : 0;
+    tally.near += near ? 1 : 0;
+    tally.accepted += acc ? 1 : 0;
+}
 
-    // The thread that finishes the last row of a candidate applies the prefix rule.
+// Candidate of a row and its row range; results of the empty candidates next to it (they
+// own no row, so a neighbour writes them).
+__device__ inline int candidate_of_row(const VerifyArgs& a, int64_t n_rows, int64_t row, int64_t& lo, int64_t& hi) {
     int c;
-    int64_t lo, hi;
     if (a.cand_offsets) {
         c = find_segment(a.cand_offsets, a.n_cands, row);
         lo = a.cand_offsets[c];
         hi = a.cand_offsets[c + 1];
-        // empty candidates own no row: their neighbours write their (empty) result
         if (row == lo)
             for (int e = c - 1; e >= 0 && a.cand_offsets[e] == a.cand_offsets[e + 1]; --e)
                 write_empty_candidate(a, e);
-        if (row == job.n_rows - 1)
+        if (row == n_rows - 1)
             for (int e = c + 1; e < a.n_cands; ++e) write_empty_candidate(a, e);
     } else {
         c = (int)(row / a.rows_per_cand);
         lo = (int64_t)c * a.rows_per_cand;
         hi = lo + a.rows_per_cand;
     }
+    return c;
+}
+
+// Row epilogue of the one-thread kernels: Eq. 4-6 for the row, then, in the thread that
+// completes a candidate, the prefix rule.
+template <int DT>
+__device__ void verify_finish(const VerifyArgs& a, const RowJob& job, int64_t row, const char* rowp,
+                              const RowPartial& merged, float neg_refc, bool centered) {
+    const int d = __ldg(a.draft_ids + row);
+    const float xd = (d >= 0 && d < job.vocab) ? Elt<DT>::load(rowp, d) : 0.f;
+    Tally tally;
+    tally.clear();
+    verify_row<DT>(a, job, row, merged, neg_refc, centered, d, xd, tally);
+    tally.flush(job.state);
+    int64_t lo, hi;
+    const int c = candidate_of_row(a, job.n_rows, row, lo, hi);
     __threadfence();
     const unsigned int t = atomicAdd(&a.cand_tickets[c], 1u);
     if (t != (unsigned int)(hi - lo) - 1u) return;
@@ -386,6 +415,44 @@ __device__ void verify_finish(const VerifyArgs& a, const RowJob& job, int64_t ro
     while (lo + n < hi && __ldcg(a.row_accept + lo + n)) ++n;
     if (a.out.accept_len) a.out.accept_len[c] = n;
     if (a.out.next_token) a.out.next_token[c] = (lo + n < hi) ? __ldcg(a.row_own + lo + n) : AASD_NONE;
+}
+
+// The same for the streaming kernel, run by a whole warp: lane 0 evaluates the row, and the
+// warp that completes a candidate scans its rows with one load per lane.
+template <int DT>
+__device__ void verify_finish_warp(const VerifyArgs& a, const RowJob& job, int64_t row, const RowPartial& merged,
+                                   float neg_refc, bool centered, int d, float xd, Tally& tally) {
+    const int lane = threadIdx.x & 31;
+    int c = 0, last = 0;
+    int64_t lo = 0, hi = 0;
+    if (lane == 0) {
+        verify_row<DT>(a, job, row, merged, neg_refc, centered, d, xd, tally);
+        c = candidate_of_row(a, job.n_rows, row, lo, hi);
+        __threadfence();
+        const unsigned int t = atomicAdd(&a.cand_tickets[c], 1u);
+        last = (t == (unsigned int)(hi - lo) - 1u);
+        if (last) a.cand_tickets[c] = 0;
+    }
+    last = __shfl_sync(0xFFFFFFFFu, last, 0);
+    if (!last) return;
+    c = __shfl_sync(0xFFFFFFFFu, c, 0);
+    lo = __shfl_sync(0xFFFFFFFFu, lo, 0);
+    hi = __shfl_sync(0xFFFFFFFFu, hi, 0);
+    __threadfence();
+    int64_t n = hi - lo;   // leading accepted rows
+    for (int64_t base = lo; base < hi; base += 32) {
+        const int64_t r = base + lane;
+        const bool stop = r < hi && __ldcg(a.row_accept + r) == 0;
+        const unsigned int bal = __ballot_sync(0xFFFFFFFFu, stop);
+        if (bal) {
+            n = base - lo + (__ffs(bal) - 1);
+            break;
+        }
+    }
+    if (lane == 0) {
+        if (a.out.accept_len) a.out.accept_len[c] = (int)n;
+        if (a.out.next_token) a.out.next_token[c] = (lo + n < hi) ? __ldcg(a.row_own + lo + n) : AASD_NONE;
+    }
 }
 
 // One CTA (or `chunks` CTAs) per row with plain vector / scalar loads: the path for logits
@@ -442,10 +509,9 @@ __global__ void align_next_kernel(const AlignArgs a) {
 }
 
 // Row epilogue of alignment sampling (Sec. 2.3 alignment test, Fig. 2 extras), one thread.
-template <int DT>
-__device__ void align_finish(const AlignArgs& a, const RowJob& job, int64_t row, const char* rowp,
-                             const RowPartial& merged, float neg_refc, bool centered) {
-    const int next = __ldg(a.next_ids + row);
+// next is the prompt's next token of the row (validated, or NONE), xn its raw logit.
+__device__ inline void align_row(const AlignArgs& a, const RowJob& job, int64_t row, const RowPartial& merged,
+                                 float neg_refc, bool centered, int next, float xn_in, Tally& tally) {
     const RowFinal f = finish_row(merged, job.c1, neg_refc, centered);
     const int KE = a.k_extra;
     int ids[kMaxK];
@@ -460,7 +526,7 @@ __device__ void align_finish(const AlignArgs& a, const RowJob& job, int64_t row,
     if (!f.bad) {
         float xn = 0.f;
         if (next != AASD_NONE) {
-            xn = Elt<DT>::load(rowp, next);
+            xn = xn_in;
             pn = f.prob(xn);
             aligned = (next == f.top1);
         }
@@ -487,11 +553,22 @@ __device__ void align_finish(const AlignArgs& a, const RowJob& job, int64_t row,
     if (a.out.entropy) a.out.entropy[row] = (float)f.H;
     if (a.out.pmax) a.out.pmax[row] = (float)f.pmax;
     if (a.out.aligned) a.out.aligned[row] = aligned ? 1 : 0;
-    atomicAdd(&job.state->counters[kCntRows], 1ull);
+    tally.rows += 1;
     if (f.bad) {
-        atomicAdd(&job.state->counters[kCntBad], 1ull);
-        atomicOr(&job.state->status, AASD_STATUS_BAD_ROW);
+        tally.bad += 1;
+        tally.status |= AASD_STATUS_BAD_ROW;
     }
+}
+
+template <int DT>
+__device__ void align_finish(const AlignArgs& a, const RowJob& job, int64_t row, const char* rowp,
+                             const RowPartial& merged, float neg_refc, bool centered) {
+    const int next = __ldg(a.next_ids + row);
+    const float xn = next != AASD_NONE ? Elt<DT>::load(rowp, next) : 0.f;
+    Tally tally;
+    tally.clear();
+    align_row(a, job, row, merged, neg_refc, centered, next, xn, tally);
+    tally.flush(job.state);
 }
 
 template <int DT, int K>

@@ -9,6 +9,12 @@
 // only meet at mbarriers, so the copies of the next rows are in flight while the current
 // row is being reduced and finished.
 //
+// Work is handed out dynamically: the producer claims the next work item from a counter in
+// global memory, so a CTA that runs on a slower path to memory simply takes fewer items.
+// An item is a whole row, or, when the host finds rows scarce, a piece of a row cut at tile
+// boundaries (rows [0, whole_rows) are whole, later rows are cut).  The pieces of a row meet
+// in global memory and the CTA that delivers the last one finishes the row.
+//
 // Every wait is bounded: a role that gives up raises AASD_STATUS_TIMEOUT, tells the other
 // roles through a shared flag and leaves; the producer first waits (bounded again) for the
 // copies it still has in flight.
@@ -24,6 +30,7 @@ constexpr int kConsumerWarps = 8;
 constexpr int kConsumers = kConsumerWarps * 32;
 constexpr int kStreamThreads = kConsumers + 64;   // + producer warp + finisher warp
 constexpr int kRing = 16;
+constexpr int kSlots = 4;                         // item results in flight between consumers and finisher
 constexpr unsigned int kWaitLimit = 1u << 24;     // polls of try_wait before giving up
 
 // ---- mbarrier / bulk copy primitives ---------------------------------------------------
@@ -81,8 +88,12 @@ __device__ __forceinline__ uint4 lds16(const void* p) {
 // ---- shared state of a streaming CTA -----------------------------------------------------
 struct ItemInfo {
     float neg_refc;   // -(reference * c1) of the item's row
-    int hint;         // hinted token of the row (validated), or NONE
+    int hint;         // hinted token of the row as given (may lie outside the vocabulary)
+    float hint_logit; // its raw logit when it lies inside
+    int row;          // logits row of the item; kNoItem: the work list is exhausted
+    int chunk;        // which piece of the row
 };
+constexpr int kNoItem = -1;
 struct WarpPartial {
     double S, A;
     u64 key[kMaxK];   // vector-level: (ordered vector maximum << 32) | ~vector index
@@ -90,21 +101,47 @@ struct WarpPartial {
 struct StreamShared {
     u64 full[kStages];
     u64 empty[kStages];
-    u64 done[2];
-    u64 freeb[2];
+    u64 done[kSlots];
+    u64 freeb[kSlots];
     ItemInfo ring[kRing];
-    WarpPartial wp[2][kConsumerWarps];
+    WarpPartial wp[kSlots][kConsumerWarps];
     int abort_flag;
 };
 constexpr size_t kStreamSmemBytes = (size_t)kStages * kTileBytes + sizeof(StreamShared) + 128;
 
 struct StreamJob {
-    RowJob row;               // logits, geometry, scratch (chunks = pieces per row)
+    RowJob row;               // logits, geometry, scratch
     const int32_t* hint_ids;  // [n_rows] token whose logit seeds the row's reference
+    unsigned int* sched;      // [2] next item, CTAs that have finished (both zero between launches)
     int tiles_per_row;
-    int tiles_per_chunk;
-    long long n_items;        // n_rows * chunks
+    int whole_rows;           // rows [0, whole_rows) are one item each
+    int tail_chunks;          // every later row is cut into this many pieces
+    long long n_items;        // whole_rows + (n_rows - whole_rows) * tail_chunks
 };
+
+// Work item -> (row, piece); pieces of a row are balanced ranges of its tiles.
+__device__ __forceinline__ void decode_item(const StreamJob& job, long long item, int& row, int& chunk) {
+    if (item < job.whole_rows) {
+        row = (int)item;
+        chunk = 0;
+    } else {
+        const long long j = item - job.whole_rows;
+        row = job.whole_rows + (int)(j / job.tail_chunks);
+        chunk = (int)(j % job.tail_chunks);
+    }
+}
+__device__ __forceinline__ int chunks_of(const StreamJob& job, int row) {
+    return row < job.whole_rows ? 1 : job.tail_chunks;
+}
+__device__ __forceinline__ void tile_range(const StreamJob& job, int row, int chunk, int& tb, int& te) {
+    if (row < job.whole_rows) {
+        tb = 0;
+        te = job.tiles_per_row;
+    } else {
+        tb = (int)(((long long)chunk * job.tiles_per_row) / job.tail_chunks);
+        te = (int)(((long long)(chunk + 1) * job.tiles_per_row) / job.tail_chunks);
+    }
+}
 
 __device__ __forceinline__ u64 make_vec_key(float vmax, int vec) {
     return ((u64)ordered_bits(vmax) << 32) | (u64)(0xFFFFFFFFu - (unsigned int)vec);
@@ -236,7 +273,7 @@ struct FinishedRow {
 };
 
 // Epilogue interface (static functions of a policy type E):
-//   E::finish(args, job, row, rowp, FinishedRow&)  - called by lane 0 of the finisher warp
+//   E::finish(args, job, row, FinishedRow&, ItemInfo&, Tally&)  - entered by the whole finisher warp
 template <int DT, int K, class E>
 __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJob job, const typename E::Args args) {
     extern __shared__ unsigned char smem_raw[];
@@ -247,7 +284,6 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
     const RowJob& rj = job.row;
-    const int chunks = rj.chunks;
     const float c1 = rj.c1;
     volatile int* abort_flag = &sh.abort_flag;
 
@@ -256,7 +292,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
             mbar_init(&sh.full[s], 1);
             mbar_init(&sh.empty[s], kConsumerWarps);
         }
-        for (int p = 0; p < 2; ++p) {
+        for (int p = 0; p < kSlots; ++p) {
             mbar_init(&sh.done[p], kConsumerWarps);
             mbar_init(&sh.freeb[p], 1);
         }
@@ -268,24 +304,32 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
     if (warp < kConsumerWarps) {
         // ------------------------------------------------------------------ consumers
         unsigned int it = 0, seq = 0;
-        for (long long item = blockIdx.x; item < job.n_items; item += gridDim.x, ++seq) {
-            const int chunk = (int)(item % chunks);
-            const int tb = chunk * job.tiles_per_chunk;
-            const int te = min(job.tiles_per_row, tb + job.tiles_per_chunk);
+        for (;; ++seq) {
             TileAccumulator<DT, K> acc;
             acc.init();
             float neg_refc = 0.f;
-            bool alive = true;
-            for (int t = tb; t < te; ++t, ++it) {
+            bool alive = true, last = false;
+            int tb = 0, te = 1;
+            for (int t = 0; t < te - tb; ++t, ++it) {
                 const int s = it % kStages;
                 if (!mbar_wait(&sh.full[s], (it / kStages) & 1u, abort_flag)) {
                     if (lane == 0) give_up(abort_flag, rj.state);
                     alive = false;
                     break;
                 }
-                if (t == tb) neg_refc = sh.ring[seq % kRing].neg_refc;
+                if (t == 0) {
+                    // the item's record was written before its first tile was announced
+                    const ItemInfo info = sh.ring[seq % kRing];
+                    if (info.row == kNoItem) {
+                        last = true;
+                        ++it;
+                        break;
+                    }
+                    neg_refc = info.neg_refc;
+                    tile_range(job, info.row, info.chunk, tb, te);
+                }
                 const unsigned char* base = tiles + (size_t)s * kTileBytes;
-                const int v0 = t * kTileVecs;
+                const int v0 = (tb + t) * kTileVecs;
                 const int nv = min(kTileVecs, rj.nvec - v0);
                 if (nv == kTileVecs) {
                     uint4 q[kTileVecs / kConsumers];
@@ -323,9 +367,13 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
                     vk[K - 1] = 0;
                 }
             }
-            const int p = seq & 1;
-            if (!mbar_wait(&sh.freeb[p], ((seq >> 1) & 1u) ^ 1u, abort_flag)) {
+            const int p = seq % kSlots;
+            if (!mbar_wait(&sh.freeb[p], ((seq / kSlots) & 1u) ^ 1u, abort_flag)) {
                 if (lane == 0) give_up(abort_flag, rj.state);
+                break;
+            }
+            if (last) {
+                if (lane == 0) mbar_arrive(&sh.done[p]);   // wakes the finisher, which sees the end too
                 break;
             }
             if (lane == 0) {
@@ -345,16 +393,43 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
         unsigned int it = 0, seq = 0;
         unsigned int armed = 0;   // bit s: a copy into stage s was issued in the current use
         bool alive = true;
-        for (long long item = blockIdx.x; item < job.n_items && alive; item += gridDim.x, ++seq) {
-            const long long row = item / chunks;
-            const int chunk = (int)(item % chunks);
+        // The first item of a CTA is its own index (the grid never exceeds the item count);
+        // later ones come from the counter, claimed one ahead so that its round trip is
+        // hidden behind the copies of the current item.
+        long long next = blockIdx.x;
+        for (; alive; ++seq) {
+            const long long item = next;
+            if (item >= job.n_items) {
+                // end of the work list: an empty stage use tells the consumers
+                if (lane == 0) {
+                    const int s = it % kStages;
+                    if (mbar_wait(&sh.empty[s], ((it / kStages) & 1u) ^ 1u, abort_flag)) {
+                        sh.ring[seq % kRing].row = kNoItem;
+                        mbar_arrive(&sh.full[s]);
+                        // the last CTA to get here leaves the counters ready for the next launch
+                        __threadfence();
+                        if (atomicAdd(job.sched + 1, 1u) == gridDim.x - 1) {
+                            job.sched[0] = 0;
+                            job.sched[1] = 0;
+                        }
+                    } else {
+                        alive = false;
+                    }
+                }
+                alive = __shfl_sync(0xFFFFFFFFu, alive ? 1 : 0, 0) != 0;
+                break;
+            }
+            if (lane == 0) next = (long long)gridDim.x + (long long)atomicAdd(job.sched, 1u);
+            int row, chunk;
+            decode_item(job, item, row, chunk);
             const char* rowp = row_pointer<DT>(rj, row);
             // reference of the row: its hinted logit and its first entries
-            int hint = __ldg(job.hint_ids + row);
-            if (hint < 0 || hint >= rj.vocab) hint = AASD_NONE;
+            const int hint = __ldg(job.hint_ids + row);
+            const bool hint_ok = hint >= 0 && hint < rj.vocab;
             float r = -CUDART_INF_F;
             if (lane < 4 && lane < rj.vocab) r = Elt<DT>::load(rowp, lane);
-            if (lane == 4 && hint >= 0) r = Elt<DT>::load(rowp, hint);
+            if (lane == 4 && hint_ok) r = Elt<DT>::load(rowp, hint);
+            const float hint_logit = __shfl_sync(0xFFFFFFFFu, r, 4);
 #pragma unroll
             for (int o = 4; o > 0; o >>= 1) r = fmaxf(r, __shfl_xor_sync(0xFFFFFFFFu, r, o));
             r = __shfl_sync(0xFFFFFFFFu, r, 0);
@@ -363,8 +438,11 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
                 ItemInfo& info = sh.ring[seq % kRing];
                 info.neg_refc = -(r * c1);
                 info.hint = hint;
-                const int tb = chunk * job.tiles_per_chunk;
-                const int te = min(job.tiles_per_row, tb + job.tiles_per_chunk);
+                info.hint_logit = hint_logit;
+                info.row = row;
+                info.chunk = chunk;
+                int tb, te;
+                tile_range(job, row, chunk, tb, te);
                 for (int t = tb; t < te; ++t, ++it) {
                     const int s = it % kStages;
                     if (!mbar_wait(&sh.empty[s], ((it / kStages) & 1u) ^ 1u, abort_flag)) {
@@ -380,6 +458,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
                 }
             }
             alive = __shfl_sync(0xFFFFFFFFu, alive ? 1 : 0, 0) != 0;
+            next = __shfl_sync(0xFFFFFFFFu, next, 0);
         }
         if (!alive && lane == 0) {
             // give the copies still in flight a bounded time to land before the CTA leaves
@@ -397,16 +476,20 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
     }
 
     // ------------------------------------------------------------------------- finisher
-    unsigned int seq = 0;
-    for (long long item = blockIdx.x; item < job.n_items; item += gridDim.x, ++seq) {
-        const long long row = item / chunks;
-        const int chunk = (int)(item % chunks);
-        const char* rowp = row_pointer<DT>(rj, row);
-        const int p = seq & 1;
-        if (!mbar_wait(&sh.done[p], (seq >> 1) & 1u, abort_flag)) {
+    Tally tally;   // lane 0's running counters, flushed when the CTA leaves
+    tally.clear();
+    for (unsigned int seq = 0;; ++seq) {
+        const int p = seq % kSlots;
+        if (!mbar_wait(&sh.done[p], (seq / kSlots) & 1u, abort_flag)) {
             if (lane == 0) give_up(abort_flag, rj.state);
-            return;
+            break;
         }
+        const ItemInfo info = sh.ring[seq % kRing];
+        if (info.row == kNoItem) break;
+        const long long row = info.row;
+        const int chunk = info.chunk;
+        const int chunks = chunks_of(job, info.row);
+        const char* rowp = row_pointer<DT>(rj, row);
         double S = 0.0, A = 0.0;
         u64 vk[K];
 #pragma unroll
@@ -418,7 +501,6 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
 #pragma unroll
             for (int j = 0; j < K; ++j) vk[j] = w.key[j];
         }
-        const ItemInfo info = sh.ring[seq % kRing];
         __syncwarp();
         if (lane == 0) mbar_arrive(&sh.freeb[p]);
         S = warp_sum_f64(S);
@@ -436,7 +518,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
         }
         if (chunks > 1) {
             // pieces of a row meet in global memory; the last one to arrive carries on
-            RowPartial* slots = rj.partials + row * chunks;
+            RowPartial* slots = rj.partials + (row - job.whole_rows) * chunks;
             int last = 0;
             if (lane == 0) {
                 RowPartial mine;
@@ -532,29 +614,33 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
                 warp_row_centered<DT>(rowp, rj.vocab, m, c1, S, A);
                 fr.neg_refc = -m;
                 fr.centered = true;
-                if (lane == 0) atomicAdd(&rj.state->counters[kCntRedo], 1ull);
+                tally.redo += 1;
             }
         }
         fr.merged.S = S;
         fr.merged.A = A;
-        if (lane == 0) E::finish(args, rj, row, rowp, fr);
+        E::finish(args, rj, row, fr, info, tally);
     }
+    if (lane == 0) tally.flush(rj.state);
 }
 
+// Epilogues are entered by the whole finisher warp.
 template <int DT>
 struct VerifyEpilogue {
     using Args = VerifyArgs;
-    static __device__ void finish(const VerifyArgs& a, const RowJob& job, int64_t row, const char* rowp,
-                                  const FinishedRow& fr) {
-        verify_finish<DT>(a, job, row, rowp, fr.merged, fr.neg_refc, fr.centered);
+    static __device__ void finish(const VerifyArgs& a, const RowJob& job, int64_t row, const FinishedRow& fr,
+                                  const ItemInfo& info, Tally& tally) {
+        verify_finish_warp<DT>(a, job, row, fr.merged, fr.neg_refc, fr.centered, info.hint, info.hint_logit, tally);
     }
 };
 template <int DT>
 struct AlignEpilogue {
     using Args = AlignArgs;
-    static __device__ void finish(const AlignArgs& a, const RowJob& job, int64_t row, const char* rowp,
-                                  const FinishedRow& fr) {
-        align_finish<DT>(a, job, row, rowp, fr.merged, fr.neg_refc, fr.centered);
+    static __device__ void finish(const AlignArgs& a, const RowJob& job, int64_t row, const FinishedRow& fr,
+                                  const ItemInfo& info, Tally& tally) {
+        // next_ids holds validated tokens only
+        if ((threadIdx.x & 31) == 0)
+            align_row(a, job, row, fr.merged, fr.neg_refc, fr.centered, info.hint, info.hint_logit, tally);
     }
 };
 
