@@ -22,7 +22,7 @@ namespace {
 struct WorkspaceLayout {
     size_t bytes;
     int64_t max_rows, max_cands;
-    size_t off_partials, off_row_tickets, off_cand_tickets, off_sched, off_row_accept, off_row_own, off_next;
+    size_t off_partials, off_row_tickets, off_cand_tickets, off_sched, off_row_accept, off_row_own, off_next, off_race;
 };
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -46,6 +46,8 @@ WorkspaceLayout make_layout(int64_t max_rows, int64_t max_cands) {
     o = align_up(o + 4 * (size_t)max_rows, 256);
     L.off_next = o;
     o = align_up(o + 4 * (size_t)max_rows, 256);
+    L.off_race = o;
+    o = align_up(o + sizeof(RaceSummary) * (size_t)kRaceSlots * kMaxK, 256);
     L.bytes = o;
     return L;
 }
@@ -105,6 +107,7 @@ int plan_rows(aasd_ctx* ctx, RowJob& job, const void* logits, int dtype, int voc
     job.vocab = vocab;
     job.vector_ok = ((uintptr_t)logits % 16 == 0) && ((row_stride * esize) % 16 == 0);
     job.nvec = job.vector_ok ? vocab / vec : 0;
+    job.vec_elts = vec;
     job.c1 = inv_temperature * kLog2e;
     // Fill the machine: aim at eight CTAs per SM, but keep at least one sweep of the CTA
     // per chunk and stay within the partial-record slots of the workspace.
@@ -134,10 +137,13 @@ int plan_rows(aasd_ctx* ctx, RowJob& job, const void* logits, int dtype, int voc
 // per SM that claim work items from a counter.  An item is a whole row unless there are
 // fewer rows than CTA slots; then every row is cut into pieces at tile boundaries.
 void plan_stream(aasd_ctx* ctx, StreamJob& sj, const RowJob& job, const int32_t* hint_ids, char* ws,
-                 const WorkspaceLayout& L, unsigned int* grid) {
+                 const WorkspaceLayout& L, const SampleJob* smp, unsigned int* grid) {
     sj.row = job;
     sj.hint_ids = hint_ids;
     sj.sched = reinterpret_cast<unsigned int*>(ws + L.off_sched);
+    sj.race_partials = reinterpret_cast<RaceSummary*>(ws + L.off_race);
+    sj.full_groups = (int)(((int64_t)job.nvec * job.vec_elts) / kGroup);
+    if (smp) sj.smp = *smp;
     const int64_t row_bytes = (int64_t)job.nvec * 16;
     const int tiles = (int)((row_bytes + kTileBytes - 1) / kTileBytes);
     const int64_t slots = (int64_t)ctx->sm_count * 2;
@@ -160,7 +166,11 @@ void plan_stream(aasd_ctx* ctx, StreamJob& sj, const RowJob& job, const int32_t*
         chunks = 1;
         tail_rows = 0;
     }
-    while (tail_rows * chunks > kPartialSlots) --tail_rows;
+    while (chunks > 1 && tail_rows * chunks > (smp ? kRaceSlots : kPartialSlots)) --chunks;
+    if (chunks <= 1) {
+        chunks = 1;
+        tail_rows = 0;
+    }
     sj.tiles_per_row = tiles;
     sj.whole_rows = (int)(job.n_rows - tail_rows);
     sj.tail_chunks = (int)chunks;
@@ -176,20 +186,52 @@ int enable_stream_smem(Kernel kernel) {
                : AASD_ERR_CUDA;
 }
 
-template <int DT, int K>
+template <int DT, int K, int ND>
 int launch_align_stream(aasd_ctx* ctx, const StreamJob& sj, const AlignArgs& a, unsigned int grid) {
-    auto kernel = stream_kernel<DT, K, AlignEpilogue<DT>>;
+    auto kernel = stream_kernel<DT, K, ND, AlignEpilogue<DT>>;
+    if (enable_stream_smem(kernel) != AASD_OK) return AASD_ERR_CUDA;
+    kernel<<<grid, kStreamThreads, kStreamSmemBytes, ctx->stream>>>(sj, a);
+    return AASD_OK;
+}
+
+// TOPK mode keeps the K best tokens and draws nothing; GUMBEL mode needs the best token
+// only (for the alignment test) and prepares ND >= k_extra draws.
+template <int DT>
+int dispatch_align_stream(aasd_ctx* ctx, const StreamJob& sj, const AlignArgs& a, unsigned int grid) {
+    const int k = a.k_extra <= 1 ? 1 : (a.k_extra == 2 ? 2 : 4);
+    if (a.mode == AASD_ALIGN_GUMBEL && a.k_extra > 0) {
+        if (k == 1) return launch_align_stream<DT, 1, 1>(ctx, sj, a, grid);
+        if (k == 2) return launch_align_stream<DT, 1, 2>(ctx, sj, a, grid);
+        return launch_align_stream<DT, 1, 4>(ctx, sj, a, grid);
+    }
+    if (k == 1) return launch_align_stream<DT, 1, 0>(ctx, sj, a, grid);
+    if (k == 2) return launch_align_stream<DT, 2, 0>(ctx, sj, a, grid);
+    return launch_align_stream<DT, 4, 0>(ctx, sj, a, grid);
+}
+
+template <int DT, int ND>
+int launch_verify_stream(aasd_ctx* ctx, const StreamJob& sj, const VerifyArgs& a, unsigned int grid) {
+    auto kernel = stream_kernel<DT, 1, ND, VerifyEpilogue<DT>>;
     if (enable_stream_smem(kernel) != AASD_OK) return AASD_ERR_CUDA;
     kernel<<<grid, kStreamThreads, kStreamSmemBytes, ctx->stream>>>(sj, a);
     return AASD_OK;
 }
 
 template <int DT>
-int launch_verify_stream(aasd_ctx* ctx, const StreamJob& sj, const VerifyArgs& a, unsigned int grid) {
-    auto kernel = stream_kernel<DT, 1, VerifyEpilogue<DT>>;
-    if (enable_stream_smem(kernel) != AASD_OK) return AASD_ERR_CUDA;
-    kernel<<<grid, kStreamThreads, kStreamSmemBytes, ctx->stream>>>(sj, a);
-    return AASD_OK;
+int dispatch_verify_stream(aasd_ctx* ctx, const StreamJob& sj, const VerifyArgs& a, unsigned int grid) {
+    return a.mode == AASD_VERIFY_STRICT_SAMPLED ? launch_verify_stream<DT, 1>(ctx, sj, a, grid)
+                                                : launch_verify_stream<DT, 0>(ctx, sj, a, grid);
+}
+
+SampleJob make_sample_job(uint64_t seed, uint32_t step, bool align, float inv_temperature) {
+    SampleJob s{};
+    s.key0 = (unsigned int)(seed & 0xFFFFFFFFull);
+    s.key1 = (unsigned int)(seed >> 32);
+    s.step = step;
+    s.dom_group = align ? kDomAlignGroup : kDomVerifyGroup;
+    s.dom_elem = align ? kDomAlignElem : kDomVerifyElem;
+    s.inv_t = inv_temperature;
+    return s;
 }
 
 }  // namespace
@@ -308,7 +350,6 @@ int aasd_align_sample(aasd_ctx* ctx, const void* prefill_logits, const int32_t* 
     if (n_seqs < 0 || n_rows < 0) return AASD_ERR_BAD_SHAPE;
     if (p->k_extra < 0 || p->k_extra > AASD_MAX_EXTRA) return AASD_ERR_INVALID_ARG;
     if (p->mode != AASD_ALIGN_TOPK && p->mode != AASD_ALIGN_GUMBEL) return AASD_ERR_INVALID_ARG;
-    if (p->mode == AASD_ALIGN_GUMBEL) return AASD_ERR_UNSUPPORTED;
     if (n_rows > 0 && (prompt_ids == nullptr || seq_offsets == nullptr || n_seqs == 0)) return AASD_ERR_INVALID_ARG;
     int err = AASD_OK;
     const WorkspaceLayout* L = find_workspace(ctx, workspace, workspace_bytes, n_rows, 0, &err);
@@ -325,24 +366,20 @@ int aasd_align_sample(aasd_ctx* ctx, const void* prefill_logits, const int32_t* 
     a.k_extra = p->k_extra;
     a.mode = p->mode;
     a.next_ids = reinterpret_cast<int32_t*>(ws + L->off_next);
+    a.smp = make_sample_job(p->seed, p->stream_tag, true, p->inv_temperature);
     a.out = *out;
     AASD_CUDA(cudaSetDevice(ctx->device));
     align_next_kernel<<<(unsigned int)((n_rows + 255) / 256), 256, 0, ctx->stream>>>(a);
-    const int K = p->k_extra <= 1 ? 1 : (p->k_extra == 2 ? 2 : 4);
+    // plain kernels: the K best tokens in TOPK mode, the best token alone in GUMBEL mode
+    const int K = (p->k_extra <= 1 || p->mode == AASD_ALIGN_GUMBEL) ? 1 : (p->k_extra == 2 ? 2 : 4);
     if (a.job.vector_ok && a.job.nvec > 0) {
         // 16-byte aligned rows: persistent TMA-fed streaming kernel
         StreamJob sj{};
         unsigned int grid = 0;
-        plan_stream(ctx, sj, a.job, a.next_ids, ws, *L, &grid);
-        int rc;
-        if (p->dtype == AASD_F32)
-            rc = K == 1 ? launch_align_stream<AASD_F32, 1>(ctx, sj, a, grid)
-                        : (K == 2 ? launch_align_stream<AASD_F32, 2>(ctx, sj, a, grid)
-                                  : launch_align_stream<AASD_F32, 4>(ctx, sj, a, grid));
-        else
-            rc = K == 1 ? launch_align_stream<AASD_BF16, 1>(ctx, sj, a, grid)
-                        : (K == 2 ? launch_align_stream<AASD_BF16, 2>(ctx, sj, a, grid)
-                                  : launch_align_stream<AASD_BF16, 4>(ctx, sj, a, grid));
+        const bool draws = p->mode == AASD_ALIGN_GUMBEL && p->k_extra > 0;
+        plan_stream(ctx, sj, a.job, a.next_ids, ws, *L, draws ? &a.smp : nullptr, &grid);
+        const int rc = p->dtype == AASD_F32 ? dispatch_align_stream<AASD_F32>(ctx, sj, a, grid)
+                                            : dispatch_align_stream<AASD_BF16>(ctx, sj, a, grid);
         if (rc != AASD_OK) return rc;
         return after_launch(ctx, 2);
     }
@@ -384,7 +421,6 @@ int aasd_verify(aasd_ctx* ctx, const void* target_logits, const int32_t* draft_i
     if (ctx == nullptr || p == nullptr || out == nullptr) return AASD_ERR_INVALID_ARG;
     if (n_cands < 0 || n_rows < 0) return AASD_ERR_BAD_SHAPE;
     if (p->mode < AASD_VERIFY_CONDITIONAL || p->mode > AASD_VERIFY_STRICT_SAMPLED) return AASD_ERR_INVALID_ARG;
-    if (p->mode == AASD_VERIFY_STRICT_SAMPLED) return AASD_ERR_UNSUPPORTED;
     if (!(p->alpha >= 0.f) || !(p->beta >= 0.f)) return AASD_ERR_INVALID_ARG;
     if (cand_offsets == nullptr) {
         if (p->rows_per_cand < 1 || (int64_t)n_cands * p->rows_per_cand != n_rows) return AASD_ERR_BAD_SHAPE;
@@ -409,6 +445,7 @@ int aasd_verify(aasd_ctx* ctx, const void* target_logits, const int32_t* draft_i
     a.cand_tickets = reinterpret_cast<unsigned int*>(ws + L->off_cand_tickets);
     a.row_accept = reinterpret_cast<uint8_t*>(ws + L->off_row_accept);
     a.row_own = reinterpret_cast<int32_t*>(ws + L->off_row_own);
+    a.smp = make_sample_job(p->seed, p->step, false, p->inv_temperature);
     a.out = *out;
     AASD_CUDA(cudaSetDevice(ctx->device));
     if (n_rows == 0) {
@@ -419,9 +456,9 @@ int aasd_verify(aasd_ctx* ctx, const void* target_logits, const int32_t* draft_i
     if (a.job.vector_ok && a.job.nvec > 0) {
         StreamJob sj{};
         unsigned int sgrid = 0;
-        plan_stream(ctx, sj, a.job, draft_ids, ws, *L, &sgrid);
-        const int rc = p->dtype == AASD_F32 ? launch_verify_stream<AASD_F32>(ctx, sj, a, sgrid)
-                                            : launch_verify_stream<AASD_BF16>(ctx, sj, a, sgrid);
+        plan_stream(ctx, sj, a.job, draft_ids, ws, *L, p->mode == AASD_VERIFY_STRICT_SAMPLED ? &a.smp : nullptr, &sgrid);
+        const int rc = p->dtype == AASD_F32 ? dispatch_verify_stream<AASD_F32>(ctx, sj, a, sgrid)
+                                            : dispatch_verify_stream<AASD_BF16>(ctx, sj, a, sgrid);
         if (rc != AASD_OK) return rc;
         return after_launch(ctx, 1);
     }
@@ -499,7 +536,8 @@ constexpr size_t kStaticWorkspaceBytes =
     ((4 * (size_t)kStaticMaxCands + 255) / 256 * 256) +                  // candidate tickets
     256 +                                                                // work-item counters
     (((size_t)kStaticMaxRows + 255) / 256 * 256) +                       // accept bits
-    2 * ((4 * (size_t)kStaticMaxRows + 255) / 256 * 256);                // own tokens, next ids
+    2 * ((4 * (size_t)kStaticMaxRows + 255) / 256 * 256) +               // own tokens, next ids
+    ((sizeof(RaceSummary) * (size_t)kRaceSlots * kMaxK + 255) / 256 * 256);   // sampler records of cut rows
 constexpr size_t kStaticBytes = kStaticWorkspaceBytes + 256;
 
 }  // namespace
@@ -529,7 +567,6 @@ extern "C" int aasd_verify_static(int device, void* stream, const void* target_l
     if (n_cands < 0 || n_rows < 0) return AASD_ERR_BAD_SHAPE;
     if (n_rows > kStaticMaxRows || n_cands > kStaticMaxCands) return AASD_ERR_WORKSPACE_TOO_SMALL;
     if (p->mode < AASD_VERIFY_CONDITIONAL || p->mode > AASD_VERIFY_STRICT_SAMPLED) return AASD_ERR_INVALID_ARG;
-    if (p->mode == AASD_VERIFY_STRICT_SAMPLED) return AASD_ERR_UNSUPPORTED;
     if (!(p->alpha >= 0.f) || !(p->beta >= 0.f)) return AASD_ERR_INVALID_ARG;
     if (cand_offsets == nullptr) {
         if (p->rows_per_cand < 1 || (int64_t)n_cands * p->rows_per_cand != n_rows) return AASD_ERR_BAD_SHAPE;
@@ -583,15 +620,16 @@ extern "C" int aasd_verify_static(int device, void* stream, const void* target_l
     a.cand_tickets = reinterpret_cast<unsigned int*>(ws + L.off_cand_tickets);
     a.row_accept = reinterpret_cast<uint8_t*>(ws + L.off_row_accept);
     a.row_own = reinterpret_cast<int32_t*>(ws + L.off_row_own);
+    a.smp = make_sample_job(p->seed, p->step, false, p->inv_temperature);
     a.out = *out;
     if (n_rows == 0) {
         if (n_cands > 0) verify_empty_kernel<<<(unsigned int)((n_cands + 255) / 256), 256, 0, s>>>(a);
     } else if (a.job.vector_ok && a.job.nvec > 0) {
         StreamJob sj{};
         unsigned int sgrid = 0;
-        plan_stream(&local, sj, a.job, draft_ids, ws, L, &sgrid);
-        const int rc = p->dtype == AASD_F32 ? launch_verify_stream<AASD_F32>(&local, sj, a, sgrid)
-                                            : launch_verify_stream<AASD_BF16>(&local, sj, a, sgrid);
+        plan_stream(&local, sj, a.job, draft_ids, ws, L, p->mode == AASD_VERIFY_STRICT_SAMPLED ? &a.smp : nullptr, &sgrid);
+        const int rc = p->dtype == AASD_F32 ? dispatch_verify_stream<AASD_F32>(&local, sj, a, sgrid)
+                                            : dispatch_verify_stream<AASD_BF16>(&local, sj, a, sgrid);
         if (rc != AASD_OK) return rc;
     } else {
         const unsigned int grid = (unsigned int)(n_rows * a.job.chunks);

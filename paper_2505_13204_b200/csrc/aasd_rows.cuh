@@ -2,6 +2,7 @@
 #pragma once
 
 #include "aasd_device.cuh"
+#include "aasd_sampler.cuh"
 
 namespace aasd {
 
@@ -13,6 +14,7 @@ struct RowJob {
     int vocab;
     int vector_ok;          // rows are 16-byte aligned: take the vector path
     int nvec;               // whole vectors per row (vector path)
+    int vec_elts;           // logits per 16-byte vector
     int chunks;             // CTAs per row
     int vec_per_chunk;      // vectors per chunk (multiple of 8)
     float c1;               // inv_temperature * log2(e)
@@ -262,6 +264,12 @@ struct RowFinal {
     }
 };
 
+// A row is bad when it held NaN or +inf, or nothing but -inf.
+__device__ inline bool partial_bad(const RowPartial& p) {
+    const float m = key_value(p.key[0]);
+    return (p.key[0] == 0) || !(fabsf(m) <= 3.0e38f) || !(p.S > 0.0) || !(p.S <= 1.0e300) || !(fabs(p.A) <= 1.0e300);
+}
+
 __device__ inline RowFinal finish_row(const RowPartial& p, float c1, float neg_refc, bool centered) {
     RowFinal f;
     f.c1 = (double)c1;
@@ -270,8 +278,7 @@ __device__ inline RowFinal finish_row(const RowPartial& p, float c1, float neg_r
     f.m = key_value(p.key[0]);
     f.top1 = key_id(p.key[0]);
     f.S = p.S;
-    f.bad = (p.key[0] == 0) || !(fabsf(f.m) <= 3.0e38f) || !(p.S > 0.0) || !(p.S <= 1.0e300) ||
-            !(fabs(p.A) <= 1.0e300);
+    f.bad = partial_bad(p);
     if (f.bad) {
         f.top1 = AASD_NONE;
         f.H = 0.0;
@@ -298,6 +305,7 @@ struct VerifyArgs {
     unsigned int* cand_tickets;
     uint8_t* row_accept;           // scratch [n_rows]
     int32_t* row_own;              // scratch [n_rows]
+    SampleJob smp;                 // STRICT_SAMPLED: the row's own token is a keyed draw
     aasd_verify_out out;
 };
 
@@ -319,30 +327,33 @@ __device__ inline void write_empty_candidate(const VerifyArgs& a, int c) {
 // What a finished row adds to the running counters and the status word.  The streaming
 // kernel keeps one per CTA in registers and flushes it when the CTA leaves.
 struct Tally {
-    unsigned int rows, bad, redo, near, accepted, status;
-    __device__ void clear() { rows = bad = redo = near = accepted = status = 0; }
+    unsigned int rows, bad, redo, near, accepted, recheck, exhaustive, status;
+    __device__ void clear() { rows = bad = redo = near = accepted = recheck = exhaustive = status = 0; }
     __device__ void flush(DeviceState* st) const {
         if (rows) atomicAdd(&st->counters[kCntRows], (u64)rows);
         if (bad) atomicAdd(&st->counters[kCntBad], (u64)bad);
         if (redo) atomicAdd(&st->counters[kCntRedo], (u64)redo);
         if (near) atomicAdd(&st->counters[kCntNear], (u64)near);
         if (accepted) atomicAdd(&st->counters[kCntAccepted], (u64)accepted);
+        if (recheck) atomicAdd(&st->counters[kCntRecheck], (u64)recheck);
+        if (exhaustive) atomicAdd(&st->counters[kCntExact], (u64)exhaustive);
         if (status) atomicOr(&st->status, status);
     }
 };
 
 // Eq. 4-6 for one row, by one thread, once the row's sums and best token are known: writes
 // the row's outputs and its accept bit / own token for the prefix rule.  d is the row's
-// draft id as given, xd its raw logit (read only when d lies inside the vocabulary).
+// draft id as given, xd its raw logit (read only when d lies inside the vocabulary), sampled
+// the row's keyed draw in STRICT_SAMPLED mode (NONE otherwise, and on a bad row).
 template <int DT>
 __device__ void verify_row(const VerifyArgs& a, const RowJob& job, int64_t row, const RowPartial& merged,
-                           float neg_refc, bool centered, int d, float xd, Tally& tally) {
+                           float neg_refc, bool centered, int d, float xd, int sampled, Tally& tally) {
     const bool d_ok = d >= 0 && d < job.vocab;
     const RowFinal f = finish_row(merged, job.c1, neg_refc, centered);
     const unsigned int flag = a.draft_flags ? a.draft_flags[row] : AASD_FLAG_CONDITIONAL;
     const double lin = (double)a.alpha * f.H + (double)a.beta;
     const double thr = f.bad ? 0.0 : fmin(lin, f.pmax);
-    const int own = f.top1;   // NONE on a bad row
+    const int own = a.mode == AASD_VERIFY_STRICT_SAMPLED ? sampled : f.top1;   // NONE on a bad row
     double pd = 0.0;
     bool acc = false, near = false;
     if (f.bad) tally.status |= AASD_STATUS_BAD_ROW;
@@ -363,7 +374,7 @@ __device__ void verify_row(const VerifyArgs& a, const RowJob& job, int64_t row, 
     if (a.out.argmax) a.out.argmax[row] = f.top1;
     if (a.out.threshold) a.out.threshold[row] = (float)thr;
     if (a.out.accept) a.out.accept[row] = acc ? 1 : 0;
-    if (a.out.sampled) a.out.sampled[row] = AASD_NONE;
+    if (a.out.sampled) a.out.sampled[row] = f.bad ? AASD_NONE : sampled;
     a.row_accept[row] = acc ? 1 : 0;
     a.row_own[row] = own;
     tally.rows += 1;
@@ -393,40 +404,16 @@ __device__ inline int candidate_of_row(const VerifyArgs& a, int64_t n_rows, int6
     return c;
 }
 
-// Row epilogue of the one-thread kernels: Eq. 4-6 for the row, then, in the thread that
-// completes a candidate, the prefix rule.
-template <int DT>
-__device__ void verify_finish(const VerifyArgs& a, const RowJob& job, int64_t row, const char* rowp,
-                              const RowPartial& merged, float neg_refc, bool centered) {
-    const int d = __ldg(a.draft_ids + row);
-    const float xd = (d >= 0 && d < job.vocab) ? Elt<DT>::load(rowp, d) : 0.f;
-    Tally tally;
-    tally.clear();
-    verify_row<DT>(a, job, row, merged, neg_refc, centered, d, xd, tally);
-    tally.flush(job.state);
-    int64_t lo, hi;
-    const int c = candidate_of_row(a, job.n_rows, row, lo, hi);
-    __threadfence();
-    const unsigned int t = atomicAdd(&a.cand_tickets[c], 1u);
-    if (t != (unsigned int)(hi - lo) - 1u) return;
-    __threadfence();
-    a.cand_tickets[c] = 0;
-    int n = 0;
-    while (lo + n < hi && __ldcg(a.row_accept + lo + n)) ++n;
-    if (a.out.accept_len) a.out.accept_len[c] = n;
-    if (a.out.next_token) a.out.next_token[c] = (lo + n < hi) ? __ldcg(a.row_own + lo + n) : AASD_NONE;
-}
-
-// The same for the streaming kernel, run by a whole warp: lane 0 evaluates the row, and the
-// warp that completes a candidate scans its rows with one load per lane.
+// Row epilogue of verification, run by a whole warp: lane 0 evaluates the row (Eq. 4-6), and
+// the warp that completes a candidate applies the prefix rule with one load per lane.
 template <int DT>
 __device__ void verify_finish_warp(const VerifyArgs& a, const RowJob& job, int64_t row, const RowPartial& merged,
-                                   float neg_refc, bool centered, int d, float xd, Tally& tally) {
+                                   float neg_refc, bool centered, int d, float xd, int sampled, Tally& tally) {
     const int lane = threadIdx.x & 31;
     int c = 0, last = 0;
     int64_t lo = 0, hi = 0;
     if (lane == 0) {
-        verify_row<DT>(a, job, row, merged, neg_refc, centered, d, xd, tally);
+        verify_row<DT>(a, job, row, merged, neg_refc, centered, d, xd, sampled, tally);
         c = candidate_of_row(a, job.n_rows, row, lo, hi);
         __threadfence();
         const unsigned int t = atomicAdd(&a.cand_tickets[c], 1u);
@@ -469,8 +456,18 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(const VerifyArgs a) {
     float neg_refc;
     bool centered;
     if (!row_reduce<DT, 1>(job, row, chunk, d_ok ? d : -1, rowp, neg_refc, centered, sc)) return;
-    if (threadIdx.x != 0) return;
-    verify_finish<DT>(a, job, row, rowp, sc.merged, neg_refc, centered);
+    if (threadIdx.x >= 32) return;
+    const float xd = d_ok ? Elt<DT>::load(rowp, d) : 0.f;
+    Tally tally;
+    tally.clear();
+    int sampled = AASD_NONE;
+    if (a.mode == AASD_VERIFY_STRICT_SAMPLED && !partial_bad(sc.merged)) {
+        // this layout takes the definition as it stands: every group scored in fp64
+        sampled = warp_sample_exhaustive<DT>(rowp, job.vocab, (unsigned int)row, 0, a.smp);
+        tally.exhaustive += 1;
+    }
+    verify_finish_warp<DT>(a, job, row, sc.merged, neg_refc, centered, d, xd, sampled, tally);
+    if (threadIdx.x == 0) tally.flush(job.state);
 }
 
 // Candidates of a call without rows.
@@ -489,6 +486,7 @@ struct AlignArgs {
     int k_extra;
     int mode;
     int32_t* next_ids;   // scratch [n_rows]: the prompt's next token of every row
+    SampleJob smp;       // GUMBEL mode: the extras are keyed draws
     aasd_align_out out;
 };
 
@@ -508,10 +506,19 @@ __global__ void align_next_kernel(const AlignArgs a) {
     a.next_ids[t] = nxt;
 }
 
+// Does the row take keyed draws?  GUMBEL mode, a usable row, and a next token that is not the
+// greedy one (Sec. 2.3: only misaligned positions get extra tokens).
+__device__ inline bool align_wants_draws(const AlignArgs& a, const RowPartial& merged, int next) {
+    if (a.mode != AASD_ALIGN_GUMBEL || a.k_extra == 0 || partial_bad(merged)) return false;
+    return !(next != AASD_NONE && next == key_id(merged.key[0]));
+}
+
 // Row epilogue of alignment sampling (Sec. 2.3 alignment test, Fig. 2 extras), one thread.
-// next is the prompt's next token of the row (validated, or NONE), xn its raw logit.
+// next is the prompt's next token of the row (validated, or NONE), xn its raw logit.  In
+// GUMBEL mode draws[j] / draw_logits[j] are the row's keyed draws (NONE where not drawn).
 __device__ inline void align_row(const AlignArgs& a, const RowJob& job, int64_t row, const RowPartial& merged,
-                                 float neg_refc, bool centered, int next, float xn_in, Tally& tally) {
+                                 float neg_refc, bool centered, int next, float xn_in, const int* draws,
+                                 const float* draw_logits, Tally& tally) {
     const RowFinal f = finish_row(merged, job.c1, neg_refc, centered);
     const int KE = a.k_extra;
     int ids[kMaxK];
@@ -530,16 +537,30 @@ __device__ inline void align_row(const AlignArgs& a, const RowJob& job, int64_t 
             pn = f.prob(xn);
             aligned = (next == f.top1);
         }
-        // the listed tokens that rank above the next token (Fig. 2)
-        for (int j = 0; j < KE; ++j) {
-            const u64 k = merged.key[j];
-            if (k == 0) break;
-            const float xv = key_value(k);
-            const int id = key_id(k);
-            if (next == AASD_NONE || xv > xn || (xv == xn && id < next)) {
-                ids[n] = id;
-                ps[n] = (float)f.prob(xv);
+        if (a.mode == AASD_ALIGN_GUMBEL) {
+            // distinct draws other than the prompt's own token, in draw order
+            for (int j = 0; j < KE && !aligned; ++j) {
+                const int tok = draws[j];
+                if (tok == AASD_NONE || tok == next) continue;
+                bool dup = false;
+                for (int q = 0; q < n; ++q) dup |= (ids[q] == tok);
+                if (dup) continue;
+                ids[n] = tok;
+                ps[n] = (float)f.prob(draw_logits[j]);
                 ++n;
+            }
+        } else {
+            // the listed tokens that rank above the next token (Fig. 2)
+            for (int j = 0; j < KE; ++j) {
+                const u64 k = merged.key[j];
+                if (k == 0) break;
+                const float xv = key_value(k);
+                const int id = key_id(k);
+                if (next == AASD_NONE || xv > xn || (xv == xn && id < next)) {
+                    ids[n] = id;
+                    ps[n] = (float)f.prob(xv);
+                    ++n;
+                }
             }
         }
     }
@@ -560,15 +581,16 @@ __device__ inline void align_row(const AlignArgs& a, const RowJob& job, int64_t 
     }
 }
 
+// Entered by a whole warp with the draws already made (the same values in every lane).
 template <int DT>
-__device__ void align_finish(const AlignArgs& a, const RowJob& job, int64_t row, const char* rowp,
-                             const RowPartial& merged, float neg_refc, bool centered) {
-    const int next = __ldg(a.next_ids + row);
-    const float xn = next != AASD_NONE ? Elt<DT>::load(rowp, next) : 0.f;
-    Tally tally;
-    tally.clear();
-    align_row(a, job, row, merged, neg_refc, centered, next, xn, tally);
-    tally.flush(job.state);
+__device__ void align_finish_warp(const AlignArgs& a, const RowJob& job, int64_t row, const char* rowp,
+                                  const RowPartial& merged, float neg_refc, bool centered, int next, float xn,
+                                  const int (&draws)[kMaxK], Tally& tally) {
+    if ((threadIdx.x & 31) != 0) return;
+    float dx[kMaxK];
+    for (int j = 0; j < kMaxK; ++j)
+        dx[j] = (a.mode == AASD_ALIGN_GUMBEL && j < a.k_extra && draws[j] >= 0) ? Elt<DT>::load(rowp, draws[j]) : 0.f;
+    align_row(a, job, row, merged, neg_refc, centered, next, xn, draws, dx, tally);
 }
 
 template <int DT, int K>
@@ -582,8 +604,21 @@ __global__ void __launch_bounds__(kThreads) align_kernel(const AlignArgs a) {
     float neg_refc;
     bool centered;
     if (!row_reduce<DT, K>(job, row, chunk, next, rowp, neg_refc, centered, sc)) return;
-    if (threadIdx.x != 0) return;
-    align_finish<DT>(a, job, row, rowp, sc.merged, neg_refc, centered);
+    if (threadIdx.x >= 32) return;
+    const float xn = next != AASD_NONE ? Elt<DT>::load(rowp, next) : 0.f;
+    Tally tally;
+    tally.clear();
+    int draws[kMaxK];
+    for (int j = 0; j < kMaxK; ++j) draws[j] = AASD_NONE;
+    if (align_wants_draws(a, sc.merged, next)) {
+        // this layout takes the definition as it stands: every group scored in fp64
+        for (int j = 0; j < a.k_extra; ++j) {
+            draws[j] = warp_sample_exhaustive<DT>(rowp, job.vocab, (unsigned int)row, j, a.smp);
+            tally.exhaustive += 1;
+        }
+    }
+    align_finish_warp<DT>(a, job, row, rowp, sc.merged, neg_refc, centered, next, xn, draws, tally);
+    if (threadIdx.x == 0) tally.flush(job.state);
 }
 
 }  // namespace aasd

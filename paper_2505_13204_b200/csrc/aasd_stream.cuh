@@ -105,6 +105,7 @@ struct StreamShared {
     u64 freeb[kSlots];
     ItemInfo ring[kRing];
     WarpPartial wp[kSlots][kConsumerWarps];
+    RaceSummary race[kSlots][kConsumerWarps][kMaxK];   // sampling kernels only
     int abort_flag;
 };
 constexpr size_t kStreamSmemBytes = (size_t)kStages * kTileBytes + sizeof(StreamShared) + 128;
@@ -117,7 +118,12 @@ struct StreamJob {
     int whole_rows;           // rows [0, whole_rows) are one item each
     int tail_chunks;          // every later row is cut into this many pieces
     long long n_items;        // whole_rows + (n_rows - whole_rows) * tail_chunks
+    // sampling kernels only
+    SampleJob smp;
+    RaceSummary* race_partials;   // [slots x kMaxK] beside the partial records of cut rows
+    int full_groups;              // sampling groups that lie wholly inside the vector part of a row
 };
+constexpr int kRaceSlots = 1024;  // cut-row pieces a sampling launch may have
 
 // Work item -> (row, piece); pieces of a row are balanced ranges of its tiles.
 __device__ __forceinline__ void decode_item(const StreamJob& job, long long item, int& row, int& chunk) {
@@ -238,6 +244,40 @@ struct TileAccumulator {
     }
 };
 
+// The same for a sampling kernel: the sum of the vector's weights goes to `gs` (the caller
+// adds a whole group's sum to S at once, and needs it for the group's ratio).
+template <int DT, int K>
+__device__ __forceinline__ void add_to_group(TileAccumulator<DT, K>& acc, const uint4& raw, int vec_index, float c1,
+                                             float neg_refc, float2& gs) {
+    constexpr int kVec = Elt<DT>::kVec;
+    float x[kVec];
+    Elt<DT>::unpack(Clamp<DT>::apply(raw), x);
+    const float2 cc = make_float2(c1, c1);
+    const float2 rr = make_float2(neg_refc, neg_refc);
+#pragma unroll
+    for (int i = 0; i < kVec / 2; ++i) {
+        float2 t = __ffma2_rn(make_float2(x[2 * i], x[2 * i + 1]), cc, rr);
+        float2 e = make_float2(ex2_approx(t.x), ex2_approx(t.y));
+        gs = __fadd2_rn(gs, e);
+        acc.A2[i] = __ffma2_rn(e, t, acc.A2[i]);
+    }
+    float vmax = Clamp<DT>::vector_max(raw);
+    int vi = vec_index;
+#pragma unroll
+    for (int j = 0; j < K; ++j) {
+        // a thread does not meet its vectors in ascending order here: equal maxima go by index
+        const bool up = vmax > acc.best[j] || (vmax == acc.best[j] && vi < acc.best_vec[j]);
+        const float hi = fmaxf(acc.best[j], vmax);
+        const float lo = fminf(acc.best[j], vmax);
+        const int hi_i = up ? vi : acc.best_vec[j];
+        const int lo_i = up ? acc.best_vec[j] : vi;
+        acc.best[j] = hi;
+        acc.best_vec[j] = hi_i;
+        vmax = lo;
+        vi = lo_i;
+    }
+}
+
 // exponent and weight of one raw logit exactly as the consumers form them
 __device__ __forceinline__ void scalar_term(float x, float c1, float neg_refc, float& e, float& t) {
     float xc;
@@ -273,8 +313,10 @@ struct FinishedRow {
 };
 
 // Epilogue interface (static functions of a policy type E):
-//   E::finish(args, job, row, FinishedRow&, ItemInfo&, Tally&)  - entered by the whole finisher warp
-template <int DT, int K, class E>
+//   E::finish<ND>(args, job, row, rowp, FinishedRow&, ItemInfo&, races, tail_group, Tally&)
+//   - entered by the whole finisher warp
+//   ND: keyed draws per row the kernel prepares (0: no sampling)
+template <int DT, int K, int ND, class E>
 __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJob job, const typename E::Args args) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* tiles = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
@@ -307,6 +349,9 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
         for (;; ++seq) {
             TileAccumulator<DT, K> acc;
             acc.init();
+            GroupRace<(ND > 0 ? ND : 1)> race;
+            race.init();
+            unsigned int row_ctr = 0;
             float neg_refc = 0.f;
             bool alive = true, last = false;
             int tb = 0, te = 1;
@@ -326,12 +371,39 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
                         break;
                     }
                     neg_refc = info.neg_refc;
+                    row_ctr = (unsigned int)info.row;
                     tile_range(job, info.row, info.chunk, tb, te);
                 }
                 const unsigned char* base = tiles + (size_t)s * kTileBytes;
                 const int v0 = (tb + t) * kTileVecs;
                 const int nv = min(kTileVecs, rj.nvec - v0);
-                if (nv == kTileVecs) {
+                if (ND > 0) {
+                    // A thread takes four neighbouring vectors: one sampling group of bf16
+                    // ids, half a group of fp32 ids (lane pairs share a group).  The order
+                    // in which it reads them is rotated by the lane so that a quarter-warp
+                    // covers all shared-memory banks.
+                    constexpr int kPer = kTileVecs / kConsumers;
+                    static_assert(kPer == 4, "four vectors per thread and tile");
+                    const int rot = (lane >> 1) & 3;
+                    uint4 q[kPer];
+                    bool ok[kPer];
+#pragma unroll
+                    for (int k = 0; k < kPer; ++k) {
+                        const int v = kPer * tid + ((k + rot) & 3);
+                        ok[k] = v < nv;
+                        if (ok[k]) q[k] = lds16(base + (size_t)v * 16);
+                    }
+                    float2 gs = make_float2(0.f, 0.f);
+#pragma unroll
+                    for (int k = 0; k < kPer; ++k)
+                        if (ok[k]) add_to_group<DT, K>(acc, q[k], v0 + kPer * tid + ((k + rot) & 3), c1, neg_refc, gs);
+                    acc.S2[0] = __fadd2_rn(acc.S2[0], gs);
+                    float gsum = gs.x + gs.y;
+                    constexpr int kThreadsPerGroup = kGroup / (kPer * kVec);   // 1 (bf16) or 2 (fp32)
+                    if (kThreadsPerGroup == 2) gsum += __shfl_xor_sync(0xFFFFFFFFu, gsum, 1);
+                    const int g = (v0 + kPer * tid) * kVec / kGroup;
+                    if (g < job.full_groups && (tid % kThreadsPerGroup) == 0) race.offer(gsum, g, row_ctr, job.smp);
+                } else if (nv == kTileVecs) {
                     uint4 q[kTileVecs / kConsumers];
 #pragma unroll
                     for (int k = 0; k < kTileVecs / kConsumers; ++k) q[k] = lds16(base + (size_t)(k * kConsumers + tid) * 16);
@@ -375,6 +447,21 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
             if (last) {
                 if (lane == 0) mbar_arrive(&sh.done[p]);   // wakes the finisher, which sees the end too
                 break;
+            }
+            if (ND > 0) {
+#pragma unroll
+                for (int j = 0; j < ND; ++j) {
+                    u64 mine[kSampleKeep] = {race_key(race.best[j], race.best_g[j]), 0ull, 0ull};
+                    u64 top[kSampleKeep];
+                    warp_merge_keys<kSampleKeep>(mine, top);
+                    const float runner = warp_max_f32(race.runner[j]);
+                    if (lane == 0) {
+                        RaceSummary& r = sh.race[p][warp][j];
+#pragma unroll
+                        for (int q = 0; q < kSampleKeep; ++q) r.key[q] = top[q];
+                        r.runner = runner;
+                    }
+                }
             }
             if (lane == 0) {
                 WarpPartial& w = sh.wp[p][warp];
@@ -494,12 +581,28 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
         u64 vk[K];
 #pragma unroll
         for (int j = 0; j < K; ++j) vk[j] = 0;
+        RaceSummary races[ND > 0 ? ND : 1];   // per draw, the same in every lane once merged
         if (lane < kConsumerWarps) {
             const WarpPartial& w = sh.wp[p][lane];
             S = w.S;
             A = w.A;
 #pragma unroll
             for (int j = 0; j < K; ++j) vk[j] = w.key[j];
+        }
+        if (ND > 0) {
+#pragma unroll
+            for (int j = 0; j < ND; ++j) {
+                u64 mine[kSampleKeep] = {0ull, 0ull, 0ull};
+                float runner = -1.f;
+                if (lane < kConsumerWarps) {
+                    const RaceSummary& r = sh.race[p][lane][j];
+#pragma unroll
+                    for (int q = 0; q < kSampleKeep; ++q) mine[q] = r.key[q];
+                    runner = r.runner;
+                }
+                warp_merge_keys<kSampleKeep>(mine, races[j].key);
+                races[j].runner = warp_max_f32(runner);
+            }
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&sh.freeb[p]);
@@ -527,6 +630,11 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
 #pragma unroll
                 for (int j = 0; j < kMaxK; ++j) mine.key[j] = j < K ? mk[j] : 0ull;
                 slots[chunk] = mine;
+                if (ND > 0) {
+                    RaceSummary* rp = job.race_partials + ((row - job.whole_rows) * chunks + chunk) * kMaxK;
+#pragma unroll
+                    for (int j = 0; j < ND; ++j) rp[j] = races[j];
+                }
                 __threadfence();
                 const unsigned int t = atomicAdd(&rj.row_tickets[row], 1u);
                 last = (t == (unsigned int)chunks - 1);
@@ -556,6 +664,21 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
 #pragma unroll
                     for (int j = 0; j + 1 < K; ++j) vk[j] = vk[j + 1];
                     vk[K - 1] = 0;
+                }
+            }
+            if (ND > 0) {
+#pragma unroll
+                for (int j = 0; j < ND; ++j) {
+                    u64 mine[kSampleKeep] = {0ull, 0ull, 0ull};
+                    float runner = -1.f;
+                    for (int c = lane; c < chunks; c += 32) {
+                        const RaceSummary* rp = job.race_partials + ((row - job.whole_rows) * chunks + c) * kMaxK + j;
+#pragma unroll
+                        for (int q = 0; q < kSampleKeep; ++q) key_insert<kSampleKeep>(mine, __ldcg(&rp->key[q]));
+                        runner = fmaxf(runner, __ldcg(&rp->runner));
+                    }
+                    warp_merge_keys<kSampleKeep>(mine, races[j].key);
+                    races[j].runner = warp_max_f32(runner);
                 }
             }
         }
@@ -619,7 +742,9 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
         }
         fr.merged.S = S;
         fr.merged.A = A;
-        E::finish(args, rj, row, fr, info, tally);
+        // ids beyond the last complete group of the vector part were not raced
+        const int tail_group = (ND > 0 && job.full_groups * kGroup < rj.vocab) ? job.full_groups : -1;
+        E::template finish<ND>(args, rj, row, rowp, fr, info, races, tail_group, tally);
     }
     if (lane == 0) tally.flush(rj.state);
 }
@@ -628,19 +753,38 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
 template <int DT>
 struct VerifyEpilogue {
     using Args = VerifyArgs;
-    static __device__ void finish(const VerifyArgs& a, const RowJob& job, int64_t row, const FinishedRow& fr,
-                                  const ItemInfo& info, Tally& tally) {
-        verify_finish_warp<DT>(a, job, row, fr.merged, fr.neg_refc, fr.centered, info.hint, info.hint_logit, tally);
+    template <int ND>
+    static __device__ void finish(const VerifyArgs& a, const RowJob& job, int64_t row, const char* rowp,
+                                  const FinishedRow& fr, const ItemInfo& info, const RaceSummary* races, int tail_group,
+                                  Tally& tally) {
+        int sampled = AASD_NONE;
+        if (ND > 0 && !partial_bad(fr.merged))
+            sampled = warp_sample_decide<DT>(rowp, job.vocab, (unsigned int)row, 0, a.smp, races[0], tail_group,
+                                             fr.centered, tally.recheck, tally.exhaustive);
+        verify_finish_warp<DT>(a, job, row, fr.merged, fr.neg_refc, fr.centered, info.hint, info.hint_logit, sampled,
+                               tally);
     }
 };
 template <int DT>
 struct AlignEpilogue {
     using Args = AlignArgs;
-    static __device__ void finish(const AlignArgs& a, const RowJob& job, int64_t row, const FinishedRow& fr,
-                                  const ItemInfo& info, Tally& tally) {
-        // next_ids holds validated tokens only
-        if ((threadIdx.x & 31) == 0)
-            align_row(a, job, row, fr.merged, fr.neg_refc, fr.centered, info.hint, info.hint_logit, tally);
+    template <int ND>
+    static __device__ void finish(const AlignArgs& a, const RowJob& job, int64_t row, const char* rowp,
+                                  const FinishedRow& fr, const ItemInfo& info, const RaceSummary* races, int tail_group,
+                                  Tally& tally) {
+        // next_ids holds validated tokens only, so the hint is the row's next token
+        int draws[kMaxK];
+#pragma unroll
+        for (int j = 0; j < kMaxK; ++j) draws[j] = AASD_NONE;
+        if (ND > 0 && align_wants_draws(a, fr.merged, info.hint)) {
+#pragma unroll
+            for (int j = 0; j < ND; ++j)
+                if (j < a.k_extra)
+                    draws[j] = warp_sample_decide<DT>(rowp, job.vocab, (unsigned int)row, j, a.smp, races[j], tail_group,
+                                                      fr.centered, tally.recheck, tally.exhaustive);
+        }
+        align_finish_warp<DT>(a, job, row, rowp, fr.merged, fr.neg_refc, fr.centered, info.hint, info.hint_logit, draws,
+                              tally);
     }
 };
 

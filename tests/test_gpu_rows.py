@@ -81,7 +81,6 @@ def test_verify_parity(ctx, V, dtype, stride, rows, mode):
     xd = _to_dev(x)
     got = ctx.verify(xd, torch.as_tensor(d).cuda(), torch.as_tensor(offs).cuda(),
                      draft_flags=torch.as_tensor(flags).cuda(), alpha=alpha, beta=beta, mode=mode)
-    got["sampled"] = None
     check_verify(got, ref, offs, dtype)
     st = ctx.poll_status()
     assert bool(st & binding.STATUS_ID_RANGE) == (rows > 10)
@@ -115,6 +114,90 @@ def test_align_parity(ctx, V, dtype, stride, rows, K):
     assert ctx.poll_status() == 0
 
 
+SAMPLED_CASES = CASES + [
+    (152064, torch.bfloat16, None, 300),   # more rows than CTA slots: whole-row items
+    (32000, torch.float32, None, 310),
+    (4096, torch.bfloat16, None, 700),
+    (33, torch.float32, 36, 20),           # one complete group and a one-token tail group
+    (31, torch.bfloat16, 32, 20),          # a single, incomplete group
+    (2000, torch.bfloat16, 2008, 50),      # 62 complete groups + a 16-token tail group
+]
+
+
+@pytest.mark.parametrize("V,dtype,stride,rows", SAMPLED_CASES)
+def test_verify_strict_sampled_parity(ctx, V, dtype, stride, rows):
+    """The row's own token is a keyed draw (Eq. 1); the GPU must draw the very same token."""
+    rng = np.random.default_rng(3 * V + rows)
+    d = rng.integers(0, V, rows).astype(np.int32)
+    x = _make_logits(rows, V, dtype, 300 + V, torch.as_tensor(d, dtype=torch.int64), stride=stride)
+    offs = _random_csr(rng, rows)
+    seed, step, invT = 0x1234567890ABCDEF + V, 7 + rows, F32(0.9)
+    ref = oracle.verify(to_oracle(x), d, offs, mode=oracle.VERIFY_STRICT_SAMPLED, seed=seed, step=step,
+                        inv_temperature=invT)
+    # half of the drafts are what the target itself draws, so that acceptance happens
+    d = np.where(rng.random(rows) < 0.5, ref["sampled"], d).astype(np.int32)
+    ref = oracle.verify(to_oracle(x), d, offs, mode=oracle.VERIFY_STRICT_SAMPLED, seed=seed, step=step,
+                        inv_temperature=invT)
+    ctx.reset_counters()
+    got = ctx.verify(_to_dev(x), torch.as_tensor(d).cuda(), torch.as_tensor(offs).cuda(),
+                     mode=binding.VERIFY_STRICT_SAMPLED, seed=seed, step=step, inv_temperature=invT)
+    assert np.array_equal(cpu(got["sampled"]), ref["sampled"])
+    check_verify(got, ref, offs, dtype)
+    assert ref["accept"].sum() > 0 and (ref["sampled"] != ref["argmax"]).any()
+    assert ctx.poll_status() == 0
+    c = ctx.counters()
+    # re-scoring in fp64 is the exception, the exhaustive routine rarer still (aligned layouts)
+    if V >= 1000 and V % 32 == 0 and stride is None:
+        assert c["sampler_recheck"] + c["sampler_exact"] <= max(2, rows // 20), c
+
+
+@pytest.mark.parametrize("V,dtype,stride,rows", SAMPLED_CASES)
+@pytest.mark.parametrize("K", [1, 2, 3, 4])
+def test_align_gumbel_parity(ctx, V, dtype, stride, rows, K):
+    if V > 40000 and K in (1, 3):
+        pytest.skip("large vocabularies run K = 2, 4")
+    rng = np.random.default_rng(11 * V + rows + K)
+    prompt = rng.integers(0, V, rows).astype(np.int32)
+    cut = sorted(set([0, rows] + [int(c) for c in rng.integers(1, rows, 2)]))
+    hints = synth.next_token_hints(torch.as_tensor(prompt))
+    x = _make_logits(rows, V, dtype, 400 + V, hints, stride=stride)
+    seed, tag = 99 + K, 5
+    ref = oracle.align_sample(to_oracle(x), prompt, cut, k_extra=K, mode=oracle.ALIGN_GUMBEL, seed=seed,
+                              stream_tag=tag)
+    got = ctx.align_sample(_to_dev(x), torch.as_tensor(prompt).cuda(), cut, k_extra=K,
+                           mode=binding.ALIGN_GUMBEL, seed=seed, stream_tag=tag)
+    check_align(got, ref, dtype)
+    assert (ref["n_extra"] > 0).any()
+    if rows >= 40 and V <= 4096:
+        assert (ref["aligned"] == 1).any()    # aligned rows take no draws
+    assert ctx.poll_status() == 0
+
+
+def test_sampler_on_flat_and_masked_rows(ctx):
+    """Rows where many groups are equally likely, rows with masked ids, one live token."""
+    V, rows = 8192, 16
+    for dtype in (torch.float32, torch.bfloat16):
+        x = torch.zeros((rows, V), dtype=torch.float32)
+        x[1] = 3.25
+        x[2, 100:8000] = -float("inf")
+        x[3, :] = -float("inf"); x[3, 4097] = 0.5
+        x[4, ::2] = -float("inf")
+        x[5] = torch.linspace(-20, 20, V)
+        x[6, :] = -80.0; x[6, 77] = 70.0          # the reference sits 150 orders below the maximum
+        x[7, 9] = float("nan")
+        x = x.to(dtype)
+        d = np.zeros(rows, np.int32)
+        offs = np.arange(rows + 1, dtype=np.int32)
+        for step in range(3):
+            ref = oracle.verify(to_oracle(x), d, offs, mode=oracle.VERIFY_STRICT_SAMPLED, seed=5, step=step)
+            got = ctx.verify(x.cuda(), torch.as_tensor(d).cuda(), torch.as_tensor(offs).cuda(),
+                             mode=binding.VERIFY_STRICT_SAMPLED, seed=5, step=step)
+            assert np.array_equal(cpu(got["sampled"]), ref["sampled"])
+            check_verify(got, ref, offs, dtype)
+        assert ref["sampled"][3] == 4097 and ref["sampled"][7] == -1
+        assert ctx.poll_status() & binding.STATUS_BAD_ROW
+
+
 def test_rows_with_masked_entries_far_maxima_and_bad_rows(ctx):
     V, rows = 4096, 12
     rng = np.random.default_rng(3)
@@ -135,7 +218,6 @@ def test_rows_with_masked_entries_far_maxima_and_bad_rows(ctx):
         ref = oracle.verify(to_oracle(x), d, offs, alpha=F32(0.1), beta=F32(0.1))
         got = ctx.verify(x.cuda(), torch.as_tensor(d).cuda(), torch.as_tensor(offs).cuda(),
                          alpha=F32(0.1), beta=F32(0.1))
-        got["sampled"] = None
         check_verify(got, ref, offs, dtype)
         assert list(ref["bad"][:9]) == [0, 0, 0, 0, 1, 1, 1, 0, 0]
         assert ctx.poll_status() & binding.STATUS_BAD_ROW
@@ -160,7 +242,6 @@ def test_temperature_and_thresholds(ctx):
         ref = oracle.verify(to_oracle(x), d, offs, alpha=alpha, beta=beta, inv_temperature=invT)
         got = ctx.verify(x.cuda(), torch.as_tensor(d).cuda(), torch.as_tensor(offs).cuda(),
                          alpha=alpha, beta=beta, inv_temperature=invT)
-        got["sampled"] = None
         check_verify(got, ref, offs, torch.bfloat16)
         gr = ctx.verify(x.cuda(), torch.as_tensor(d).cuda(), None, alpha=alpha, beta=beta,
                         inv_temperature=invT, rows_per_cand=8)
