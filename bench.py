@@ -42,6 +42,16 @@ ALPHA = float(np.float32(0.1))
 BETA = float(np.float32(0.1))
 K_EXTRA = 2
 N_BUF = 8
+# DRAM bytes (read + write) per captured launch of the streaming kernels, from the ncu
+# captures summarised under profiles/: (workload, kernel) -> (rows captured, bytes).  Traffic
+# is proportional to rows (each row is read once), so it is scaled to the launch's rows.
+# An entry is set to None whenever the kernel has changed since its capture.
+NCU_TRAFFIC = {("cfg5-serving-256", "verify"): None, ("cfg5-serving-256", "align"): None}
+
+
+def ncu_traffic(workload: str, kernel: str, rows: int):
+    cap = NCU_TRAFFIC.get((workload, kernel))
+    return None if cap is None else cap[1] * rows / cap[0]
 
 
 def measured_peaks():
@@ -193,9 +203,12 @@ class Bench:
                               outputs=self.pre_out[j])
         if events is not None:
             events[1].record()
-        self.state.step(self.ver_bufs[j], j)
+        self.state.run_draft()
         if events is not None:
             events[2].record()
+        self.state.step(self.ver_bufs[j], j, reuse_draft=True)
+        if events is not None:
+            events[3].record()
 
 
 def run_ours(args, rank, world, local_rank):
@@ -218,7 +231,7 @@ def run_ours(args, rank, world, local_rank):
         torch.cuda.synchronize()
 
     launches0 = bench.ctx.launch_count()
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K)]
     t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     clocks = ClockSampler(local_rank)
@@ -232,7 +245,8 @@ def run_ours(args, rank, world, local_rank):
     ms = t_begin.elapsed_time(t_end)
     launches = bench.ctx.launch_count() - launches0
     align_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in evs]))
-    decode_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in evs]))
+    draft_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in evs]))
+    verify_ms = float(np.mean([e[2].elapsed_time(e[3]) for e in evs]))
     if world > 1:
         t = torch.tensor([ms], device=dev)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -252,8 +266,9 @@ def run_ours(args, rank, world, local_rank):
     esize = 2 if w.dtype == "bf16" else 4
     peak, peak_src = measured_peaks()
     row_bytes = w.vocab * esize
-    # the decode part is draft + verify + select + append; verification is all but a few us
-    ver_gbs = bench.R * row_bytes / (decode_ms * 1e-3) / 1e9
+    # events bracket the verification launch alone (selection and append ride on it) and the
+    # two launches of aasd_align_sample (next-token gather, ~3 us, + streaming kernel)
+    ver_gbs = bench.R * row_bytes / (verify_ms * 1e-3) / 1e9
     ali_gbs = bench.pre_rows * row_bytes / (align_ms * 1e-3) / 1e9
     value = world * bench.R * K / (ms * 1e-3)
     line = {
@@ -273,13 +288,18 @@ def run_ours(args, rank, world, local_rank):
                 "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
                 "ms_per_step": e2e["ms_per_step"]},
         "gpu_launches": int(launches),
-        "roofline": {"bound": "hbm", "kernel": "verify_kernel<bf16> (timed with draft/select/append, <1% of it)",
+        "roofline": {"bound": "hbm",
+                     "kernel": "stream_kernel<%s, K=1, ND=0, VerifyEpilogue> (verification with the accept scan, "
+                               "selection and append fused)" % w.dtype,
                      "achieved": ver_gbs, "peak": peak, "unit": "GB/s", "frac": ver_gbs / peak,
-                     "peak_source": peak_src + ", sustained copy figure", "traffic": None,
-                     "ms_per_launch": decode_ms, "bytes_per_launch": bench.R * row_bytes},
-        "roofline_align": {"bound": "hbm", "kernel": "align_kernel<bf16,2>", "achieved": ali_gbs, "peak": peak,
-                           "unit": "GB/s", "frac": ali_gbs / peak, "ms_per_launch": align_ms,
-                           "bytes_per_launch": bench.pre_rows * row_bytes},
+                     "peak_source": peak_src, "traffic": ncu_traffic(w.name, "verify", bench.R),
+                     "ms_per_launch": verify_ms, "bytes_per_launch": bench.R * row_bytes},
+        "roofline_align": {"bound": "hbm",
+                           "kernel": "align_next_kernel + stream_kernel<%s, K=%d, ND=0, AlignEpilogue>" % (w.dtype, K_EXTRA),
+                           "achieved": ali_gbs, "peak": peak, "unit": "GB/s", "frac": ali_gbs / peak,
+                           "peak_source": peak_src, "traffic": ncu_traffic(w.name, "align", bench.pre_rows),
+                           "ms_per_launch": align_ms, "bytes_per_launch": bench.pre_rows * row_bytes},
+        "draft_us_per_launch": draft_ms * 1e3,
         "logits_gbs": (bench.R + bench.pre_rows) * row_bytes * K / (ms * 1e-3) / 1e9,
         "accepted_tokens_per_s": world * bench.accepted_per_cycle / N_BUF * K / (ms * 1e-3),
         "mean_tokens_per_seq_step": bench.accepted_per_cycle / N_BUF / w.batch,
@@ -440,6 +460,12 @@ def run_micro(args):
         nonlocal outs
         if args.micro == "verify":
             outs = ctx.verify(bufs[j], ids[j], None, alpha=ALPHA, beta=BETA, rows_per_cand=rpc, outputs=outs)
+        elif args.micro == "verify-sampled":
+            outs = ctx.verify(bufs[j], ids[j], None, rows_per_cand=rpc, outputs=outs, seed=17, step=j,
+                              mode=binding.VERIFY_STRICT_SAMPLED)
+        elif args.micro == "align-gumbel":
+            outs = ctx.align_sample(bufs[j], ids[j], offs, k_extra=K_EXTRA, outputs=outs, seed=17,
+                                    mode=binding.ALIGN_GUMBEL)
         else:
             outs = ctx.align_sample(bufs[j], ids[j], offs, k_extra=K_EXTRA, outputs=outs)
 
@@ -485,7 +511,7 @@ def run_micro(args):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--micro", default=None, choices=["verify", "align"],
+    ap.add_argument("--micro", default=None, choices=["verify", "align", "verify-sampled", "align-gumbel"],
                     help="time one kernel alone on --rows rows of the workload")
     ap.add_argument("--rows", type=int, default=1024)
     ap.add_argument("--graph", action="store_true", help="--micro: replay the launches from a CUDA graph")

@@ -266,6 +266,10 @@ int aasd_append(aasd_ctx* ctx, int32_t* hist_ids, const int32_t* hist_offsets,
 
 /* ---- one decoding step of the batched driver (Algorithm 1, loop body) ------------- */
 
+/* aasd_step_args.flags */
+#define AASD_STEP_REUSE_DRAFT 1u /* draft_out already holds this state's candidates (the caller
+                                    ran aasd_draft, e.g. to feed the model): do not draft again */
+
 typedef struct aasd_step_args {
     aasd_draft_in draft_in;        /* recent_ids == NULL: the key is the history's own tail */
     aasd_draft_params draft;
@@ -278,12 +282,15 @@ typedef struct aasd_step_args {
     int32_t* best_cand;            /* [n_seqs] */
     int32_t* n_emit;               /* [n_seqs] */
     int32_t* emit_ids;             /* [n_seqs x (draft_len+1)] */
+    uint32_t flags;                /* AASD_STEP_* */
 } aasd_step_args;
 
-/* draft -> verify -> select -> append on the context's stream.  The target logits of the
- * step must already be resident: row (b, c, i) judges token i of candidate c of sequence
- * b, so the caller's model runs on the candidates of the previous aasd_draft of the same
- * state (the benchmark replays logits drawn for exactly those candidates). */
+/* draft -> verify -> select -> append on the context's stream (Algorithm 1, loop body), in
+ * two launches: the drafting kernel, and the verification kernel, in which the warp that
+ * completes a sequence's last candidate also selects and appends.  Row (b, c, i) of the
+ * target logits judges token i of candidate c of sequence b, so the logits come from a
+ * model run on the candidates aasd_draft emits for the same state; a caller that has just
+ * made that call passes AASD_STEP_REUSE_DRAFT and the step is the second launch alone. */
 int aasd_step(aasd_ctx* ctx, const aasd_step_args* args, void* workspace,
               size_t workspace_bytes);
 

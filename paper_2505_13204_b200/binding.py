@@ -20,6 +20,7 @@ VERIFY_CONDITIONAL, VERIFY_STRICT_GREEDY, VERIFY_STRICT_SAMPLED = 0, 1, 2
 STATUS_BAD_ROW, STATUS_ID_RANGE, STATUS_HIST_OVERFLOW, STATUS_BAD_OFFSETS = 1, 2, 4, 8
 FLAG_CONDITIONAL, FLAG_EXTRA = 1, 2
 DRAFT_MATCH_ALIGN = 1
+STEP_REUSE_DRAFT = 1
 
 EXPORTS = [
     "aasd_create", "aasd_destroy", "aasd_set_stream", "aasd_status_str", "aasd_poll_status",
@@ -75,7 +76,7 @@ class StepArgs(C.Structure):
     _fields_ = [("draft_in", DraftIn), ("draft", DraftParams), ("draft_out", DraftOut),
                 ("target_logits", _vp), ("verify", VerifyParams), ("verify_out", VerifyOut),
                 ("hist_ids", _vp), ("hist_len", _vp), ("best_cand", _vp), ("n_emit", _vp),
-                ("emit_ids", _vp)]
+                ("emit_ids", _vp), ("flags", C.c_uint32)]
 
 
 class Counters(C.Structure):
@@ -455,12 +456,14 @@ class DecodeState:
                                        C.byref(a.draft_out)), "aasd_draft")
         return self.draft_out
 
-    def step(self, target_logits: torch.Tensor, step_index: int = 0):
-        """aasd_step: draft -> verify -> select -> append with resident logits."""
+    def step(self, target_logits: torch.Tensor, step_index: int = 0, reuse_draft: bool = False):
+        """aasd_step: draft -> verify -> select -> append with resident logits.
+        ``reuse_draft``: ``run_draft`` was just called on this state, do not draft again."""
         assert target_logits.shape[0] == self.rows and target_logits.stride(1) == 1
         a = self.args
         a.target_logits = _p(target_logits)
         a.verify.row_stride = target_logits.stride(0)
+        a.flags = STEP_REUSE_DRAFT if reuse_draft else 0
         a.verify.step = int(step_index)
         _check(self.ctx.lib.aasd_step(self.ctx._h, C.byref(a), _p(self.ws), self.ws.numel()),
                "aasd_step")

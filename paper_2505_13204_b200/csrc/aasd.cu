@@ -22,7 +22,7 @@ namespace {
 struct WorkspaceLayout {
     size_t bytes;
     int64_t max_rows, max_cands;
-    size_t off_partials, off_row_tickets, off_cand_tickets, off_sched, off_row_accept, off_row_own, off_next, off_race;
+    size_t off_partials, off_row_tickets, off_cand_tickets, off_seq_tickets, off_sched, off_row_accept, off_row_own, off_next, off_race;
 };
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -37,6 +37,8 @@ WorkspaceLayout make_layout(int64_t max_rows, int64_t max_cands) {
     L.off_row_tickets = o;
     o = align_up(o + 4 * (size_t)max_rows, 256);
     L.off_cand_tickets = o;
+    o = align_up(o + 4 * (size_t)max_cands, 256);
+    L.off_seq_tickets = o;
     o = align_up(o + 4 * (size_t)max_cands, 256);
     L.off_sched = o;
     o = align_up(o + 2 * sizeof(unsigned int), 256);
@@ -70,6 +72,25 @@ namespace {
         cudaError_t e__ = (call);                         \
         if (e__ != cudaSuccess) return AASD_ERR_CUDA;     \
     } while (0)
+
+// Every kernel of the library is launched with programmatic stream serialization: it may be
+// scheduled while its predecessor in the stream drains, and waits (griddepcontrol.wait,
+// first thing in each kernel) for that predecessor to complete before it touches memory.
+template <class... Params, class... Args>
+void launch(void (*kernel)(Params...), unsigned int grid, unsigned int block, size_t smem, cudaStream_t stream,
+            Args&&... args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(grid, 1, 1);
+    cfg.blockDim = dim3(block, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, kernel, Params(args)...);   // errors surface in cudaGetLastError
+}
 
 int after_launch(aasd_ctx* ctx, int n) {
     ctx->launches += (uint64_t)n;
@@ -190,7 +211,7 @@ template <int DT, int K, int ND>
 int launch_align_stream(aasd_ctx* ctx, const StreamJob& sj, const AlignArgs& a, unsigned int grid) {
     auto kernel = stream_kernel<DT, K, ND, AlignEpilogue<DT>>;
     if (enable_stream_smem(kernel) != AASD_OK) return AASD_ERR_CUDA;
-    kernel<<<grid, kStreamThreads, kStreamSmemBytes, ctx->stream>>>(sj, a);
+    launch(kernel, grid, kStreamThreads, kStreamSmemBytes, ctx->stream, sj, a);
     return AASD_OK;
 }
 
@@ -213,7 +234,7 @@ template <int DT, int ND>
 int launch_verify_stream(aasd_ctx* ctx, const StreamJob& sj, const VerifyArgs& a, unsigned int grid) {
     auto kernel = stream_kernel<DT, 1, ND, VerifyEpilogue<DT>>;
     if (enable_stream_smem(kernel) != AASD_OK) return AASD_ERR_CUDA;
-    kernel<<<grid, kStreamThreads, kStreamSmemBytes, ctx->stream>>>(sj, a);
+    launch(kernel, grid, kStreamThreads, kStreamSmemBytes, ctx->stream, sj, a);
     return AASD_OK;
 }
 
@@ -369,7 +390,7 @@ int aasd_align_sample(aasd_ctx* ctx, const void* prefill_logits, const int32_t* 
     a.smp = make_sample_job(p->seed, p->stream_tag, true, p->inv_temperature);
     a.out = *out;
     AASD_CUDA(cudaSetDevice(ctx->device));
-    align_next_kernel<<<(unsigned int)((n_rows + 255) / 256), 256, 0, ctx->stream>>>(a);
+    launch(align_next_kernel, (unsigned int)((n_rows + 255) / 256), 256, 0, ctx->stream, a);
     // plain kernels: the K best tokens in TOPK mode, the best token alone in GUMBEL mode
     const int K = (p->k_extra <= 1 || p->mode == AASD_ALIGN_GUMBEL) ? 1 : (p->k_extra == 2 ? 2 : 4);
     if (a.job.vector_ok && a.job.nvec > 0) {
@@ -385,13 +406,13 @@ int aasd_align_sample(aasd_ctx* ctx, const void* prefill_logits, const int32_t* 
     }
     const unsigned int grid = (unsigned int)(n_rows * a.job.chunks);
     if (p->dtype == AASD_F32) {
-        if (K == 1) align_kernel<AASD_F32, 1><<<grid, kThreads, 0, ctx->stream>>>(a);
-        else if (K == 2) align_kernel<AASD_F32, 2><<<grid, kThreads, 0, ctx->stream>>>(a);
-        else align_kernel<AASD_F32, 4><<<grid, kThreads, 0, ctx->stream>>>(a);
+        if (K == 1) launch(align_kernel<AASD_F32, 1>, grid, kThreads, 0, ctx->stream, a);
+        else if (K == 2) launch(align_kernel<AASD_F32, 2>, grid, kThreads, 0, ctx->stream, a);
+        else launch(align_kernel<AASD_F32, 4>, grid, kThreads, 0, ctx->stream, a);
     } else {
-        if (K == 1) align_kernel<AASD_BF16, 1><<<grid, kThreads, 0, ctx->stream>>>(a);
-        else if (K == 2) align_kernel<AASD_BF16, 2><<<grid, kThreads, 0, ctx->stream>>>(a);
-        else align_kernel<AASD_BF16, 4><<<grid, kThreads, 0, ctx->stream>>>(a);
+        if (K == 1) launch(align_kernel<AASD_BF16, 1>, grid, kThreads, 0, ctx->stream, a);
+        else if (K == 2) launch(align_kernel<AASD_BF16, 2>, grid, kThreads, 0, ctx->stream, a);
+        else launch(align_kernel<AASD_BF16, 4>, grid, kThreads, 0, ctx->stream, a);
     }
     return after_launch(ctx, 2);
 }
@@ -410,14 +431,19 @@ int aasd_draft(aasd_ctx* ctx, const aasd_draft_in* in, const aasd_draft_params* 
         return AASD_ERR_INVALID_ARG;
     DraftArgs a{*in, *p, *out, ctx->state};
     AASD_CUDA(cudaSetDevice(ctx->device));
-    draft_kernel<<<(unsigned int)p->n_seqs, kThreads, 0, ctx->stream>>>(a);
+    launch(draft_kernel, (unsigned int)p->n_seqs, kThreads, 0, ctx->stream, a);
     return after_launch(ctx, 1);
 }
 
-int aasd_verify(aasd_ctx* ctx, const void* target_logits, const int32_t* draft_ids,
-                const uint8_t* draft_flags, const int32_t* cand_offsets, int32_t n_cands,
-                int64_t n_rows, const aasd_verify_params* p, void* workspace, size_t workspace_bytes,
-                const aasd_verify_out* out) {
+}  // extern "C"
+
+namespace {
+
+// aasd_verify, optionally followed inside the same launch by selection and append
+// (`seq`, regular candidate layout only).
+int verify_impl(aasd_ctx* ctx, const void* target_logits, const int32_t* draft_ids, const uint8_t* draft_flags,
+                const int32_t* cand_offsets, int32_t n_cands, int64_t n_rows, const aasd_verify_params* p,
+                void* workspace, size_t workspace_bytes, const aasd_verify_out* out, const SeqTail* seq) {
     if (ctx == nullptr || p == nullptr || out == nullptr) return AASD_ERR_INVALID_ARG;
     if (n_cands < 0 || n_rows < 0) return AASD_ERR_BAD_SHAPE;
     if (p->mode < AASD_VERIFY_CONDITIONAL || p->mode > AASD_VERIFY_STRICT_SAMPLED) return AASD_ERR_INVALID_ARG;
@@ -447,10 +473,15 @@ int aasd_verify(aasd_ctx* ctx, const void* target_logits, const int32_t* draft_i
     a.row_own = reinterpret_cast<int32_t*>(ws + L->off_row_own);
     a.smp = make_sample_job(p->seed, p->step, false, p->inv_temperature);
     a.out = *out;
+    if (seq) {
+        a.seq = *seq;
+        a.seq.enabled = 1;
+        a.seq.seq_tickets = reinterpret_cast<unsigned int*>(ws + L->off_seq_tickets);
+    }
     AASD_CUDA(cudaSetDevice(ctx->device));
     if (n_rows == 0) {
         if (n_cands == 0) return AASD_OK;
-        verify_empty_kernel<<<(unsigned int)((n_cands + 255) / 256), 256, 0, ctx->stream>>>(a);
+        launch(verify_empty_kernel, (unsigned int)((n_cands + 255) / 256), 256, 0, ctx->stream, a);
         return after_launch(ctx, 1);
     }
     if (a.job.vector_ok && a.job.nvec > 0) {
@@ -463,9 +494,21 @@ int aasd_verify(aasd_ctx* ctx, const void* target_logits, const int32_t* draft_i
         return after_launch(ctx, 1);
     }
     const unsigned int grid = (unsigned int)(n_rows * a.job.chunks);
-    if (p->dtype == AASD_F32) verify_kernel<AASD_F32><<<grid, kThreads, 0, ctx->stream>>>(a);
-    else verify_kernel<AASD_BF16><<<grid, kThreads, 0, ctx->stream>>>(a);
+    if (p->dtype == AASD_F32) launch(verify_kernel<AASD_F32>, grid, kThreads, 0, ctx->stream, a);
+    else launch(verify_kernel<AASD_BF16>, grid, kThreads, 0, ctx->stream, a);
     return after_launch(ctx, 1);
+}
+
+}  // namespace
+
+extern "C" {
+
+int aasd_verify(aasd_ctx* ctx, const void* target_logits, const int32_t* draft_ids,
+                const uint8_t* draft_flags, const int32_t* cand_offsets, int32_t n_cands,
+                int64_t n_rows, const aasd_verify_params* p, void* workspace, size_t workspace_bytes,
+                const aasd_verify_out* out) {
+    return verify_impl(ctx, target_logits, draft_ids, draft_flags, cand_offsets, n_cands, n_rows, p, workspace,
+                       workspace_bytes, out, nullptr);
 }
 
 int aasd_select(aasd_ctx* ctx, const int32_t* accept_len, const int32_t* next_token,
@@ -481,7 +524,7 @@ int aasd_select(aasd_ctx* ctx, const int32_t* accept_len, const int32_t* next_to
     SelectArgs a{accept_len, next_token, draft_ids, cand_offsets, rows_per_cand, seq_cand_offsets,
                  cands_per_seq, n_seqs, emit_stride, best_cand, n_emit, emit_ids};
     AASD_CUDA(cudaSetDevice(ctx->device));
-    select_kernel<<<(unsigned int)((n_seqs + 127) / 128), 128, 0, ctx->stream>>>(a);
+    launch(select_kernel, (unsigned int)((n_seqs + 127) / 128), 128, 0, ctx->stream, a);
     return after_launch(ctx, 1);
 }
 
@@ -493,7 +536,7 @@ int aasd_append(aasd_ctx* ctx, int32_t* hist_ids, const int32_t* hist_offsets, i
     if (!hist_ids || !hist_offsets || !hist_len || !emit_ids || !n_emit) return AASD_ERR_INVALID_ARG;
     AppendArgs a{hist_ids, hist_offsets, hist_len, emit_ids, n_emit, n_seqs, emit_stride, ctx->state};
     AASD_CUDA(cudaSetDevice(ctx->device));
-    append_kernel<<<(unsigned int)((n_seqs + 127) / 128), 128, 0, ctx->stream>>>(a);
+    launch(append_kernel, (unsigned int)((n_seqs + 127) / 128), 128, 0, ctx->stream, a);
     return after_launch(ctx, 1);
 }
 
@@ -502,21 +545,31 @@ int aasd_step(aasd_ctx* ctx, const aasd_step_args* s, void* workspace, size_t wo
     const aasd_draft_params& dp = s->draft;
     if (!s->hist_ids || !s->hist_len || !s->best_cand || !s->n_emit || !s->emit_ids) return AASD_ERR_INVALID_ARG;
     if (!s->verify_out.accept_len || !s->verify_out.next_token) return AASD_ERR_INVALID_ARG;
-    int err = aasd_draft(ctx, &s->draft_in, &dp, &s->draft_out);
-    if (err != AASD_OK) return err;
+    int err = AASD_OK;
+    if (!(s->flags & AASD_STEP_REUSE_DRAFT)) {
+        err = aasd_draft(ctx, &s->draft_in, &dp, &s->draft_out);
+        if (err != AASD_OK) return err;
+    } else if (dp.n_seqs < 0 || dp.draft_len < 1 || dp.max_cands < 1 || !s->draft_out.draft_ids) {
+        return AASD_ERR_INVALID_ARG;
+    }
     aasd_verify_params vp = s->verify;
     vp.rows_per_cand = dp.draft_len;
     const int32_t n_cands = dp.n_seqs * dp.max_cands;
     const int64_t n_rows = (int64_t)n_cands * dp.draft_len;
-    err = aasd_verify(ctx, s->target_logits, s->draft_out.draft_ids, s->draft_out.draft_flags, nullptr, n_cands,
-                      n_rows, &vp, workspace, workspace_bytes, &s->verify_out);
-    if (err != AASD_OK) return err;
-    err = aasd_select(ctx, s->verify_out.accept_len, s->verify_out.next_token, s->draft_out.draft_ids, nullptr,
-                      dp.draft_len, nullptr, dp.max_cands, dp.n_seqs, dp.draft_len + 1, s->best_cand, s->n_emit,
-                      s->emit_ids);
-    if (err != AASD_OK) return err;
-    return aasd_append(ctx, s->hist_ids, s->draft_in.hist_offsets, s->hist_len, s->emit_ids, s->n_emit, dp.n_seqs,
-                       dp.draft_len + 1);
+    if (n_rows == 0) return AASD_OK;
+    // selection and append ride on the verification launch: the warp that completes a
+    // sequence's last candidate does both
+    SeqTail tail{};
+    tail.cands_per_seq = dp.max_cands;
+    tail.emit_stride = dp.draft_len + 1;
+    tail.best_cand = s->best_cand;
+    tail.n_emit = s->n_emit;
+    tail.emit_ids = s->emit_ids;
+    tail.hist_ids = s->hist_ids;
+    tail.hist_offsets = s->draft_in.hist_offsets;
+    tail.hist_len = s->hist_len;
+    return verify_impl(ctx, s->target_logits, s->draft_out.draft_ids, s->draft_out.draft_flags, nullptr, n_cands,
+                       n_rows, &vp, workspace, workspace_bytes, &s->verify_out, &tail);
 }
 
 }  // extern "C"
@@ -533,7 +586,7 @@ constexpr int64_t kStaticMaxCands = AASD_STATIC_MAX_CANDS;
 constexpr size_t kStaticWorkspaceBytes =
     ((sizeof(RowPartial) * (size_t)kPartialSlots + 255) / 256 * 256) +   // pieces of split rows
     ((4 * (size_t)kStaticMaxRows + 255) / 256 * 256) +                   // row tickets
-    ((4 * (size_t)kStaticMaxCands + 255) / 256 * 256) +                  // candidate tickets
+    2 * ((4 * (size_t)kStaticMaxCands + 255) / 256 * 256) +              // candidate and sequence tickets
     256 +                                                                // work-item counters
     (((size_t)kStaticMaxRows + 255) / 256 * 256) +                       // accept bits
     2 * ((4 * (size_t)kStaticMaxRows + 255) / 256 * 256) +               // own tokens, next ids
@@ -623,7 +676,7 @@ extern "C" int aasd_verify_static(int device, void* stream, const void* target_l
     a.smp = make_sample_job(p->seed, p->step, false, p->inv_temperature);
     a.out = *out;
     if (n_rows == 0) {
-        if (n_cands > 0) verify_empty_kernel<<<(unsigned int)((n_cands + 255) / 256), 256, 0, s>>>(a);
+        if (n_cands > 0) launch(verify_empty_kernel, (unsigned int)((n_cands + 255) / 256), 256, 0, s, a);
     } else if (a.job.vector_ok && a.job.nvec > 0) {
         StreamJob sj{};
         unsigned int sgrid = 0;
@@ -633,8 +686,8 @@ extern "C" int aasd_verify_static(int device, void* stream, const void* target_l
         if (rc != AASD_OK) return rc;
     } else {
         const unsigned int grid = (unsigned int)(n_rows * a.job.chunks);
-        if (p->dtype == AASD_F32) verify_kernel<AASD_F32><<<grid, kThreads, 0, s>>>(a);
-        else verify_kernel<AASD_BF16><<<grid, kThreads, 0, s>>>(a);
+        if (p->dtype == AASD_F32) launch(verify_kernel<AASD_F32>, grid, kThreads, 0, s, a);
+        else launch(verify_kernel<AASD_BF16>, grid, kThreads, 0, s, a);
     }
     if (cudaGetLastError() != cudaSuccess) return AASD_ERR_CUDA;
     if (status_bits != nullptr)

@@ -84,6 +84,12 @@ __device__ __forceinline__ float ex2_approx(float x) {
     return y;
 }
 
+// ---- programmatic dependent launch -----------------------------------------------------
+// Lets the next kernel of the stream be scheduled early; it still waits for this grid.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
+// Blocks until the preceding kernel of the stream has completed and its writes are visible.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ---- element access ---------------------------------------------------------------------
 template <int DT> struct Elt;
 template <> struct Elt<AASD_F32> {

@@ -293,6 +293,23 @@ __device__ inline RowFinal finish_row(const RowPartial& p, float c1, float neg_r
 
 // ---- conditional verification -----------------------------------------------------------------
 
+// Optional tail of a verification launch: once the last candidate of a sequence is done,
+// choose the longest passing candidate (Sec. 3.3) and append what it emits to the
+// sequence's history (Algorithm 1).  Regular layout only: cands_per_seq candidates per
+// sequence, rows_per_cand rows per candidate.
+struct SeqTail {
+    int enabled;
+    int cands_per_seq;
+    int emit_stride;
+    unsigned int* seq_tickets;   // [n_seqs], zero between launches
+    int32_t* best_cand;
+    int32_t* n_emit;
+    int32_t* emit_ids;
+    int32_t* hist_ids;
+    const int32_t* hist_offsets;
+    int32_t* hist_len;
+};
+
 struct VerifyArgs {
     RowJob job;
     const int32_t* draft_ids;
@@ -306,6 +323,7 @@ struct VerifyArgs {
     uint8_t* row_accept;           // scratch [n_rows]
     int32_t* row_own;              // scratch [n_rows]
     SampleJob smp;                 // STRICT_SAMPLED: the row's own token is a keyed draw
+    SeqTail seq;
     aasd_verify_out out;
 };
 
@@ -440,6 +458,57 @@ __device__ void verify_finish_warp(const VerifyArgs& a, const RowJob& job, int64
         if (a.out.accept_len) a.out.accept_len[c] = (int)n;
         if (a.out.next_token) a.out.next_token[c] = (lo + n < hi) ? __ldcg(a.row_own + lo + n) : AASD_NONE;
     }
+    if (!a.seq.enabled) return;
+
+    // The warp that completes a sequence's last candidate selects and appends.
+    const int cps = a.seq.cands_per_seq;
+    const int b = c / cps;
+    if (lane == 0) {
+        __threadfence();
+        const unsigned int t = atomicAdd(&a.seq.seq_tickets[b], 1u);
+        last = (t == (unsigned int)cps - 1u);
+        if (last) a.seq.seq_tickets[b] = 0;
+    }
+    last = __shfl_sync(0xFFFFFFFFu, last, 0);
+    if (!last) return;
+    __threadfence();
+    // longest accepted prefix, ties to the lowest candidate: key = (length + 1, ~candidate)
+    u64 key = 0;
+    for (int j = lane; j < cps; j += 32) {
+        const int cj = b * cps + j;
+        const u64 k = ((u64)(unsigned int)(__ldcg(a.out.accept_len + cj) + 1) << 32) | (u64)(0xFFFFFFFFu - (unsigned int)cj);
+        key = k > key ? k : key;
+    }
+    key = warp_max_u64(key);
+    int best = AASD_NONE, best_a = 0, ne = 0;
+    if (key != 0) {
+        best = (int)(0xFFFFFFFFu - (unsigned int)key);
+        best_a = (int)(key >> 32) - 1;
+    }
+    const int stride = a.seq.emit_stride;
+    int32_t* e = a.seq.emit_ids + (int64_t)b * stride;
+    const int off = a.seq.hist_offsets[b];
+    const int cap = a.seq.hist_offsets[b + 1] - off;
+    const int len = a.seq.hist_len[b];
+    int nt = AASD_NONE;
+    if (best != AASD_NONE) {
+        nt = __ldcg(a.out.next_token + best);
+        ne = min(best_a, stride);
+        if (nt != AASD_NONE && ne < stride) ne += 1;
+    }
+    for (int i = lane; i < stride; i += 32) {
+        int tok = AASD_NONE;
+        if (i < ne) tok = (i < best_a) ? a.draft_ids[(int64_t)best * a.rows_per_cand + i] : nt;
+        e[i] = tok;
+        if (i < ne && len + i < cap) a.seq.hist_ids[off + len + i] = tok;
+    }
+    __syncwarp();
+    if (lane == 0) {
+        a.seq.best_cand[b] = best;
+        a.seq.n_emit[b] = ne;
+        a.seq.hist_len[b] = min(len + ne, cap);
+        if (len + ne > cap) tally.status |= AASD_STATUS_HIST_OVERFLOW;
+    }
 }
 
 // One CTA (or `chunks` CTAs) per row with plain vector / scalar loads: the path for logits
@@ -447,6 +516,8 @@ __device__ void verify_finish_warp(const VerifyArgs& a, const RowJob& job, int64
 template <int DT>
 __global__ void __launch_bounds__(kThreads) verify_kernel(const VerifyArgs a) {
     __shared__ BlockScratch sc;
+    pdl_launch_dependents();
+    pdl_wait();
     const RowJob& job = a.job;
     const int64_t row = blockIdx.x / job.chunks;
     const int chunk = blockIdx.x % job.chunks;
@@ -472,6 +543,8 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(const VerifyArgs a) {
 
 // Candidates of a call without rows.
 __global__ void verify_empty_kernel(const VerifyArgs a) {
+    pdl_launch_dependents();
+    pdl_wait();
     int c = blockIdx.x * blockDim.x + threadIdx.x;
     if (c < a.n_cands) write_empty_candidate(a, c);
 }
@@ -492,6 +565,8 @@ struct AlignArgs {
 
 // next_ids[t] = prompt_ids[t+1] unless t is the last row of its sequence.
 __global__ void align_next_kernel(const AlignArgs a) {
+    pdl_launch_dependents();
+    pdl_wait();
     int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= a.job.n_rows) return;
     int b = find_segment(a.seq_offsets, a.n_seqs, t);
@@ -596,6 +671,8 @@ __device__ void align_finish_warp(const AlignArgs& a, const RowJob& job, int64_t
 template <int DT, int K>
 __global__ void __launch_bounds__(kThreads) align_kernel(const AlignArgs a) {
     __shared__ BlockScratch sc;
+    pdl_launch_dependents();
+    pdl_wait();
     const RowJob& job = a.job;
     const int64_t row = blockIdx.x / job.chunks;
     const int chunk = blockIdx.x % job.chunks;

@@ -341,7 +341,9 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
         sh.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    pdl_launch_dependents();
     __syncthreads();
+    pdl_wait();   // everything above overlapped the end of the preceding kernel
 
     if (warp < kConsumerWarps) {
         // ------------------------------------------------------------------ consumers

@@ -6,6 +6,7 @@
 namespace aasd {
 
 constexpr int kMaxCands = 64;   // candidates per sequence a draft call can emit
+constexpr int kExtScan = 32;    // depths per main whose extra counts are fetched in parallel
 
 struct DraftArgs {
     aasd_draft_in in;
@@ -25,7 +26,10 @@ __global__ void __launch_bounds__(kThreads) draft_kernel(const DraftArgs a) {
     __shared__ int s_warp[kWarps];
     __shared__ int s_count;
     __shared__ int s_kstar;
+    __shared__ unsigned char s_next[kMaxCands * kExtScan];
 
+    pdl_launch_dependents();
+    pdl_wait();
     const int b = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n = a.p.n, draft_len = a.p.draft_len, max_cands = a.p.max_cands, K = a.p.k_extra;
@@ -125,17 +129,27 @@ __global__ void __launch_bounds__(kThreads) draft_kernel(const DraftArgs a) {
         c_len[c] = c < n_main ? min(draft_len, len - s_pos[c]) : 0;
         c_pos[c] = c < n_main ? s_pos[c] : AASD_NONE;
     }
+    // how many extras each (main, depth) has: fetched by all threads at once, so that the
+    // serial walk below does not pay a trip to memory per step
+    const int scan = min(draft_len, kExtScan);
+    if (have_align && n_main < max_cands) {
+        for (int i = tid; i < n_main * scan; i += kThreads) {
+            const int c = i / scan, depth = i % scan;
+            const int p = s_pos[c];
+            s_next[c * kExtScan + depth] = (unsigned char)(depth < min(draft_len, len - p) ? n_ext(p + depth) : 0);
+        }
+    }
     __syncthreads();
 
     // alternatives: a main's prefix plus one alignment-sampled token (Sec. 3.2), in
     // (main, depth, extra slot) order while slots remain
     if (tid == 0) {
         int total = n_main;
-        for (int c = 0; c < n_main && total < max_cands; ++c) {
+        for (int c = 0; c < n_main && total < max_cands && have_align; ++c) {
             const int p = s_pos[c];
             const int L = min(draft_len, len - p);
             for (int i = 0; i < L && total < max_cands; ++i) {
-                const int ne = n_ext(p + i);
+                const int ne = i < scan ? (int)s_next[c * kExtScan + i] : n_ext(p + i);
                 for (int s = 0; s < ne && total < max_cands; ++s) {
                     const int slot = total++;
                     for (int q = 0; q < i; ++q) {
@@ -171,6 +185,8 @@ struct SelectArgs {
 
 // Longest passing candidate per sequence (Sec. 3.3), ties to the lowest index.
 __global__ void select_kernel(const SelectArgs a) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= a.n_seqs) return;
     const int lo = a.seq_cand_offsets ? a.seq_cand_offsets[b] : b * a.cands_per_seq;
@@ -209,6 +225,8 @@ struct AppendArgs {
 
 // q <- q + y (Algorithm 1), in place, clipped at the buffer's capacity.
 __global__ void append_kernel(const AppendArgs a) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= a.n_seqs) return;
     const int off = a.hist_offsets[b];
