@@ -34,7 +34,7 @@ import torch
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-from paper_2505_13204_b200 import synth  # noqa: E402
+from paper_2505_13204_b200 import shard, synth  # noqa: E402
 
 METRIC = "verified draft positions/sec"
 UNIT = "positions/s"
@@ -46,7 +46,8 @@ N_BUF = 8
 # captures summarised under profiles/: (workload, kernel) -> (rows captured, bytes).  Traffic
 # is proportional to rows (each row is read once), so it is scaled to the launch's rows.
 # An entry is set to None whenever the kernel has changed since its capture.
-NCU_TRAFFIC = {("cfg5-serving-256", "verify"): None, ("cfg5-serving-256", "align"): None}
+NCU_TRAFFIC = {("cfg5-serving-256", "verify"): (2048, 623.016448e6 + 3.948032e6),
+               ("cfg5-serving-256", "align"): (2048, 623.323904e6 + 6.476032e6)}
 
 
 def ncu_traffic(workload: str, kernel: str, rows: int):
@@ -126,7 +127,7 @@ class Bench:
         self.seqs_per_step = max(1, w.batch // w.steps)          # arriving sequences per step
         self.pre_rows = self.seqs_per_step * w.prompt_len
         self.R = w.rows_per_step
-        seed0 = w.seed + 1000 * rank
+        seed0 = shard.rank_seed(w.seed, rank)
         t0 = time.time()
         self.prompts = [synth.prompt_ids(synth.scaled(w, seed=seed0), b) for b in range(w.batch)]
         ids_all = torch.cat(self.prompts).to(device)
@@ -247,17 +248,11 @@ def run_ours(args, rank, world, local_rank):
     align_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in evs]))
     draft_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in evs]))
     verify_ms = float(np.mean([e[2].elapsed_time(e[3]) for e in evs]))
-    if world > 1:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = shard.max_over_ranks(ms, dev)
 
     # end to end: the same step fed from pinned host memory through the C ABI
     e2e = run_e2e(bench, dev, min(K, 4))
-    if world > 1:
-        t = torch.tensor([e2e["ms_per_step"]], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e["ms_per_step"] = float(t.item())
+    e2e["ms_per_step"] = shard.max_over_ranks(e2e["ms_per_step"], dev)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -270,7 +265,7 @@ def run_ours(args, rank, world, local_rank):
     # two launches of aasd_align_sample (next-token gather, ~3 us, + streaming kernel)
     ver_gbs = bench.R * row_bytes / (verify_ms * 1e-3) / 1e9
     ali_gbs = bench.pre_rows * row_bytes / (align_ms * 1e-3) / 1e9
-    value = world * bench.R * K / (ms * 1e-3)
+    value = shard.whole_job_rate(bench.R, K, world, ms)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -516,8 +511,8 @@ def main():
     ap.add_argument("--rows", type=int, default=1024)
     ap.add_argument("--graph", action="store_true", help="--micro: replay the launches from a CUDA graph")
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=64)
-    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--steps", type=int, default=1024)
+    ap.add_argument("--warmup", type=int, default=16)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=4, help="0-based index of the configuration")
     ap.add_argument("--no-cpu-baseline", action="store_true")
