@@ -20,7 +20,7 @@ _lib = None
 NONE = -1
 F32, BF16 = 0, 1
 ALIGN_TOPK, ALIGN_GUMBEL = 0, 1
-VERIFY_CONDITIONAL, VERIFY_STRICT_GREEDY, VERIFY_STRICT_SAMPLED = 0, 1, 2
+VERIFY_CONDITIONAL, VERIFY_STRICT_GREEDY, VERIFY_STRICT_SAMPLED, VERIFY_TOP_K = 0, 1, 2, 3
 
 
 def build(force: bool = False) -> str:
@@ -160,7 +160,7 @@ def draft(hist_ids, hist_offsets, hist_len, prompt_len, recent_ids, recent_len, 
 
 
 def verify(logits, draft_ids, cand_offsets, draft_flags=None, alpha=0.1, beta=0.1,
-           mode=VERIFY_CONDITIONAL, seed=0, step=0, inv_temperature=1.0, threads=1):
+           mode=VERIFY_CONDITIONAL, seed=0, step=0, inv_temperature=1.0, threads=1, top_k=5):
     x, code, stride = _logits(logits)
     R, V = x.shape
     d = _i32(draft_ids).reshape(-1)
@@ -172,14 +172,15 @@ def verify(logits, draft_ids, cand_offsets, draft_flags=None, alpha=0.1, beta=0.
                argmax=np.zeros(R, np.int32), threshold=np.zeros(R),
                accept=np.zeros(R, np.uint8), sampled=np.zeros(R, np.int32),
                near=np.zeros(R, np.uint8), bad=np.zeros(R, np.uint8),
+               n_greater=np.zeros(R, np.int32),
                accept_len=np.zeros(Cn, np.int32), next_token=np.zeros(Cn, np.int32))
     rc = lib().oracle_verify(
         _ptr(x), code, _ptr(d), _ptr(fl), _ptr(offs), Cn, C.c_int64(V), C.c_int64(stride),
         C.c_double(alpha), C.c_double(beta), C.c_double(inv_temperature), int(mode),
-        C.c_uint64(seed), C.c_uint32(step), int(threads), _ptr(out["p_draft"]),
+        C.c_uint64(seed), C.c_uint32(step), int(top_k), int(threads), _ptr(out["p_draft"]),
         _ptr(out["entropy"]), _ptr(out["pmax"]), _ptr(out["argmax"]), _ptr(out["threshold"]),
         _ptr(out["accept"]), _ptr(out["sampled"]), _ptr(out["near"]), _ptr(out["bad"]),
-        _ptr(out["accept_len"]), _ptr(out["next_token"]))
+        _ptr(out["n_greater"]), _ptr(out["accept_len"]), _ptr(out["next_token"]))
     assert rc == 0
     return out
 

@@ -14,7 +14,8 @@
 // (1/2,1/4,1/8,1/8)), hand-computed thresholds of Eq. 5, the worked alignment examples of
 // Sec. 2.3 and Fig. 2, brute-force sorts and 2^len accept patterns on tiny inputs, a
 // naive double loop for the Algorithm-1 dictionary, published Philox4x32-10 known-answer
-// vectors and a chi-square test of the sampler against the exact softmax.
+// vectors and a chi-square test of the sampler against the exact softmax; top-k verification
+// against a full stable sort and the two extreme rows of Sec. 3.3.
 // Parity unpinned: the end-to-end mean acceptance length of the closed-loop driver (it
 // is a statistic of the synthetic inputs; the paper's figures need its datasets and
 // model weights).
@@ -484,6 +485,12 @@ int oracle_draft(const int32_t* hist_ids, const int32_t* hist_offsets, const int
 //   otherwise strict: accept iff d == the target's own token of that row, which is the
 //        argmax (modes 0 and 1 STRICT_GREEDY) or the row's sampled token (mode 2
 //        STRICT_SAMPLED: draw 0 of the sampler, counters row = r, step = step).
+//   mode 3 TOP_K (the alternative the paper argues against in Sec. 3.3 and ablates with
+//        k = 5 in Sec. 4.4) and f.bit0 -> accept iff fewer than top_k tokens are ahead of d
+//        in the order (logit desc, id asc), i.e. d is one of the row's top_k tokens; a
+//        token of probability 0 (logit -inf) never passes; tokens without f.bit0 strict
+//        greedy as in mode 0.
+// n_greater[r] = number of tokens ahead of d in that order (NONE when d is NONE).
 // Candidates are CSR ranges of rows (cand_offsets[C+1]); accept_len = number of leading
 // accepted rows; next_token = the target's own token of row accept_len when that row
 // exists, else NONE.  near[r] = 1 when a conditional decision has
@@ -492,11 +499,11 @@ int oracle_draft(const int32_t* hist_ids, const int32_t* hist_offsets, const int
 int oracle_verify(const void* logits, int dtype, const int32_t* draft_ids,
                   const uint8_t* draft_flags, const int32_t* cand_offsets, int32_t C, int64_t V,
                   int64_t row_stride, double alpha, double beta, double invT, int mode,
-                  uint64_t seed, uint32_t step, int threads, double* p_draft, double* entropy,
-                  double* pmax, int32_t* argmax, double* threshold, uint8_t* accept,
-                  int32_t* sampled, uint8_t* near, uint8_t* bad, int32_t* accept_len,
-                  int32_t* next_token) {
-    if (C < 0 || V <= 0 || mode < 0 || mode > 2) return 1;
+                  uint64_t seed, uint32_t step, int top_k, int threads, double* p_draft,
+                  double* entropy, double* pmax, int32_t* argmax, double* threshold, uint8_t* accept,
+                  int32_t* sampled, uint8_t* near, uint8_t* bad, int32_t* n_greater,
+                  int32_t* accept_len, int32_t* next_token) {
+    if (C < 0 || V <= 0 || mode < 0 || mode > 3) return 1;
     Rows X{logits, dtype, row_stride};
     const int64_t R = cand_offsets[C];
     std::vector<uint8_t> acc(R, 0);
@@ -510,6 +517,13 @@ int oracle_verify(const void* logits, int dtype, const int32_t* draft_ids,
         double pd = 0.0, thr = 0.0;
         int32_t smp = NONE;
         bool a = false, is_near = false;
+        int32_t ahead_of_d = NONE;
+        if (!st.bad && d != NONE) {
+            double yd = X.at(r, d) * invT;
+            ahead_of_d = 0;
+            for (int64_t i = 0; i < V; ++i)
+                if (i != d && ahead(X.at(r, i) * invT, i, yd, d)) ++ahead_of_d;
+        }
         if (!st.bad) {
             if (mode == 2)
                 smp = sample_row(X, r, V, invT, seed, (uint32_t)r, step, DOM_VERIFY_GROUP,
@@ -523,6 +537,9 @@ int oracle_verify(const void* logits, int dtype, const int32_t* draft_ids,
                     bool at_max = (X.at(r, d) * invT == st.m);
                     a = at_max || (pd >= lin);
                     is_near = !at_max && std::fabs(pd - lin) <= 1e-6;
+                } else if (mode == 3 && (f & 1)) {
+                    bool live = X.at(r, d) * invT != -std::numeric_limits<double>::infinity();
+                    a = live && ahead_of_d < top_k;
                 } else {
                     a = (d == own[r]);
                 }
@@ -538,6 +555,7 @@ int oracle_verify(const void* logits, int dtype, const int32_t* draft_ids,
         if (sampled) sampled[r] = smp;
         if (near) near[r] = is_near ? 1 : 0;
         if (bad) bad[r] = st.bad ? 1 : 0;
+        if (n_greater) n_greater[r] = ahead_of_d;
     }
     for (int32_t c = 0; c < C; ++c) {
         int64_t lo = cand_offsets[c], hi = cand_offsets[c + 1];

@@ -262,3 +262,51 @@ def test_select_and_append():
     ov = oracle.append(hist, [0, 4, 8, 12], hist_len, sel["emit_ids"], sel["n_emit"])
     assert list(hist_len) == [4, 1, 4] and list(ov) == [1, 0, 0]
     assert list(hist[2:4]) == [104, 105] and hist[11] == 14
+
+
+def test_top_k_verification_against_full_sort():
+    """Top-k verification (Sec. 3.3, Sec. 4.4 with k = 5): a token passes iff it is one of
+    the k best of its row under (logit descending, id ascending)."""
+    rng = np.random.default_rng(21)
+    R, V = 60, 37
+    x = np.round(rng.standard_normal((R, V)) * 2, 1).astype(np.float32)   # rounded: many ties
+    d = rng.integers(0, V, R).astype(np.int32)
+    offs = np.arange(R + 1, dtype=np.int32)
+    order = np.argsort(-x, axis=1, kind="stable")           # stable: equal logits keep id order
+    rank = np.array([int(np.where(order[r] == d[r])[0][0]) for r in range(R)])
+    for k in (1, 2, 5, 37):
+        out = oracle.verify(x, d, offs, mode=oracle.VERIFY_TOP_K, top_k=k)
+        assert np.array_equal(out["n_greater"], rank)
+        assert np.array_equal(out["accept"], (rank < k).astype(np.uint8))
+    # k = 1 is strict greedy verification
+    g = oracle.verify(x, d, offs, mode=oracle.VERIFY_STRICT_GREEDY)
+    assert np.array_equal(oracle.verify(x, d, offs, mode=oracle.VERIFY_TOP_K, top_k=1)["accept"], g["accept"])
+    # tokens that are not eligible (flag bit 0 clear) are verified strictly
+    fl = np.zeros(R, np.uint8)
+    assert np.array_equal(oracle.verify(x, d, offs, draft_flags=fl, mode=oracle.VERIFY_TOP_K, top_k=5)["accept"],
+                          g["accept"])
+
+
+def test_top_k_on_the_papers_extreme_rows():
+    """Sec. 3.3: with one dominant token top-k still passes k tokens where the probability
+    threshold passes one; with all tokens equal it passes k of them and rejects the rest,
+    where the threshold treats them alike."""
+    V = 16
+    peaked = np.full((V, V), -30.0, np.float32)
+    peaked[:, 3] = 10.0
+    flat = np.zeros((V, V), np.float32)
+    d = np.arange(V, dtype=np.int32)
+    offs = np.arange(V + 1, dtype=np.int32)
+    topk = oracle.verify(peaked, d, offs, mode=oracle.VERIFY_TOP_K, top_k=5)
+    cond = oracle.verify(peaked, d, offs, alpha=0.1, beta=0.1)
+    assert topk["accept"].sum() == 5 and topk["accept"][3] == 1
+    assert cond["accept"].tolist() == [1 if i == 3 else 0 for i in range(V)]
+    topk = oracle.verify(flat, d, offs, mode=oracle.VERIFY_TOP_K, top_k=5)
+    cond = oracle.verify(flat, d, offs, alpha=0.1, beta=0.1)
+    assert topk["accept"].tolist() == [1] * 5 + [0] * 11
+    assert cond["accept"].min() == cond["accept"].max() == 1
+    # a masked token never passes, whatever k
+    masked = np.zeros((1, 4), np.float32)
+    masked[0, 2] = -np.inf
+    out = oracle.verify(masked, np.array([2], np.int32), [0, 1], mode=oracle.VERIFY_TOP_K, top_k=4)
+    assert out["accept"][0] == 0
