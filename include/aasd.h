@@ -66,7 +66,10 @@ typedef enum aasd_align_mode {
 typedef enum aasd_verify_mode {
     AASD_VERIFY_CONDITIONAL = 0,   /* Eq. 4-6 for eligible tokens, strict for the others */
     AASD_VERIFY_STRICT_GREEDY = 1, /* accept iff draft == argmax (Sec. 2.1) */
-    AASD_VERIFY_STRICT_SAMPLED = 2 /* accept iff draft == the row's keyed sample (Eq. 1) */
+    AASD_VERIFY_STRICT_SAMPLED = 2,/* accept iff draft == the row's keyed sample (Eq. 1) */
+    AASD_VERIFY_TOP_K = 3          /* eligible tokens pass iff they are among the row's top_k tokens
+                                      (the alternative of Sec. 3.3, ablated with k = 5 in Sec. 4.4);
+                                      the others strict as in CONDITIONAL */
 } aasd_verify_mode;
 
 /* Bits of the device status word. */
@@ -218,6 +221,7 @@ typedef struct aasd_verify_params {
     int32_t rows_per_cand;  /* used when cand_offsets == NULL: every candidate has this many rows */
     uint32_t step;          /* decoding step, part of the sampler's counter */
     uint64_t seed;
+    int32_t top_k;          /* AASD_VERIFY_TOP_K: how many of the row's best tokens pass (>= 1) */
 } aasd_verify_params;
 
 typedef struct aasd_verify_out {
@@ -230,13 +234,18 @@ typedef struct aasd_verify_out {
     int32_t* sampled;     /* [n_rows] the row's keyed sample (STRICT_SAMPLED), else NONE */
     int32_t* accept_len;  /* [n_cands] leading accepted rows */
     int32_t* next_token;  /* [n_cands] target's own token at the first rejected row, or NONE */
+    int32_t* n_greater;   /* [n_rows] AASD_VERIFY_TOP_K only: tokens ahead of the draft token in the
+                             order (logit descending, id ascending); NONE for a NONE or masked
+                             (-inf) draft token and on bad rows; NONE in the other modes */
 } aasd_verify_out;
 
 /* Row r holds the target distribution that judges draft_ids[r].  draft_flags may be NULL
  * (every row conditional-eligible).  A row is accepted when: CONDITIONAL mode and its flag
  * has AASD_FLAG_CONDITIONAL: p_draft >= min(alpha*H + beta, Delta), where a draft logit
- * equal to the row maximum always passes; otherwise draft == the target's own token
- * (argmax, or the keyed sample in STRICT_SAMPLED).  NONE never passes.  Candidates are CSR
+ * equal to the row maximum always passes; TOP_K mode and that flag: fewer than top_k tokens
+ * are ahead of it (logit descending, id ascending) and its probability is not 0; otherwise
+ * draft == the target's own token (argmax, or the keyed sample in STRICT_SAMPLED).  NONE
+ * never passes.  Candidates are CSR
  * row ranges (cand_offsets[n_cands+1], or regular when NULL); accept_len counts the leading
  * accepted rows and next_token is the target's own token of row accept_len if the
  * candidate has such a row.  n_rows must equal the last offset. */

@@ -490,7 +490,7 @@ int oracle_draft(const int32_t* hist_ids, const int32_t* hist_offsets, const int
 //        in the order (logit desc, id asc), i.e. d is one of the row's top_k tokens; a
 //        token of probability 0 (logit -inf) never passes; tokens without f.bit0 strict
 //        greedy as in mode 0.
-// n_greater[r] = number of tokens ahead of d in that order (NONE when d is NONE).
+// n_greater[r] = number of tokens ahead of d in that order (NONE when d is NONE or masked).
 // Candidates are CSR ranges of rows (cand_offsets[C+1]); accept_len = number of leading
 // accepted rows; next_token = the target's own token of row accept_len when that row
 // exists, else NONE.  near[r] = 1 when a conditional decision has
@@ -520,9 +520,11 @@ int oracle_verify(const void* logits, int dtype, const int32_t* draft_ids,
         int32_t ahead_of_d = NONE;
         if (!st.bad && d != NONE) {
             double yd = X.at(r, d) * invT;
-            ahead_of_d = 0;
-            for (int64_t i = 0; i < V; ++i)
-                if (i != d && ahead(X.at(r, i) * invT, i, yd, d)) ++ahead_of_d;
+            if (yd != -std::numeric_limits<double>::infinity()) {   // a masked token has no rank
+                ahead_of_d = 0;
+                for (int64_t i = 0; i < V; ++i)
+                    if (i != d && ahead(X.at(r, i) * invT, i, yd, d)) ++ahead_of_d;
+            }
         }
         if (!st.bad) {
             if (mode == 2)
@@ -538,8 +540,7 @@ int oracle_verify(const void* logits, int dtype, const int32_t* draft_ids,
                     a = at_max || (pd >= lin);
                     is_near = !at_max && std::fabs(pd - lin) <= 1e-6;
                 } else if (mode == 3 && (f & 1)) {
-                    bool live = X.at(r, d) * invT != -std::numeric_limits<double>::infinity();
-                    a = live && ahead_of_d < top_k;
+                    a = ahead_of_d != NONE && ahead_of_d < top_k;
                 } else {
                     a = (d == own[r]);
                 }

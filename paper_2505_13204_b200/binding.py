@@ -16,7 +16,7 @@ from . import build as _build
 NONE = -1
 F32, BF16 = 0, 1
 ALIGN_TOPK, ALIGN_GUMBEL = 0, 1
-VERIFY_CONDITIONAL, VERIFY_STRICT_GREEDY, VERIFY_STRICT_SAMPLED = 0, 1, 2
+VERIFY_CONDITIONAL, VERIFY_STRICT_GREEDY, VERIFY_STRICT_SAMPLED, VERIFY_TOP_K = 0, 1, 2, 3
 STATUS_BAD_ROW, STATUS_ID_RANGE, STATUS_HIST_OVERFLOW, STATUS_BAD_OFFSETS = 1, 2, 4, 8
 FLAG_CONDITIONAL, FLAG_EXTRA = 1, 2
 DRAFT_MATCH_ALIGN = 1
@@ -64,12 +64,12 @@ class VerifyParams(C.Structure):
     _fields_ = [("vocab", C.c_int32), ("dtype", C.c_int32), ("row_stride", C.c_int64),
                 ("alpha", C.c_float), ("beta", C.c_float), ("inv_temperature", C.c_float),
                 ("mode", C.c_int32), ("rows_per_cand", C.c_int32), ("step", C.c_uint32),
-                ("seed", C.c_uint64)]
+                ("seed", C.c_uint64), ("top_k", C.c_int32)]
 
 
 class VerifyOut(C.Structure):
     _fields_ = [(n, _vp) for n in ("p_draft", "entropy", "pmax", "argmax", "threshold",
-                                   "accept", "sampled", "accept_len", "next_token")]
+                                   "accept", "sampled", "accept_len", "next_token", "n_greater")]
 
 
 class StepArgs(C.Structure):
@@ -163,7 +163,7 @@ def _dev_i32(x, device):
 
 def verify_static(target_logits, draft_ids, cand_offsets=None, draft_flags=None, alpha=0.1,
                   beta=0.1, mode=VERIFY_CONDITIONAL, seed=0, step=0, inv_temperature=1.0,
-                  rows_per_cand=0, outputs=None, status_bits=None, stream=None):
+                  rows_per_cand=0, outputs=None, status_bits=None, stream=None, top_k=5):
     """aasd_verify_static: verification for callers that cannot allocate device memory.
 
     No context and no workspace: the library's own fixed scratch block is used, and the
@@ -191,9 +191,10 @@ def verify_static(target_logits, draft_ids, cand_offsets=None, draft_flags=None,
         accept=torch.empty(R, dtype=torch.uint8, device=dev),
         sampled=torch.empty(R, dtype=torch.int32, device=dev),
         accept_len=torch.empty(Cn, dtype=torch.int32, device=dev),
-        next_token=torch.empty(Cn, dtype=torch.int32, device=dev))
+        next_token=torch.empty(Cn, dtype=torch.int32, device=dev),
+        n_greater=torch.empty(R, dtype=torch.int32, device=dev))
     prm = VerifyParams(V, _dtype_code(x), x.stride(0), float(alpha), float(beta),
-                       float(inv_temperature), int(mode), int(rows_per_cand), int(step), int(seed))
+                       float(inv_temperature), int(mode), int(rows_per_cand), int(step), int(seed), int(top_k))
     out = VerifyOut(*[_p(o.get(n)) for n, _ in VerifyOut._fields_])
     fl = None if draft_flags is None else draft_flags.reshape(-1)
     stream = stream or torch.cuda.current_stream(dev)
@@ -329,7 +330,7 @@ class Context:
 
     def verify(self, target_logits, draft_ids, cand_offsets=None, draft_flags=None, alpha=0.1,
                beta=0.1, mode=VERIFY_CONDITIONAL, seed=0, step=0, inv_temperature=1.0,
-               rows_per_cand=0, outputs=None):
+               rows_per_cand=0, outputs=None, top_k=5):
         """aasd_verify.  ``cand_offsets=None`` means regular candidates of ``rows_per_cand``."""
         x = target_logits
         assert x.is_cuda and x.dim() == 2 and x.stride(1) == 1
@@ -347,10 +348,11 @@ class Context:
             accept=torch.empty(R, dtype=torch.uint8, device=dev),
             sampled=torch.empty(R, dtype=torch.int32, device=dev),
             accept_len=torch.empty(Cn, dtype=torch.int32, device=dev),
-            next_token=torch.empty(Cn, dtype=torch.int32, device=dev))
+            next_token=torch.empty(Cn, dtype=torch.int32, device=dev),
+            n_greater=torch.empty(R, dtype=torch.int32, device=dev))
         prm = VerifyParams(V, _dtype_code(x), x.stride(0), float(alpha), float(beta),
                            float(inv_temperature), int(mode), int(rows_per_cand), int(step),
-                           int(seed))
+                           int(seed), int(top_k))
         out = VerifyOut(*[_p(o.get(n)) for n, _ in VerifyOut._fields_])
         ws = self.workspace(R, Cn)
         fl = None if draft_flags is None else draft_flags.reshape(-1)
@@ -386,7 +388,7 @@ class DecodeState:
 
     def __init__(self, ctx: Context, prompts, capacity_extra: int, n: int, draft_len: int,
                  max_cands: int, vocab: int, dtype: torch.dtype, align=None, alpha=0.1, beta=0.1,
-                 mode=VERIFY_CONDITIONAL, inv_temperature=1.0, seed=0, match_align=False):
+                 mode=VERIFY_CONDITIONAL, inv_temperature=1.0, seed=0, match_align=False, top_k=5):
         dev = ctx.device
         self.ctx = ctx
         B = len(prompts)
@@ -426,7 +428,8 @@ class DecodeState:
             accept=torch.empty(R, dtype=torch.uint8, device=dev),
             sampled=torch.empty(R, dtype=torch.int32, device=dev),
             accept_len=torch.empty(Cn, dtype=torch.int32, device=dev),
-            next_token=torch.empty(Cn, dtype=torch.int32, device=dev))
+            next_token=torch.empty(Cn, dtype=torch.int32, device=dev),
+            n_greater=torch.empty(R, dtype=torch.int32, device=dev))
         self.best_cand = torch.empty(B, dtype=torch.int32, device=dev)
         self.n_emit = torch.empty(B, dtype=torch.int32, device=dev)
         self.emit_ids = torch.empty((B, draft_len + 1), dtype=torch.int32, device=dev)
@@ -443,7 +446,7 @@ class DecodeState:
         a.draft_out = DraftOut(*[_p(self.draft_out[k]) for k, _ in DraftOut._fields_])
         a.verify = VerifyParams(vocab, F32 if dtype == torch.float32 else BF16, vocab, float(alpha),
                                 float(beta), float(inv_temperature), int(mode), draft_len, 0,
-                                int(seed))
+                                int(seed), int(top_k))
         a.verify_out = VerifyOut(*[_p(self.verify_out[k]) for k, _ in VerifyOut._fields_])
         a.hist_ids, a.hist_len = _p(self.hist_ids), _p(self.hist_len)
         a.best_cand, a.n_emit, a.emit_ids = _p(self.best_cand), _p(self.n_emit), _p(self.emit_ids)

@@ -209,7 +209,7 @@ int enable_stream_smem(Kernel kernel) {
 
 template <int DT, int K, int ND>
 int launch_align_stream(aasd_ctx* ctx, const StreamJob& sj, const AlignArgs& a, unsigned int grid) {
-    auto kernel = stream_kernel<DT, K, ND, AlignEpilogue<DT>>;
+    auto kernel = stream_kernel<DT, K, ND, false, AlignEpilogue<DT>>;
     if (enable_stream_smem(kernel) != AASD_OK) return AASD_ERR_CUDA;
     launch(kernel, grid, kStreamThreads, kStreamSmemBytes, ctx->stream, sj, a);
     return AASD_OK;
@@ -230,9 +230,9 @@ int dispatch_align_stream(aasd_ctx* ctx, const StreamJob& sj, const AlignArgs& a
     return launch_align_stream<DT, 4, 0>(ctx, sj, a, grid);
 }
 
-template <int DT, int ND>
+template <int DT, int ND, bool TK>
 int launch_verify_stream(aasd_ctx* ctx, const StreamJob& sj, const VerifyArgs& a, unsigned int grid) {
-    auto kernel = stream_kernel<DT, 1, ND, VerifyEpilogue<DT>>;
+    auto kernel = stream_kernel<DT, 1, ND, TK, VerifyEpilogue<DT>>;
     if (enable_stream_smem(kernel) != AASD_OK) return AASD_ERR_CUDA;
     launch(kernel, grid, kStreamThreads, kStreamSmemBytes, ctx->stream, sj, a);
     return AASD_OK;
@@ -240,8 +240,9 @@ int launch_verify_stream(aasd_ctx* ctx, const StreamJob& sj, const VerifyArgs& a
 
 template <int DT>
 int dispatch_verify_stream(aasd_ctx* ctx, const StreamJob& sj, const VerifyArgs& a, unsigned int grid) {
-    return a.mode == AASD_VERIFY_STRICT_SAMPLED ? launch_verify_stream<DT, 1>(ctx, sj, a, grid)
-                                                : launch_verify_stream<DT, 0>(ctx, sj, a, grid);
+    if (a.mode == AASD_VERIFY_STRICT_SAMPLED) return launch_verify_stream<DT, 1, false>(ctx, sj, a, grid);
+    if (a.mode == AASD_VERIFY_TOP_K) return launch_verify_stream<DT, 0, true>(ctx, sj, a, grid);
+    return launch_verify_stream<DT, 0, false>(ctx, sj, a, grid);
 }
 
 SampleJob make_sample_job(uint64_t seed, uint32_t step, bool align, float inv_temperature) {
@@ -446,7 +447,8 @@ int verify_impl(aasd_ctx* ctx, const void* target_logits, const int32_t* draft_i
                 void* workspace, size_t workspace_bytes, const aasd_verify_out* out, const SeqTail* seq) {
     if (ctx == nullptr || p == nullptr || out == nullptr) return AASD_ERR_INVALID_ARG;
     if (n_cands < 0 || n_rows < 0) return AASD_ERR_BAD_SHAPE;
-    if (p->mode < AASD_VERIFY_CONDITIONAL || p->mode > AASD_VERIFY_STRICT_SAMPLED) return AASD_ERR_INVALID_ARG;
+    if (p->mode < AASD_VERIFY_CONDITIONAL || p->mode > AASD_VERIFY_TOP_K) return AASD_ERR_INVALID_ARG;
+    if (p->mode == AASD_VERIFY_TOP_K && p->top_k < 1) return AASD_ERR_INVALID_ARG;
     if (!(p->alpha >= 0.f) || !(p->beta >= 0.f)) return AASD_ERR_INVALID_ARG;
     if (cand_offsets == nullptr) {
         if (p->rows_per_cand < 1 || (int64_t)n_cands * p->rows_per_cand != n_rows) return AASD_ERR_BAD_SHAPE;
@@ -468,6 +470,7 @@ int verify_impl(aasd_ctx* ctx, const void* target_logits, const int32_t* draft_i
     a.alpha = p->alpha;
     a.beta = p->beta;
     a.mode = p->mode;
+    a.top_k = p->top_k;
     a.cand_tickets = reinterpret_cast<unsigned int*>(ws + L->off_cand_tickets);
     a.row_accept = reinterpret_cast<uint8_t*>(ws + L->off_row_accept);
     a.row_own = reinterpret_cast<int32_t*>(ws + L->off_row_own);
@@ -619,7 +622,8 @@ extern "C" int aasd_verify_static(int device, void* stream, const void* target_l
     if (device < 0 || device >= kStaticMaxDevices) return AASD_ERR_INVALID_ARG;
     if (n_cands < 0 || n_rows < 0) return AASD_ERR_BAD_SHAPE;
     if (n_rows > kStaticMaxRows || n_cands > kStaticMaxCands) return AASD_ERR_WORKSPACE_TOO_SMALL;
-    if (p->mode < AASD_VERIFY_CONDITIONAL || p->mode > AASD_VERIFY_STRICT_SAMPLED) return AASD_ERR_INVALID_ARG;
+    if (p->mode < AASD_VERIFY_CONDITIONAL || p->mode > AASD_VERIFY_TOP_K) return AASD_ERR_INVALID_ARG;
+    if (p->mode == AASD_VERIFY_TOP_K && p->top_k < 1) return AASD_ERR_INVALID_ARG;
     if (!(p->alpha >= 0.f) || !(p->beta >= 0.f)) return AASD_ERR_INVALID_ARG;
     if (cand_offsets == nullptr) {
         if (p->rows_per_cand < 1 || (int64_t)n_cands * p->rows_per_cand != n_rows) return AASD_ERR_BAD_SHAPE;
@@ -670,6 +674,7 @@ extern "C" int aasd_verify_static(int device, void* stream, const void* target_l
     a.alpha = p->alpha;
     a.beta = p->beta;
     a.mode = p->mode;
+    a.top_k = p->top_k;
     a.cand_tickets = reinterpret_cast<unsigned int*>(ws + L.off_cand_tickets);
     a.row_accept = reinterpret_cast<uint8_t*>(ws + L.off_row_accept);
     a.row_own = reinterpret_cast<int32_t*>(ws + L.off_row_own);

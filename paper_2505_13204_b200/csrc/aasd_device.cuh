@@ -37,6 +37,7 @@ struct RowPartial {
     double S;          // sum 2^(x*c1 - refc)
     double A;          // sum 2^(x*c1 - refc) * (x*c1 - refc)
     u64 key[kMaxK];    // best tokens, descending; 0 = empty
+    long long ahead;   // top-k verification: tokens counted ahead of the draft token so far
 };
 
 // ---- ordered keys: larger logit first, equal logits by lower id --------------------
@@ -73,6 +74,12 @@ __device__ __forceinline__ u64 warp_max_u64(u64 v) {
     return v;
 }
 __device__ __forceinline__ double warp_sum_f64(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+
+__device__ __forceinline__ long long warp_sum_i64(long long v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
     return v;

@@ -323,6 +323,7 @@ struct VerifyArgs {
     uint8_t* row_accept;           // scratch [n_rows]
     int32_t* row_own;              // scratch [n_rows]
     SampleJob smp;                 // STRICT_SAMPLED: the row's own token is a keyed draw
+    int top_k;                     // TOP_K mode
     SeqTail seq;
     aasd_verify_out out;
 };
@@ -362,7 +363,8 @@ struct Tally {
 // Eq. 4-6 for one row, by one thread, once the row's sums and best token are known: writes
 // the row's outputs and its accept bit / own token for the prefix rule.  d is the row's
 // draft id as given, xd its raw logit (read only when d lies inside the vocabulary), sampled
-// the row's keyed draw in STRICT_SAMPLED mode (NONE otherwise, and on a bad row).
+// the row's keyed draw in STRICT_SAMPLED mode (NONE otherwise, and on a bad row).  In TOP_K
+// mode merged.ahead is the number of tokens ahead of d in the order (logit desc, id asc).
 template <int DT>
 __device__ void verify_row(const VerifyArgs& a, const RowJob& job, int64_t row, const RowPartial& merged,
                            float neg_refc, bool centered, int d, float xd, int sampled, Tally& tally) {
@@ -382,10 +384,15 @@ __device__ void verify_row(const VerifyArgs& a, const RowJob& job, int64_t row, 
             const bool at_max = (xd == f.m);
             acc = at_max || (pd >= lin);
             near = !at_max && fabs(pd - lin) <= 1.0e-6;
+        } else if (a.mode == AASD_VERIFY_TOP_K && (flag & AASD_FLAG_CONDITIONAL)) {
+            acc = xd > -CUDART_INF_F && merged.ahead < (long long)a.top_k;
         } else {
             acc = (d == own);
         }
     }
+    if (a.out.n_greater)
+        a.out.n_greater[row] = (a.mode == AASD_VERIFY_TOP_K && d_ok && !f.bad && xd > -CUDART_INF_F)
+                                   ? (int)merged.ahead : AASD_NONE;
     if (a.out.p_draft) a.out.p_draft[row] = (float)pd;
     if (a.out.entropy) a.out.entropy[row] = (float)f.H;
     if (a.out.pmax) a.out.pmax[row] = (float)f.pmax;
@@ -536,6 +543,19 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(const VerifyArgs a) {
         // this layout takes the definition as it stands: every group scored in fp64
         sampled = warp_sample_exhaustive<DT>(rowp, job.vocab, (unsigned int)row, 0, a.smp);
         tally.exhaustive += 1;
+    }
+    if (a.mode == AASD_VERIFY_TOP_K) {
+        // and counts the tokens ahead of the draft token by going over the row once more
+        long long n = 0;
+        if (d_ok)
+            for (int i = threadIdx.x; i < job.vocab; i += 32) {
+                const float x = Elt<DT>::load(rowp, i);
+                n += (x > xd || (x == xd && i < d)) ? 1 : 0;
+            }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) n += __shfl_xor_sync(0xFFFFFFFFu, n, o);
+        sc.merged.ahead = n;
+        __syncwarp();
     }
     verify_finish_warp<DT>(a, job, row, sc.merged, neg_refc, centered, d, xd, sampled, tally);
     if (threadIdx.x == 0) tally.flush(job.state);

@@ -97,6 +97,7 @@ constexpr int kNoItem = -1;
 struct WarpPartial {
     double S, A;
     u64 key[kMaxK];   // vector-level: (ordered vector maximum << 32) | ~vector index
+    long long ahead;  // top-k verification: tokens counted ahead of the draft token
 };
 struct StreamShared {
     u64 full[kStages];
@@ -244,6 +245,79 @@ struct TileAccumulator {
     }
 };
 
+// Top-k verification (Sec. 3.3): counts, per thread, the tokens that are ahead of the row's
+// draft token d in the order (logit descending, id ascending).  A token with a lower id is
+// ahead when its logit is >= x_d, one with a higher id when it is > x_d; ">= x_d" is taken
+// as "> the next value below x_d", so every vector needs one comparison per lane with a
+// threshold chosen by its position relative to d's own vector.  The vector that holds d is
+// compared with "> x_d" and the finisher adds its lower-id ties.
+template <int DT> struct AheadCounter;
+template <> struct AheadCounter<AASD_BF16> {
+    unsigned int thr_gt, thr_ge;   // bf16x2: x_d twice, and the next bf16 below x_d twice
+    unsigned int acc;              // bf16x2 running counts of the current tile (exact: <= 16 each)
+    int vd;                        // vector index of d
+    int count;
+    __device__ __forceinline__ void begin_item(int d, float xd, bool valid) {
+        count = 0;
+        acc = 0;
+        vd = d / 8;
+        unsigned int b = __float_as_uint(xd) >> 16;
+        unsigned int below = (b & 0x7FFFu) == 0 ? 0x8001u : ((b & 0x8000u) ? b + 1 : b - 1);
+        if (!valid || !(xd > -CUDART_INF_F)) b = below = 0x7F80u;   // +inf: nothing is ahead
+        thr_gt = b | (b << 16);
+        thr_ge = (below & 0xFFFFu) | (below << 16);
+    }
+    __device__ __forceinline__ void add(const uint4& q, int vec) {
+        const unsigned int thr = vec < vd ? thr_ge : thr_gt;
+        unsigned int r;
+        asm("set.gt.bf16x2.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(q.x), "r"(thr));
+        asm("add.rn.bf16x2 %0, %1, %2;" : "=r"(acc) : "r"(acc), "r"(r));
+        asm("set.gt.bf16x2.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(q.y), "r"(thr));
+        asm("add.rn.bf16x2 %0, %1, %2;" : "=r"(acc) : "r"(acc), "r"(r));
+        asm("set.gt.bf16x2.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(q.z), "r"(thr));
+        asm("add.rn.bf16x2 %0, %1, %2;" : "=r"(acc) : "r"(acc), "r"(r));
+        asm("set.gt.bf16x2.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(q.w), "r"(thr));
+        asm("add.rn.bf16x2 %0, %1, %2;" : "=r"(acc) : "r"(acc), "r"(r));
+    }
+    // after at most 4 vectors (32 ids): move the packed counts to the integer counter
+    __device__ __forceinline__ void end_tile() {
+        count += (int)__uint_as_float(acc << 16) + (int)__uint_as_float(acc & 0xFFFF0000u);
+        acc = 0;
+    }
+};
+template <> struct AheadCounter<AASD_F32> {
+    float thr_gt, thr_ge;
+    float acc;
+    int vd;
+    int count;
+    __device__ __forceinline__ void begin_item(int d, float xd, bool valid) {
+        count = 0;
+        acc = 0.f;
+        vd = d / 4;
+        const unsigned int b = __float_as_uint(xd);
+        const unsigned int below = (b & 0x7FFFFFFFu) == 0 ? 0x80000001u : ((b & 0x80000000u) ? b + 1 : b - 1);
+        thr_gt = xd;
+        thr_ge = __uint_as_float(below);
+        if (!valid || !(xd > -CUDART_INF_F)) thr_gt = thr_ge = CUDART_INF_F;
+    }
+    __device__ __forceinline__ void add(const uint4& q, int vec) {
+        const float thr = vec < vd ? thr_ge : thr_gt;
+        float r;
+        asm("set.gt.f32.f32 %0, %1, %2;" : "=f"(r) : "f"(__uint_as_float(q.x)), "f"(thr));
+        acc += r;
+        asm("set.gt.f32.f32 %0, %1, %2;" : "=f"(r) : "f"(__uint_as_float(q.y)), "f"(thr));
+        acc += r;
+        asm("set.gt.f32.f32 %0, %1, %2;" : "=f"(r) : "f"(__uint_as_float(q.z)), "f"(thr));
+        acc += r;
+        asm("set.gt.f32.f32 %0, %1, %2;" : "=f"(r) : "f"(__uint_as_float(q.w)), "f"(thr));
+        acc += r;
+    }
+    __device__ __forceinline__ void end_tile() {
+        count += (int)acc;
+        acc = 0.f;
+    }
+};
+
 // The same for a sampling kernel: the sum of the vector's weights goes to `gs` (the caller
 // adds a whole group's sum to S at once, and needs it for the group's ratio).
 template <int DT, int K>
@@ -316,7 +390,8 @@ struct FinishedRow {
 //   E::finish<ND>(args, job, row, rowp, FinishedRow&, ItemInfo&, races, tail_group, Tally&)
 //   - entered by the whole finisher warp
 //   ND: keyed draws per row the kernel prepares (0: no sampling)
-template <int DT, int K, int ND, class E>
+//   TK: count the tokens ahead of the hinted token (top-k verification)
+template <int DT, int K, int ND, bool TK, class E>
 __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJob job, const typename E::Args args) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* tiles = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
@@ -353,6 +428,8 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
             acc.init();
             GroupRace<(ND > 0 ? ND : 1)> race;
             race.init();
+            AheadCounter<DT> ahead;
+            ahead.count = 0;
             unsigned int row_ctr = 0;
             float neg_refc = 0.f;
             bool alive = true, last = false;
@@ -374,6 +451,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
                     }
                     neg_refc = info.neg_refc;
                     row_ctr = (unsigned int)info.row;
+                    if (TK) ahead.begin_item(info.hint, info.hint_logit, info.hint >= 0 && info.hint < rj.vocab);
                     tile_range(job, info.row, info.chunk, tb, te);
                 }
                 const unsigned char* base = tiles + (size_t)s * kTileBytes;
@@ -411,8 +489,18 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
                     for (int k = 0; k < kTileVecs / kConsumers; ++k) q[k] = lds16(base + (size_t)(k * kConsumers + tid) * 16);
 #pragma unroll
                     for (int k = 0; k < kTileVecs / kConsumers; ++k) acc.add(q[k], v0 + k * kConsumers + tid, c1, neg_refc);
+                    if (TK) {
+#pragma unroll
+                        for (int k = 0; k < kTileVecs / kConsumers; ++k) ahead.add(q[k], v0 + k * kConsumers + tid);
+                        ahead.end_tile();
+                    }
                 } else {
-                    for (int v = tid; v < nv; v += kConsumers) acc.add(lds16(base + (size_t)v * 16), v0 + v, c1, neg_refc);
+                    for (int v = tid; v < nv; v += kConsumers) {
+                        const uint4 q = lds16(base + (size_t)v * 16);
+                        acc.add(q, v0 + v, c1, neg_refc);
+                        if (TK) ahead.add(q, v0 + v);
+                    }
+                    if (TK) ahead.end_tile();
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sh.empty[s]);
@@ -465,8 +553,11 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
                     }
                 }
             }
+            int n_ahead = 0;
+            if (TK) n_ahead = __reduce_add_sync(0xFFFFFFFFu, ahead.count);
             if (lane == 0) {
                 WarpPartial& w = sh.wp[p][warp];
+                w.ahead = n_ahead;
                 w.S = S;
                 w.A = A;
 #pragma unroll
@@ -584,10 +675,12 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
 #pragma unroll
         for (int j = 0; j < K; ++j) vk[j] = 0;
         RaceSummary races[ND > 0 ? ND : 1];   // per draw, the same in every lane once merged
+        long long n_ahead = 0;
         if (lane < kConsumerWarps) {
             const WarpPartial& w = sh.wp[p][lane];
             S = w.S;
             A = w.A;
+            if (TK) n_ahead = w.ahead;
 #pragma unroll
             for (int j = 0; j < K; ++j) vk[j] = w.key[j];
         }
@@ -610,6 +703,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
         if (lane == 0) mbar_arrive(&sh.freeb[p]);
         S = warp_sum_f64(S);
         A = warp_sum_f64(A);
+        if (TK) n_ahead = warp_sum_i64(n_ahead);
         u64 mk[K];   // merged vector keys, identical in every lane
 #pragma unroll
         for (int r = 0; r < K; ++r) {
@@ -631,6 +725,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
                 mine.A = A;
 #pragma unroll
                 for (int j = 0; j < kMaxK; ++j) mine.key[j] = j < K ? mk[j] : 0ull;
+                mine.ahead = n_ahead;
                 slots[chunk] = mine;
                 if (ND > 0) {
                     RaceSummary* rp = job.race_partials + ((row - job.whole_rows) * chunks + chunk) * kMaxK;
@@ -647,17 +742,20 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
             __threadfence();
             S = 0.0;
             A = 0.0;
+            n_ahead = 0;
 #pragma unroll
             for (int j = 0; j < K; ++j) vk[j] = 0;
             for (int c = lane; c < chunks; c += 32) {
                 const RowPartial* q = slots + c;
                 S += __ldcg(&q->S);
                 A += __ldcg(&q->A);
+                if (TK) n_ahead += __ldcg(&q->ahead);
 #pragma unroll
                 for (int j = 0; j < K; ++j) key_insert<K>(vk, __ldcg(&q->key[j]));
             }
             S = warp_sum_f64(S);
             A = warp_sum_f64(A);
+            if (TK) n_ahead = warp_sum_i64(n_ahead);
 #pragma unroll
             for (int r = 0; r < K; ++r) {
                 const u64 m = warp_max_u64(vk[0]);
@@ -744,6 +842,26 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
         }
         fr.merged.S = S;
         fr.merged.A = A;
+        fr.merged.ahead = 0;
+        if (TK) {
+            // what the consumers could not see: lower-id ties inside d's own vector, and the
+            // ids of the ragged tail
+            const int d = info.hint;
+            long long extra = 0;
+            if (d >= 0 && d < rj.vocab && info.hint_logit > -CUDART_INF_F) {
+                const float xd = info.hint_logit;
+                const int vd = d / kVec;
+                if (vd < rj.nvec) {
+                    const int i = vd * kVec + lane;
+                    if (lane < kVec && i < d && Elt<DT>::load(rowp, i) == xd) extra += 1;
+                }
+                for (int i = rj.nvec * kVec + lane; i < rj.vocab; i += 32) {
+                    const float x = Elt<DT>::load(rowp, i);
+                    extra += (x > xd || (x == xd && i < d)) ? 1 : 0;
+                }
+            }
+            fr.merged.ahead = n_ahead + warp_sum_i64(extra);
+        }
         // ids beyond the last complete group of the vector part were not raced
         const int tail_group = (ND > 0 && job.full_groups * kGroup < rj.vocab) ? job.full_groups : -1;
         E::template finish<ND>(args, rj, row, rowp, fr, info, races, tail_group, tally);

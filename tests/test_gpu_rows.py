@@ -173,6 +173,36 @@ def test_align_gumbel_parity(ctx, V, dtype, stride, rows, K):
     assert ctx.poll_status() == 0
 
 
+@pytest.mark.parametrize("V,dtype,stride,rows", SAMPLED_CASES)
+def test_verify_top_k_parity(ctx, V, dtype, stride, rows):
+    """Top-k verification (Sec. 3.3 / Sec. 4.4): the count of tokens ahead of the draft token
+    is an integer and must be exact, ties included (bf16 rows are full of equal logits)."""
+    rng = np.random.default_rng(5 * V + rows)
+    d = rng.integers(0, V, rows).astype(np.int32)
+    x = _make_logits(rows, V, dtype, 500 + V, torch.as_tensor(d, dtype=torch.int64), stride=stride)
+    xf = x.float().numpy()
+    order = np.argsort(-xf, axis=1, kind="stable")
+    pick = rng.random(rows)
+    for r in range(rows):          # drafts spread over the top ranks, where the decision is taken
+        if pick[r] < 0.6:
+            d[r] = order[r, int(rng.integers(0, min(V, 9)))]
+    d[pick > 0.97] = -1
+    if rows > 10:
+        d[3] = V + 5
+        x[5, d[5] if d[5] >= 0 else 0] = -float("inf")     # a masked draft token
+        x[6, :] = x[6, 0]                                   # every token equal: ids decide
+    flags = rng.integers(0, 4, rows).astype(np.uint8)
+    offs = _random_csr(rng, rows)
+    for k in (1, 5):
+        ref = oracle.verify(to_oracle(x), d, offs, draft_flags=flags, mode=oracle.VERIFY_TOP_K, top_k=k)
+        got = ctx.verify(_to_dev(x), torch.as_tensor(d).cuda(), torch.as_tensor(offs).cuda(),
+                         draft_flags=torch.as_tensor(flags).cuda(), mode=binding.VERIFY_TOP_K, top_k=k)
+        assert np.array_equal(cpu(got["n_greater"]), ref["n_greater"])
+        check_verify(got, ref, offs, dtype)
+    assert ref["accept"].sum() > 0
+    ctx.poll_status()
+
+
 def test_sampler_on_flat_and_masked_rows(ctx):
     """Rows where many groups are equally likely, rows with masked ids, one live token."""
     V, rows = 8192, 16
@@ -288,7 +318,7 @@ def test_host_side_errors(ctx):
     assert e.value.code == 1
     # an unregistered workspace is refused before anything is launched
     import ctypes as C
-    prm = binding.VerifyParams(64, 0, 64, 0.1, 0.1, 1.0, 0, 0, 0, 0)
+    prm = binding.VerifyParams(64, 0, 64, 0.1, 0.1, 1.0, 0, 0, 0, 0, 5)
     out = binding.VerifyOut()
     junk = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
     rc = ctx.lib.aasd_verify(ctx._h, xf.data_ptr(), d.data_ptr(), None,
