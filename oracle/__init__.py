@@ -185,6 +185,48 @@ def verify(logits, draft_ids, cand_offsets, draft_flags=None, alpha=0.1, beta=0.
     return out
 
 
+def tree_build(draft_ids, draft_flags, cand_len, n_cands):
+    """Draft candidates [B x max_cands x draft_len] -> draft trees (Eq. 2), one per sequence,
+    each in 1 + max_cands*draft_len node slots."""
+    d = np.ascontiguousarray(draft_ids, np.int32)
+    f = np.ascontiguousarray(draft_flags, np.uint8)
+    B, Cm, Ld = d.shape
+    cap = 1 + Cm * Ld
+    out = dict(node_token=np.zeros((B, cap), np.int32), node_parent=np.zeros((B, cap), np.int32),
+               node_flags=np.zeros((B, cap), np.uint8), node_depth=np.zeros((B, cap), np.int32),
+               n_nodes=np.zeros(B, np.int32))
+    rc = lib().oracle_tree_build(_ptr(d), _ptr(f), _ptr(_i32(cand_len)), _ptr(_i32(n_cands)), B, Cm, Ld,
+                                 _ptr(out["node_token"]), _ptr(out["node_parent"]),
+                                 _ptr(out["node_flags"]), _ptr(out["node_depth"]), _ptr(out["n_nodes"]))
+    assert rc == 0
+    return out
+
+
+def verify_tree(logits, node_token, node_parent, tree_offsets, emit_stride, node_flags=None, alpha=0.1,
+                beta=0.1, mode=VERIFY_CONDITIONAL, seed=0, step=0, inv_temperature=1.0, threads=1):
+    x, code, stride = _logits(logits)
+    R, V = x.shape
+    tok, par = _i32(node_token).reshape(-1), _i32(node_parent).reshape(-1)
+    offs = _i32(tree_offsets)
+    T = len(offs) - 1
+    assert offs[-1] == R == tok.size == par.size
+    fl = None if node_flags is None else np.ascontiguousarray(node_flags, np.uint8).reshape(-1)
+    out = dict(p_token=np.zeros(R), entropy=np.zeros(R), pmax=np.zeros(R), argmax=np.zeros(R, np.int32),
+               threshold=np.zeros(R), accept=np.zeros(R, np.uint8), sampled=np.zeros(R, np.int32),
+               near=np.zeros(R, np.uint8), bad=np.zeros(R, np.uint8), best_node=np.zeros(T, np.int32),
+               n_accept=np.zeros(T, np.int32), n_emit=np.zeros(T, np.int32),
+               emit_ids=np.zeros((T, emit_stride), np.int32))
+    rc = lib().oracle_verify_tree(
+        _ptr(x), code, _ptr(tok), _ptr(par), _ptr(fl), _ptr(offs), T, C.c_int64(V), C.c_int64(stride),
+        C.c_double(alpha), C.c_double(beta), C.c_double(inv_temperature), int(mode), C.c_uint64(seed),
+        C.c_uint32(step), int(threads), int(emit_stride), _ptr(out["p_token"]), _ptr(out["entropy"]),
+        _ptr(out["pmax"]), _ptr(out["argmax"]), _ptr(out["threshold"]), _ptr(out["accept"]),
+        _ptr(out["sampled"]), _ptr(out["near"]), _ptr(out["bad"]), _ptr(out["best_node"]),
+        _ptr(out["n_accept"]), _ptr(out["n_emit"]), _ptr(out["emit_ids"]))
+    assert rc == 0
+    return out
+
+
 def select(accept_len, next_token, draft_ids, cand_offsets, seq_cand_offsets, emit_stride):
     accept_len, next_token = _i32(accept_len), _i32(next_token)
     d = _i32(draft_ids).reshape(-1)

@@ -15,7 +15,9 @@
 // Sec. 2.3 and Fig. 2, brute-force sorts and 2^len accept patterns on tiny inputs, a
 // naive double loop for the Algorithm-1 dictionary, published Philox4x32-10 known-answer
 // vectors and a chi-square test of the sampler against the exact softmax; top-k verification
-// against a full stable sort and the two extreme rows of Sec. 3.3.
+// against a full stable sort and the two extreme rows of Sec. 3.3; the draft tree against the
+// set of distinct candidate prefixes, tree verification against the longest passing flat
+// candidate over all root-to-leaf paths and against plain sampled decoding along the tree.
 // Parity unpinned: the end-to-end mean acceptance length of the closed-loop driver (it
 // is a statistic of the synthetic inputs; the paper's figures need its datasets and
 // model weights).
@@ -564,6 +566,166 @@ int oracle_verify(const void* logits, int dtype, const int32_t* draft_ids,
         while (lo + a < hi && acc[lo + a]) ++a;
         if (accept_len) accept_len[c] = a;
         if (next_token) next_token[c] = (lo + a < hi) ? own[lo + a] : NONE;
+    }
+    return 0;
+}
+
+// ---------------------------------------------------------------------------------
+// O-T: the draft tree of Eq. 2 (Sec. 3.2): the candidate n-grams of a sequence, expanded
+// by alignment sampling, are merged into one tree.  Node 0 of a tree is its root (the last
+// token of the current sequence; it carries no draft token).  The candidates are walked in
+// order; at each depth the walk moves to the child that carries the same token (children
+// are searched in creation order) or creates it, so nodes are numbered in creation order
+// and a parent always precedes its children.  A node reached by several candidates keeps
+// the OR of their token flags.
+// Inputs per sequence b: draft_ids/draft_flags [max_cands x draft_len], cand_len, n_cands as
+// oracle_draft writes them.  Outputs per sequence, max_nodes = 1 + max_cands*draft_len slots:
+// node_token (NONE for the root and unused slots), node_parent (index inside the tree, NONE
+// for the root and unused slots), node_flags, node_depth, and n_nodes[b].
+// ---------------------------------------------------------------------------------
+int oracle_tree_build(const int32_t* draft_ids, const uint8_t* draft_flags, const int32_t* cand_len,
+                      const int32_t* n_cands, int32_t B, int max_cands, int draft_len,
+                      int32_t* node_token, int32_t* node_parent, uint8_t* node_flags,
+                      int32_t* node_depth, int32_t* n_nodes) {
+    if (B < 0 || max_cands < 1 || draft_len < 1) return 1;
+    const int64_t cap = 1 + (int64_t)max_cands * draft_len;
+    for (int32_t b = 0; b < B; ++b) {
+        int32_t* tok = node_token + b * cap;
+        int32_t* par = node_parent + b * cap;
+        uint8_t* fl = node_flags + b * cap;
+        int32_t* dep = node_depth + b * cap;
+        for (int64_t v = 0; v < cap; ++v) {
+            tok[v] = NONE;
+            par[v] = NONE;
+            fl[v] = 0;
+            dep[v] = 0;
+        }
+        int32_t n = 1;  // the root
+        for (int32_t c = 0; c < n_cands[b]; ++c) {
+            const int32_t* d = draft_ids + ((int64_t)b * max_cands + c) * draft_len;
+            const uint8_t* f = draft_flags + ((int64_t)b * max_cands + c) * draft_len;
+            int32_t u = 0;
+            for (int32_t i = 0; i < cand_len[(int64_t)b * max_cands + c]; ++i) {
+                if (d[i] == NONE) break;
+                int32_t child = NONE;
+                for (int32_t v = 1; v < n && child == NONE; ++v)
+                    if (par[v] == u && tok[v] == d[i]) child = v;
+                if (child == NONE) {
+                    child = n++;
+                    tok[child] = d[i];
+                    par[child] = u;
+                    dep[child] = dep[u] + 1;
+                }
+                fl[child] |= f[i];
+                u = child;
+            }
+        }
+        n_nodes[b] = n;
+    }
+    return 0;
+}
+
+// ---------------------------------------------------------------------------------
+// O-VT: verification of draft trees (Eq. 2, Sec. 3.3).  Row v of the logits is the target
+// distribution P_M(. | F(v)) that follows node v, F(v) being the path from the root to v;
+// so the token of node v is judged by the row of its parent, with the rules of O-V (modes
+// 0-2).  A node passes when it and all its ancestors are accepted (prefix rule, Sec. 2.1);
+// the result of a tree is its deepest passing node (ties: lowest node index; the root when
+// nothing passes): "the longest draft candidate that passes verification".  Emitted: the
+// tokens on the path to that node, followed by the target's own token of that node's row.
+// Trees are CSR ranges of nodes (tree_offsets[T+1]); node_parent holds indices inside the
+// tree (NONE for the root, which is node 0 of its tree); parents precede children.
+// Per row: entropy, pmax, argmax, threshold, sampled, bad.  Per node: p_token, accept (the
+// node's own bit; 0 for roots), near.  Per tree: best_node (inside the tree), n_accept
+// (its depth), n_emit, emit_ids [T x emit_stride] (NONE padded, clipped at emit_stride).
+// ---------------------------------------------------------------------------------
+int oracle_verify_tree(const void* logits, int dtype, const int32_t* node_token,
+                       const int32_t* node_parent, const uint8_t* node_flags,
+                       const int32_t* tree_offsets, int32_t T, int64_t V, int64_t row_stride,
+                       double alpha, double beta, double invT, int mode, uint64_t seed, uint32_t step,
+                       int threads, int emit_stride, double* p_token, double* entropy, double* pmax,
+                       int32_t* argmax, double* threshold, uint8_t* accept, int32_t* sampled,
+                       uint8_t* near, uint8_t* bad, int32_t* best_node, int32_t* n_accept,
+                       int32_t* n_emit, int32_t* emit_ids) {
+    if (T < 0 || V <= 0 || mode < 0 || mode > 2 || emit_stride < 1) return 1;
+    Rows X{logits, dtype, row_stride};
+    const int64_t R = tree_offsets[T];
+    std::vector<RowStats> st(R);
+    std::vector<int32_t> own(R, NONE);
+#pragma omp parallel for schedule(static) num_threads(threads > 0 ? threads : 1)
+    for (int64_t r = 0; r < R; ++r) {
+        st[r] = row_stats(X, r, V, invT);
+        int32_t smp = NONE;
+        if (!st[r].bad && mode == 2)
+            smp = sample_row(X, r, V, invT, seed, (uint32_t)r, step, DOM_VERIFY_GROUP, DOM_VERIFY_ELEM, 0);
+        own[r] = st[r].bad ? NONE : (mode == 2 ? smp : st[r].argmax);
+        if (entropy) entropy[r] = st[r].H;
+        if (pmax) pmax[r] = st[r].pmax;
+        if (argmax) argmax[r] = st[r].argmax;
+        if (threshold) threshold[r] = st[r].bad ? 0.0 : std::min(alpha * st[r].H + beta, st[r].pmax);
+        if (sampled) sampled[r] = smp;
+        if (bad) bad[r] = st[r].bad ? 1 : 0;
+    }
+    for (int32_t t = 0; t < T; ++t) {
+        const int64_t lo = tree_offsets[t], hi = tree_offsets[t + 1];
+        const int64_t n = hi - lo;
+        std::vector<uint8_t> ok(n, 0);
+        std::vector<int32_t> depth(n, 0);
+        int32_t best = 0;
+        for (int64_t v = 0; v < n; ++v) {
+            const int64_t g = lo + v;
+            const int32_t par = node_parent[g];
+            double pt = 0.0;
+            bool a = false, is_near = false;
+            if (v == 0 || par < 0 || par >= v) {   // the root (or a malformed node: never passes)
+                ok[v] = (v == 0);
+            } else {
+                const RowStats& ps = st[lo + par];
+                int32_t d = node_token[g];
+                if (d < 0 || d >= V) d = NONE;
+                const uint8_t f = node_flags ? node_flags[g] : 1;
+                if (!ps.bad && d != NONE) {
+                    pt = prob_of(X, lo + par, d, invT, ps);
+                    if (mode == 0 && (f & 1)) {
+                        const double lin = alpha * ps.H + beta;
+                        const bool at_max = (X.at(lo + par, d) * invT == ps.m);
+                        a = at_max || (pt >= lin);
+                        is_near = !at_max && std::fabs(pt - lin) <= 1e-6;
+                    } else {
+                        a = (d == own[lo + par]);
+                    }
+                }
+                depth[v] = depth[par] + 1;
+                ok[v] = a && ok[par];
+                if (ok[v] && depth[v] > depth[best]) best = (int32_t)v;
+            }
+            if (p_token) p_token[g] = pt;
+            if (accept) accept[g] = a ? 1 : 0;
+            if (near) near[g] = is_near ? 1 : 0;
+        }
+        if (n == 0) {
+            if (best_node) best_node[t] = NONE;
+            if (n_accept) n_accept[t] = 0;
+            if (n_emit) n_emit[t] = 0;
+            for (int i = 0; i < emit_stride; ++i) emit_ids[(int64_t)t * emit_stride + i] = NONE;
+            continue;
+        }
+        std::vector<int32_t> path;
+        for (int32_t v = best; v != 0; v = node_parent[lo + v]) path.push_back(node_token[lo + v]);
+        std::reverse(path.begin(), path.end());
+        if (own[lo + best] != NONE) path.push_back(own[lo + best]);
+        int32_t ne = 0;
+        for (int i = 0; i < emit_stride; ++i) {
+            int32_t tok = NONE;
+            if (i < (int)path.size()) {
+                tok = path[i];
+                ++ne;
+            }
+            emit_ids[(int64_t)t * emit_stride + i] = tok;
+        }
+        if (best_node) best_node[t] = best;
+        if (n_accept) n_accept[t] = depth[best];
+        if (n_emit) n_emit[t] = ne;
     }
     return 0;
 }
