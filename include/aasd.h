@@ -303,6 +303,53 @@ typedef struct aasd_step_args {
 int aasd_step(aasd_ctx* ctx, const aasd_step_args* args, void* workspace,
               size_t workspace_bytes);
 
+/* ---- draft trees (Eq. 2, Sec. 3.2) and their verification (Sec. 3.3) ---------------- */
+
+/* Merges the candidates of every sequence (as aasd_draft writes them) into one draft tree
+ * per sequence.  Tree b owns node slots [b*cap, (b+1)*cap), cap = 1 + max_cands*draft_len;
+ * node 0 is the root (no token), nodes are numbered in creation order while the candidates
+ * are walked in order (a parent precedes its children; children are matched by token, the
+ * lowest node index first); a node reached by several candidates carries the OR of their
+ * token flags.  node_parent holds indices inside the tree, NONE for the root and for unused
+ * slots; node_token is NONE there too.  All outputs are required.
+ * AASD_ERR_UNSUPPORTED when a tree's slots do not fit the shared memory of one CTA. */
+int aasd_tree_build(aasd_ctx* ctx, const int32_t* draft_ids, const uint8_t* draft_flags,
+                    const int32_t* cand_len, const int32_t* n_cands, int32_t n_seqs,
+                    int32_t max_cands, int32_t draft_len, int32_t* node_token, int32_t* node_parent,
+                    uint8_t* node_flags, int32_t* node_depth, int32_t* n_nodes);
+
+typedef struct aasd_tree_out {
+    float* p_token;       /* [n_rows] probability of the node's token under its parent's row (0 for roots) */
+    uint8_t* accept;      /* [n_rows] the node's own accept bit (0 for roots) */
+    float* entropy;       /* [n_rows] per row, as in aasd_verify_out */
+    float* pmax;          /* [n_rows] */
+    int32_t* argmax;      /* [n_rows] */
+    float* threshold;     /* [n_rows] */
+    int32_t* sampled;     /* [n_rows] the row's keyed sample (STRICT_SAMPLED), else NONE */
+    int32_t* best_node;   /* [n_trees] deepest node whose whole path passes (index inside the tree;
+                             the root when nothing passes; NONE for a tree without nodes) */
+    int32_t* n_accept;    /* [n_trees] its depth = accepted draft tokens */
+    int32_t* n_emit;      /* [n_trees] tokens in emit_ids */
+    int32_t* emit_ids;    /* [n_trees x emit_stride] the tokens on the path to best_node followed by
+                             the target's own token of best_node's row; NONE padded, clipped */
+} aasd_tree_out;
+
+/* Verifies draft trees.  Trees are CSR ranges of nodes (tree_offsets[n_trees+1], the last
+ * offset equals n_rows); row v of target_logits is the distribution that follows node v
+ * given the path from the root, so the token of node v is judged with its parent's row by
+ * the rules of aasd_verify (modes CONDITIONAL, STRICT_GREEDY, STRICT_SAMPLED; node_flags may
+ * be NULL: every node conditional-eligible).  A node passes when it and all its ancestors
+ * are accepted; per tree the deepest passing node wins (ties: lowest index), which is the
+ * longest candidate that passes.  Because every node has a row of its own, the token after
+ * the accepted path is always available.  params->rows_per_cand and top_k are ignored.
+ * A node whose parent index is not smaller than its own raises AASD_STATUS_BAD_OFFSETS and
+ * never passes.  best_node, n_accept, n_emit and emit_ids are required. */
+int aasd_verify_tree(aasd_ctx* ctx, const void* target_logits, const int32_t* node_token,
+                     const int32_t* node_parent, const uint8_t* node_flags,
+                     const int32_t* tree_offsets, int32_t n_trees, int64_t n_rows,
+                     const aasd_verify_params* params, int32_t emit_stride, void* workspace,
+                     size_t workspace_bytes, const aasd_tree_out* out);
+
 /* ---- verification for callers that cannot allocate ------------------------------- */
 
 #define AASD_STATIC_MAX_ROWS 8192   /* most logits rows per aasd_verify_static call */

@@ -27,6 +27,7 @@ EXPORTS = [
     "aasd_get_counters", "aasd_reset_counters", "aasd_launch_count", "aasd_workspace_bytes",
     "aasd_workspace_init", "aasd_workspace_release", "aasd_align_sample", "aasd_draft",
     "aasd_verify", "aasd_select", "aasd_append", "aasd_step", "aasd_verify_static",
+    "aasd_tree_build", "aasd_verify_tree",
 ]
 STATIC_MAX_ROWS = STATIC_MAX_CANDS = 8192
 
@@ -70,6 +71,11 @@ class VerifyParams(C.Structure):
 class VerifyOut(C.Structure):
     _fields_ = [(n, _vp) for n in ("p_draft", "entropy", "pmax", "argmax", "threshold",
                                    "accept", "sampled", "accept_len", "next_token", "n_greater")]
+
+
+class TreeOut(C.Structure):
+    _fields_ = [(n, _vp) for n in ("p_token", "accept", "entropy", "pmax", "argmax", "threshold",
+                                   "sampled", "best_node", "n_accept", "n_emit", "emit_ids")]
 
 
 class StepArgs(C.Structure):
@@ -121,6 +127,11 @@ def load_library(path: str | None = None):
                                 C.c_int32, _vp, _vp, _vp]
     lib.aasd_append.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, C.c_int32, C.c_int32]
     lib.aasd_step.argtypes = [_vp, C.POINTER(StepArgs), _vp, C.c_size_t]
+    lib.aasd_tree_build.argtypes = [_vp, _vp, _vp, _vp, _vp, C.c_int32, C.c_int32, C.c_int32, _vp, _vp,
+                                    _vp, _vp, _vp]
+    lib.aasd_verify_tree.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, C.c_int32, C.c_int64,
+                                     C.POINTER(VerifyParams), C.c_int32, _vp, C.c_size_t,
+                                     C.POINTER(TreeOut)]
     lib.aasd_verify_static.argtypes = [C.c_int, _vp, _vp, _vp, _vp, _vp, C.c_int32, C.c_int64,
                                        C.POINTER(VerifyParams), C.POINTER(VerifyOut), _vp]
     if path == _build.LIB:
@@ -358,6 +369,56 @@ class Context:
         fl = None if draft_flags is None else draft_flags.reshape(-1)
         _check(self.lib.aasd_verify(self._h, _p(x), _p(d), _p(fl), _p(offs), Cn, R, C.byref(prm),
                                     _p(ws), ws.numel(), C.byref(out)), "aasd_verify")
+        return o
+
+    def tree_build(self, draft_ids, draft_flags, cand_len, n_cands):
+        """aasd_tree_build: candidates [B x max_cands x draft_len] -> one draft tree per sequence
+        in 1 + max_cands*draft_len node slots (Eq. 2)."""
+        B, Cm, Ld = draft_ids.shape
+        cap = 1 + Cm * Ld
+        dev = draft_ids.device
+        o = dict(node_token=torch.empty((B, cap), dtype=torch.int32, device=dev),
+                 node_parent=torch.empty((B, cap), dtype=torch.int32, device=dev),
+                 node_flags=torch.empty((B, cap), dtype=torch.uint8, device=dev),
+                 node_depth=torch.empty((B, cap), dtype=torch.int32, device=dev),
+                 n_nodes=torch.empty(B, dtype=torch.int32, device=dev))
+        _check(self.lib.aasd_tree_build(self._h, _p(draft_ids), _p(draft_flags), _p(cand_len), _p(n_cands),
+                                        B, Cm, Ld, _p(o["node_token"]), _p(o["node_parent"]),
+                                        _p(o["node_flags"]), _p(o["node_depth"]), _p(o["n_nodes"])),
+               "aasd_tree_build")
+        return o
+
+    def verify_tree(self, target_logits, node_token, node_parent, tree_offsets, emit_stride,
+                    node_flags=None, alpha=0.1, beta=0.1, mode=VERIFY_CONDITIONAL, seed=0, step=0,
+                    inv_temperature=1.0, outputs=None):
+        """aasd_verify_tree: trees are CSR ranges of nodes, row v follows node v."""
+        x = target_logits
+        assert x.is_cuda and x.dim() == 2 and x.stride(1) == 1
+        R, V = x.shape
+        dev = x.device
+        offs = _dev_i32(tree_offsets, dev)
+        T = offs.numel() - 1
+        o = outputs or dict(
+            p_token=torch.empty(R, dtype=torch.float32, device=dev),
+            accept=torch.empty(R, dtype=torch.uint8, device=dev),
+            entropy=torch.empty(R, dtype=torch.float32, device=dev),
+            pmax=torch.empty(R, dtype=torch.float32, device=dev),
+            argmax=torch.empty(R, dtype=torch.int32, device=dev),
+            threshold=torch.empty(R, dtype=torch.float32, device=dev),
+            sampled=torch.empty(R, dtype=torch.int32, device=dev),
+            best_node=torch.empty(T, dtype=torch.int32, device=dev),
+            n_accept=torch.empty(T, dtype=torch.int32, device=dev),
+            n_emit=torch.empty(T, dtype=torch.int32, device=dev),
+            emit_ids=torch.empty((T, emit_stride), dtype=torch.int32, device=dev))
+        prm = VerifyParams(V, _dtype_code(x), x.stride(0), float(alpha), float(beta),
+                           float(inv_temperature), int(mode), 0, int(step), int(seed), 0)
+        out = TreeOut(*[_p(o.get(n)) for n, _ in TreeOut._fields_])
+        ws = self.workspace(R, T)
+        fl = None if node_flags is None else node_flags.reshape(-1)
+        _check(self.lib.aasd_verify_tree(self._h, _p(x), _p(node_token.reshape(-1)),
+                                         _p(node_parent.reshape(-1)), _p(fl), _p(offs), T, R, C.byref(prm),
+                                         int(emit_stride), _p(ws), ws.numel(), C.byref(out)),
+               "aasd_verify_tree")
         return o
 
     def select(self, accept_len, next_token, draft_ids, emit_stride, cand_offsets=None,

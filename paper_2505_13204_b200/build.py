@@ -10,7 +10,7 @@ CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libaasd.so")
 SOURCES = ["aasd.cu"]
 DEPENDS = ["aasd.cu", "aasd_device.cuh", "aasd_rows.cuh", "aasd_sampler.cuh", "aasd_stream.cuh",
-           "aasd_tokens.cuh",
+           "aasd_tokens.cuh", "aasd_tree.cuh",
            os.path.join("..", "..", "include", "aasd.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-shared", "-Xcompiler", "-fPIC"]

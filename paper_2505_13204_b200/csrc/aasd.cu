@@ -14,6 +14,7 @@
 #include "aasd_rows.cuh"
 #include "aasd_stream.cuh"
 #include "aasd_tokens.cuh"
+#include "aasd_tree.cuh"
 
 using namespace aasd;
 
@@ -22,12 +23,15 @@ namespace {
 struct WorkspaceLayout {
     size_t bytes;
     int64_t max_rows, max_cands;
-    size_t off_partials, off_row_tickets, off_cand_tickets, off_seq_tickets, off_sched, off_row_accept, off_row_own, off_next, off_race;
+    size_t off_partials, off_row_tickets, off_cand_tickets, off_seq_tickets, off_sched, off_row_accept, off_row_own, off_next, off_race,
+        off_tree_stats;
 };
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-WorkspaceLayout make_layout(int64_t max_rows, int64_t max_cands) {
+// with_tree: room for the per-row statistics of tree verification (the fixed block of
+// aasd_verify_static does without).
+WorkspaceLayout make_layout(int64_t max_rows, int64_t max_cands, bool with_tree = true) {
     WorkspaceLayout L{};
     L.max_rows = max_rows;
     L.max_cands = max_cands;
@@ -50,6 +54,8 @@ WorkspaceLayout make_layout(int64_t max_rows, int64_t max_cands) {
     o = align_up(o + 4 * (size_t)max_rows, 256);
     L.off_race = o;
     o = align_up(o + sizeof(RaceSummary) * (size_t)kRaceSlots * kMaxK, 256);
+    L.off_tree_stats = o;
+    if (with_tree) o = align_up(o + sizeof(TreeRowStat) * (size_t)max_rows, 256);
     L.bytes = o;
     return L;
 }
@@ -577,6 +583,104 @@ int aasd_step(aasd_ctx* ctx, const aasd_step_args* s, void* workspace, size_t wo
 
 }  // extern "C"
 
+// ---- draft trees ----------------------------------------------------------------------------
+
+namespace {
+
+template <int DT, int ND>
+int launch_tree_stream(aasd_ctx* ctx, const StreamJob& sj, const TreeArgs& a, unsigned int grid) {
+    auto kernel = stream_kernel<DT, 1, ND, false, TreeEpilogue<DT>>;
+    if (enable_stream_smem(kernel) != AASD_OK) return AASD_ERR_CUDA;
+    launch(kernel, grid, kStreamThreads, kStreamSmemBytes, ctx->stream, sj, a);
+    return AASD_OK;
+}
+
+template <int DT>
+int dispatch_tree_stream(aasd_ctx* ctx, const StreamJob& sj, const TreeArgs& a, unsigned int grid) {
+    return a.mode == AASD_VERIFY_STRICT_SAMPLED ? launch_tree_stream<DT, 1>(ctx, sj, a, grid)
+                                                : launch_tree_stream<DT, 0>(ctx, sj, a, grid);
+}
+
+}  // namespace
+
+extern "C" int aasd_tree_build(aasd_ctx* ctx, const int32_t* draft_ids, const uint8_t* draft_flags,
+                               const int32_t* cand_len, const int32_t* n_cands, int32_t n_seqs, int32_t max_cands,
+                               int32_t draft_len, int32_t* node_token, int32_t* node_parent, uint8_t* node_flags,
+                               int32_t* node_depth, int32_t* n_nodes) {
+    if (ctx == nullptr) return AASD_ERR_INVALID_ARG;
+    if (n_seqs < 0 || max_cands < 1 || draft_len < 1) return AASD_ERR_BAD_SHAPE;
+    if (n_seqs == 0) return AASD_OK;
+    if (!draft_ids || !draft_flags || !cand_len || !n_cands || !node_token || !node_parent || !node_flags ||
+        !node_depth || !n_nodes)
+        return AASD_ERR_INVALID_ARG;
+    const int64_t cap = 1 + (int64_t)max_cands * draft_len;
+    const size_t smem = (size_t)cap * 2 * sizeof(int);
+    if (smem > 48 * 1024) return AASD_ERR_UNSUPPORTED;
+    TreeBuildArgs a{draft_ids, draft_flags, cand_len, n_cands, max_cands, draft_len, (int)cap,
+                    node_token, node_parent, node_flags, node_depth, n_nodes};
+    AASD_CUDA(cudaSetDevice(ctx->device));
+    launch(tree_build_kernel, (unsigned int)n_seqs, 32u, smem, ctx->stream, a);
+    return after_launch(ctx, 1);
+}
+
+extern "C" int aasd_verify_tree(aasd_ctx* ctx, const void* target_logits, const int32_t* node_token,
+                                const int32_t* node_parent, const uint8_t* node_flags, const int32_t* tree_offsets,
+                                int32_t n_trees, int64_t n_rows, const aasd_verify_params* p, int32_t emit_stride,
+                                void* workspace, size_t workspace_bytes, const aasd_tree_out* out) {
+    if (ctx == nullptr || p == nullptr || out == nullptr) return AASD_ERR_INVALID_ARG;
+    if (n_trees < 0 || n_rows < 0 || emit_stride < 1) return AASD_ERR_BAD_SHAPE;
+    if (p->mode < AASD_VERIFY_CONDITIONAL || p->mode > AASD_VERIFY_STRICT_SAMPLED) return AASD_ERR_UNSUPPORTED;
+    if (!(p->alpha >= 0.f) || !(p->beta >= 0.f)) return AASD_ERR_INVALID_ARG;
+    if (n_trees > 0 && tree_offsets == nullptr) return AASD_ERR_INVALID_ARG;
+    if (n_rows > 0 && (node_token == nullptr || node_parent == nullptr || n_trees == 0)) return AASD_ERR_INVALID_ARG;
+    if (!out->best_node || !out->n_accept || !out->n_emit || !out->emit_ids) return AASD_ERR_INVALID_ARG;
+    int err = AASD_OK;
+    const WorkspaceLayout* L = find_workspace(ctx, workspace, workspace_bytes, n_rows, n_trees, &err);
+    if (L == nullptr) return err;
+    char* ws = static_cast<char*>(workspace);
+    TreeArgs a{};
+    err = plan_rows(ctx, a.job, target_logits, p->dtype, p->vocab, p->row_stride, n_rows, p->inv_temperature, ws, *L);
+    if (err != AASD_OK) return err;
+    if (n_rows * (int64_t)a.job.chunks > 0x7FFFFFFFLL) return AASD_ERR_BAD_SHAPE;
+    a.node_token = node_token;
+    a.node_parent = node_parent;
+    a.node_flags = node_flags;
+    a.tree_offsets = tree_offsets;
+    a.n_trees = n_trees;
+    a.alpha = p->alpha;
+    a.beta = p->beta;
+    a.mode = p->mode;
+    a.emit_stride = emit_stride;
+    a.smp = make_sample_job(p->seed, p->step, false, p->inv_temperature);
+    a.hint = reinterpret_cast<int32_t*>(ws + L->off_next);
+    a.stats = reinterpret_cast<TreeRowStat*>(ws + L->off_tree_stats);
+    a.tree_tickets = reinterpret_cast<unsigned int*>(ws + L->off_cand_tickets);
+    a.node_ok = reinterpret_cast<uint8_t*>(ws + L->off_row_accept);
+    a.out = *out;
+    AASD_CUDA(cudaSetDevice(ctx->device));
+    if (n_rows == 0) {
+        if (n_trees == 0) return AASD_OK;
+        launch(tree_empty_kernel, (unsigned int)((n_trees + 255) / 256), 256u, 0, ctx->stream, a);
+        return after_launch(ctx, 1);
+    }
+    // rows without children keep the hint NONE (all bits set)
+    AASD_CUDA(cudaMemsetAsync(a.hint, 0xFF, 4 * (size_t)n_rows, ctx->stream));
+    launch(tree_hint_kernel, (unsigned int)((n_rows + 255) / 256), 256u, 0, ctx->stream, a);
+    if (a.job.vector_ok && a.job.nvec > 0) {
+        StreamJob sj{};
+        unsigned int grid = 0;
+        plan_stream(ctx, sj, a.job, a.hint, ws, *L, p->mode == AASD_VERIFY_STRICT_SAMPLED ? &a.smp : nullptr, &grid);
+        const int rc = p->dtype == AASD_F32 ? dispatch_tree_stream<AASD_F32>(ctx, sj, a, grid)
+                                            : dispatch_tree_stream<AASD_BF16>(ctx, sj, a, grid);
+        if (rc != AASD_OK) return rc;
+        return after_launch(ctx, 2);
+    }
+    const unsigned int grid = (unsigned int)(n_rows * a.job.chunks);
+    if (p->dtype == AASD_F32) launch(tree_kernel<AASD_F32>, grid, (unsigned int)kThreads, 0, ctx->stream, a);
+    else launch(tree_kernel<AASD_BF16>, grid, (unsigned int)kThreads, 0, ctx->stream, a);
+    return after_launch(ctx, 2);
+}
+
 // ---- verification without any allocation ---------------------------------------------------
 //
 // Scratch of aasd_verify_static: one block per GPU that loads the library, held until the
@@ -629,7 +733,7 @@ extern "C" int aasd_verify_static(int device, void* stream, const void* target_l
         if (p->rows_per_cand < 1 || (int64_t)n_cands * p->rows_per_cand != n_rows) return AASD_ERR_BAD_SHAPE;
     }
     if (n_rows > 0 && (draft_ids == nullptr || n_cands == 0)) return AASD_ERR_INVALID_ARG;
-    const WorkspaceLayout L = make_layout(kStaticMaxRows, kStaticMaxCands);
+    const WorkspaceLayout L = make_layout(kStaticMaxRows, kStaticMaxCands, false);
     if (L.bytes != kStaticWorkspaceBytes) return AASD_ERR_WORKSPACE_TOO_SMALL;   // layouts out of step
 
     std::lock_guard<std::mutex> guard(g_static_mutex);
