@@ -245,6 +245,89 @@ struct TileAccumulator {
     }
 };
 
+// Kernels that need the best token only (K = 1, no sampling) do not track where a thread met
+// its maximum: a thread keeps the running maximum of its logits (one packed max per word),
+// the warp reports the maximum and which lanes hold it, and the finisher, which has time to
+// spare, finds the first vector that attains it among those lanes' vectors.
+template <int DT> struct RunMax;
+template <> struct RunMax<AASD_BF16> {
+    unsigned int m2;   // bf16x2
+    __device__ __forceinline__ void init() { m2 = 0xFF80FF80u; }
+    __device__ __forceinline__ void update(const uint4& q) {
+        unsigned int a, b;
+        asm("max.bf16x2 %0, %1, %2;" : "=r"(a) : "r"(q.x), "r"(q.y));
+        asm("max.bf16x2 %0, %1, %2;" : "=r"(b) : "r"(q.z), "r"(q.w));
+        asm("max.bf16x2 %0, %1, %2;" : "=r"(a) : "r"(a), "r"(b));
+        asm("max.bf16x2 %0, %1, %2;" : "=r"(m2) : "r"(m2), "r"(a));
+    }
+    __device__ __forceinline__ float value() const {
+        return fmaxf(__uint_as_float(m2 << 16), __uint_as_float(m2 & 0xFFFF0000u));
+    }
+};
+template <> struct RunMax<AASD_F32> {
+    float m;
+    __device__ __forceinline__ void init() { m = -CUDART_INF_F; }
+    __device__ __forceinline__ void update(const uint4& q) {
+        m = fmaxf(fmaxf(m, __uint_as_float(q.x)),
+                  fmaxf(fmaxf(__uint_as_float(q.y), __uint_as_float(q.z)), __uint_as_float(q.w)));
+    }
+    __device__ __forceinline__ float value() const { return m; }
+};
+
+// The sums of one vector without any maximum tracking.
+template <int DT, int K>
+__device__ __forceinline__ void add_sums(TileAccumulator<DT, K>& acc, const uint4& raw, float c1, float neg_refc) {
+    constexpr int kVec = Elt<DT>::kVec;
+    float x[kVec];
+    Elt<DT>::unpack(Clamp<DT>::apply(raw), x);
+    const float2 cc = make_float2(c1, c1);
+    const float2 rr = make_float2(neg_refc, neg_refc);
+#pragma unroll
+    for (int i = 0; i < kVec / 2; ++i) {
+        float2 t = __ffma2_rn(make_float2(x[2 * i], x[2 * i + 1]), cc, rr);
+        float2 e = make_float2(ex2_approx(t.x), ex2_approx(t.y));
+        acc.S2[i] = __fadd2_rn(acc.S2[i], e);
+        acc.A2[i] = __ffma2_rn(e, t, acc.A2[i]);
+    }
+}
+
+// First vector (lowest index) with maximum m among the vectors thread `tid` of the consumers
+// met in tiles [tb, te): vectors t * 1024 + k * 256 + tid.  By a whole warp; -1 if none.
+template <int DT>
+__device__ int first_vector_of_thread(const char* rowp, int nvec, int tb, int te, int tid, float m) {
+    constexpr int kTileVecs = kTileBytes / 16;
+    constexpr int kPer = kTileVecs / kConsumers;
+    const int lane = threadIdx.x & 31;
+    const int total = (te - tb) * kPer;
+    for (int base = 0; base < total; base += 32) {
+        const int j = base + lane;
+        const int v = (tb + j / kPer) * kTileVecs + (j % kPer) * kConsumers + tid;
+        bool hit = false;
+        if (j < total && v < nvec) hit = Clamp<DT>::vector_max(__ldg(reinterpret_cast<const uint4*>(rowp) + v)) == m;
+        const unsigned int bal = __ballot_sync(0xFFFFFFFFu, hit);
+        if (bal) {
+            const int jj = base + __ffs(bal) - 1;
+            return (tb + jj / kPer) * kTileVecs + (jj % kPer) * kConsumers + tid;
+        }
+    }
+    return -1;
+}
+// The same over every vector of tiles [tb, te) (many lanes tie for the maximum).
+template <int DT>
+__device__ int first_vector_of_range(const char* rowp, int nvec, int tb, int te, float m) {
+    constexpr int kTileVecs = kTileBytes / 16;
+    const int lane = threadIdx.x & 31;
+    const int end = min(te * kTileVecs, nvec);
+    for (int base = tb * kTileVecs; base < end; base += 32) {
+        const int v = base + lane;
+        bool hit = false;
+        if (v < end) hit = Clamp<DT>::vector_max(__ldg(reinterpret_cast<const uint4*>(rowp) + v)) == m;
+        const unsigned int bal = __ballot_sync(0xFFFFFFFFu, hit);
+        if (bal) return base + __ffs(bal) - 1;
+    }
+    return -1;
+}
+
 // Top-k verification (Sec. 3.3): counts, per thread, the tokens that are ahead of the row's
 // draft token d in the order (logit descending, id ascending).  A token with a lower id is
 // ahead when its logit is >= x_d, one with a higher id when it is > x_d; ">= x_d" is taken
@@ -430,6 +513,9 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
             race.init();
             AheadCounter<DT> ahead;
             ahead.count = 0;
+            constexpr bool kLazyMax = (K == 1 && ND == 0);   // maximum by value, place found later
+            RunMax<DT> runmax;
+            runmax.init();
             unsigned int row_ctr = 0;
             float neg_refc = 0.f;
             bool alive = true, last = false;
@@ -488,7 +574,14 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
 #pragma unroll
                     for (int k = 0; k < kTileVecs / kConsumers; ++k) q[k] = lds16(base + (size_t)(k * kConsumers + tid) * 16);
 #pragma unroll
-                    for (int k = 0; k < kTileVecs / kConsumers; ++k) acc.add(q[k], v0 + k * kConsumers + tid, c1, neg_refc);
+                    for (int k = 0; k < kTileVecs / kConsumers; ++k) {
+                        if (kLazyMax) {
+                            add_sums<DT, K>(acc, q[k], c1, neg_refc);
+                            runmax.update(q[k]);
+                        } else {
+                            acc.add(q[k], v0 + k * kConsumers + tid, c1, neg_refc);
+                        }
+                    }
                     if (TK) {
 #pragma unroll
                         for (int k = 0; k < kTileVecs / kConsumers; ++k) ahead.add(q[k], v0 + k * kConsumers + tid);
@@ -497,7 +590,12 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
                 } else {
                     for (int v = tid; v < nv; v += kConsumers) {
                         const uint4 q = lds16(base + (size_t)v * 16);
-                        acc.add(q, v0 + v, c1, neg_refc);
+                        if (kLazyMax) {
+                            add_sums<DT, K>(acc, q, c1, neg_refc);
+                            runmax.update(q);
+                        } else {
+                            acc.add(q, v0 + v, c1, neg_refc);
+                        }
                         if (TK) ahead.add(q, v0 + v);
                     }
                     if (TK) ahead.end_tile();
@@ -519,14 +617,22 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
 #pragma unroll
             for (int j = 0; j < K; ++j) vk[j] = acc.best_vec[j] >= 0 ? make_vec_key(acc.best[j], acc.best_vec[j]) : 0ull;
             u64 wk[K];
+            if (kLazyMax) {
+                // (warp maximum, lanes that hold it); nothing when every logit was -inf or NaN
+                const float mt = runmax.value();
+                const float mw = warp_max_f32(mt);
+                const unsigned int holders = __ballot_sync(0xFFFFFFFFu, mt == mw);
+                wk[0] = mw > -CUDART_INF_F ? (((u64)ordered_bits(mw) << 32) | (u64)holders) : 0ull;
+            } else {
 #pragma unroll
-            for (int r = 0; r < K; ++r) {
-                const u64 m = warp_max_u64(vk[0]);
-                wk[r] = m;
-                if (m != 0 && vk[0] == m) {
+                for (int r = 0; r < K; ++r) {
+                    const u64 m = warp_max_u64(vk[0]);
+                    wk[r] = m;
+                    if (m != 0 && vk[0] == m) {
 #pragma unroll
-                    for (int j = 0; j + 1 < K; ++j) vk[j] = vk[j + 1];
-                    vk[K - 1] = 0;
+                        for (int j = 0; j + 1 < K; ++j) vk[j] = vk[j + 1];
+                        vk[K - 1] = 0;
+                    }
                 }
             }
             const int p = seq % kSlots;
@@ -705,14 +811,45 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
         A = warp_sum_f64(A);
         if (TK) n_ahead = warp_sum_i64(n_ahead);
         u64 mk[K];   // merged vector keys, identical in every lane
+        if (K == 1 && ND == 0) {
+            // the consumers reported (maximum, lanes holding it) per warp: find the first vector
+            // of the item that attains the maximum
+            const unsigned int top = (unsigned int)(vk[0] >> 32);
+            const unsigned int best = __reduce_max_sync(0xFFFFFFFFu, top);
+            mk[0] = 0;
+            if (best != 0) {
+                const float m = unordered_bits(best);
+                const unsigned int mine = (lane < kConsumerWarps && top == best) ? (unsigned int)vk[0] : 0u;
+                int n_holders = __reduce_add_sync(0xFFFFFFFFu, __popc(mine));
+                int tb, te;
+                tile_range(job, info.row, info.chunk, tb, te);
+                int vfirst = 0x7FFFFFFF;
+                if (n_holders <= 8) {
+                    for (int w = 0; w < kConsumerWarps; ++w) {
+                        unsigned int lanes = __shfl_sync(0xFFFFFFFFu, mine, w);
+                        while (lanes) {
+                            const int l = __ffs(lanes) - 1;
+                            lanes &= lanes - 1;
+                            const int v = first_vector_of_thread<DT>(rowp, rj.nvec, tb, te, w * 32 + l, m);
+                            if (v >= 0 && v < vfirst) vfirst = v;
+                        }
+                    }
+                } else {
+                    const int v = first_vector_of_range<DT>(rowp, rj.nvec, tb, te, m);
+                    if (v >= 0) vfirst = v;
+                }
+                if (vfirst != 0x7FFFFFFF) mk[0] = make_vec_key(m, vfirst);
+            }
+        } else {
 #pragma unroll
-        for (int r = 0; r < K; ++r) {
-            const u64 m = warp_max_u64(vk[0]);
-            mk[r] = m;
-            if (m != 0 && vk[0] == m) {
+            for (int r = 0; r < K; ++r) {
+                const u64 m = warp_max_u64(vk[0]);
+                mk[r] = m;
+                if (m != 0 && vk[0] == m) {
 #pragma unroll
-                for (int j = 0; j + 1 < K; ++j) vk[j] = vk[j + 1];
-                vk[K - 1] = 0;
+                    for (int j = 0; j + 1 < K; ++j) vk[j] = vk[j + 1];
+                    vk[K - 1] = 0;
+                }
             }
         }
         if (chunks > 1) {
