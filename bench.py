@@ -46,8 +46,7 @@ N_BUF = 8
 # captures summarised under profiles/: (workload, kernel) -> (rows captured, bytes).  Traffic
 # is proportional to rows (each row is read once), so it is scaled to the launch's rows.
 # An entry is set to None whenever the kernel has changed since its capture.
-NCU_TRAFFIC = {("cfg5-serving-256", "verify"): (2048, 623.016448e6 + 3.948032e6),
-               ("cfg5-serving-256", "align"): (2048, 623.323904e6 + 6.476032e6)}
+NCU_TRAFFIC = {("cfg5-serving-256", "verify"): None, ("cfg5-serving-256", "align"): None}
 
 
 def ncu_traffic(workload: str, kernel: str, rows: int):
@@ -198,10 +197,11 @@ class Bench:
         j = s % N_BUF
         if j == 0 and s > 0:
             self.restore()
+        ja = j % len(self.pre_bufs)     # small configurations have fewer prefill blocks than steps
         if events is not None:
             events[0].record()
-        self.ctx.align_sample(self.pre_bufs[j], self.pre_ids[j], self.pre_offs[j], k_extra=K_EXTRA,
-                              outputs=self.pre_out[j])
+        self.ctx.align_sample(self.pre_bufs[ja], self.pre_ids[ja], self.pre_offs[ja], k_extra=K_EXTRA,
+                              outputs=self.pre_out[ja])
         if events is not None:
             events[1].record()
         self.state.run_draft()
@@ -300,11 +300,60 @@ def run_ours(args, rank, world, local_rank):
         "mean_tokens_per_seq_step": bench.accepted_per_cycle / N_BUF / w.batch,
         "counters": bench.ctx.counters(),
     }
+    if world == 1 and not args.no_latency:
+        del bench
+        torch.cuda.empty_cache()
+        line["decode_step_latency_us"] = {synth.workload(i).name: decode_step_latency(i, dev) for i in range(4)}
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = cpu_baseline(w, seconds=args.cpu_seconds)
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+
+
+def decode_step_latency(index: int, dev, n_buf: int = 4, reps: int = 50):
+    """One decoding step (aasd_draft + aasd_step) of a small configuration, in microseconds.
+
+    The single-sequence configurations verify 8-12 rows per step: that is latency, not
+    bandwidth, so the figure is microseconds per step, measured by replaying a CUDA graph of
+    n_buf consecutive steps (a launch from Python costs more than such a step runs).  The
+    logits of step j are drawn for the candidates the drafter emits at state j."""
+    from paper_2505_13204_b200 import binding
+    w = synth.workload(index)
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        ctx = binding.Context(stream=side)
+        prompts = [synth.prompt_ids(w, b) for b in range(w.batch)]
+        st = binding.DecodeState(ctx, prompts, n_buf * (w.draft_len + 1) + 8, w.ngram, w.draft_len, w.max_cands,
+                                 w.vocab, w.torch_dtype, alpha=ALPHA, beta=BETA)
+        hist0, len0 = st.hist_ids.clone(), st.hist_len.clone()
+        bufs = []
+        for j in range(n_buf):
+            d = st.run_draft()["draft_ids"].reshape(-1).to(torch.int64)
+            x = synth.logits(st.rows, w.vocab, w.torch_dtype, w.recipe, d, w.seed + 977 * (j + 1), device=dev,
+                             chunk_rows=1024)
+            bufs.append(x)
+            st.step(x, j, reuse_draft=True)
+        side.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            st.hist_ids.copy_(hist0)
+            st.hist_len.copy_(len0)
+            for j in range(n_buf):
+                st.run_draft()
+                st.step(bufs[j], j, reuse_draft=True)
+        for _ in range(3):
+            graph.replay()
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record()
+        for _ in range(reps):
+            graph.replay()
+        t1.record()
+    torch.cuda.synchronize()
+    us = t0.elapsed_time(t1) * 1e3 / (reps * n_buf)
+    ctx.close()
+    return {"us_per_step": us, "verify_rows": st.rows, "sequences": w.batch,
+            "note": "draft + verify/select/append, graph replay; includes 1/%d of a state restore" % n_buf}
 
 
 def run_e2e(bench: Bench, dev, steps: int):
@@ -516,6 +565,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=4, help="0-based index of the configuration")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-latency", action="store_true", help="skip the decode-step latencies of configs 1-4")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))

@@ -107,6 +107,7 @@ struct StreamShared {
     ItemInfo ring[kRing];
     WarpPartial wp[kSlots][kConsumerWarps];
     RaceSummary race[kSlots][kConsumerWarps][kMaxK];   // sampling kernels only
+    unsigned short max_tile[kSlots][kConsumerWarps][32];   // tile (within the item) where a lane met its maximum
     int abort_flag;
 };
 constexpr size_t kStreamSmemBytes = (size_t)kStages * kTileBytes + sizeof(StreamShared) + 128;
@@ -245,10 +246,11 @@ struct TileAccumulator {
     }
 };
 
-// Kernels that need the best token only (K = 1, no sampling) do not track where a thread met
-// its maximum: a thread keeps the running maximum of its logits (one packed max per word),
-// the warp reports the maximum and which lanes hold it, and the finisher, which has time to
-// spare, finds the first vector that attains it among those lanes' vectors.
+// Kernels that need the best token only (K = 1, no sampling) do not track the vector in
+// which a thread met its maximum: a thread keeps the maximum of each tile's logits (one
+// packed max per word) and, once per tile, the running maximum with the tile that first
+// reached it; the warp reports the maximum and which lanes hold it, and the finisher looks
+// the first such vector up among the four vectors that lane read in that tile.
 template <int DT> struct RunMax;
 template <> struct RunMax<AASD_BF16> {
     unsigned int m2;   // bf16x2
@@ -292,25 +294,17 @@ __device__ __forceinline__ void add_sums(TileAccumulator<DT, K>& acc, const uint
 }
 
 // First vector (lowest index) with maximum m among the vectors thread `tid` of the consumers
-// met in tiles [tb, te): vectors t * 1024 + k * 256 + tid.  By a whole warp; -1 if none.
+// read in tile t: vectors t * 1024 + k * 256 + tid.  By a whole warp; -1 if none.
 template <int DT>
-__device__ int first_vector_of_thread(const char* rowp, int nvec, int tb, int te, int tid, float m) {
+__device__ int first_vector_in_tile(const char* rowp, int nvec, int t, int tid, float m) {
     constexpr int kTileVecs = kTileBytes / 16;
     constexpr int kPer = kTileVecs / kConsumers;
     const int lane = threadIdx.x & 31;
-    const int total = (te - tb) * kPer;
-    for (int base = 0; base < total; base += 32) {
-        const int j = base + lane;
-        const int v = (tb + j / kPer) * kTileVecs + (j % kPer) * kConsumers + tid;
-        bool hit = false;
-        if (j < total && v < nvec) hit = Clamp<DT>::vector_max(__ldg(reinterpret_cast<const uint4*>(rowp) + v)) == m;
-        const unsigned int bal = __ballot_sync(0xFFFFFFFFu, hit);
-        if (bal) {
-            const int jj = base + __ffs(bal) - 1;
-            return (tb + jj / kPer) * kTileVecs + (jj % kPer) * kConsumers + tid;
-        }
-    }
-    return -1;
+    const int v = t * kTileVecs + lane * kConsumers + tid;
+    bool hit = false;
+    if (lane < kPer && v < nvec) hit = Clamp<DT>::vector_max(__ldg(reinterpret_cast<const uint4*>(rowp) + v)) == m;
+    const unsigned int bal = __ballot_sync(0xFFFFFFFFu, hit);
+    return bal ? t * kTileVecs + (__ffs(bal) - 1) * kConsumers + tid : -1;
 }
 // The same over every vector of tiles [tb, te) (many lanes tie for the maximum).
 template <int DT>
@@ -514,8 +508,9 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
             AheadCounter<DT> ahead;
             ahead.count = 0;
             constexpr bool kLazyMax = (K == 1 && ND == 0);   // maximum by value, place found later
-            RunMax<DT> runmax;
-            runmax.init();
+            RunMax<DT> tilemax;     // maximum of the current tile's logits
+            float m_run = -CUDART_INF_F;   // maximum so far and the tile (within the item) that first reached it
+            int m_tile = 0;
             unsigned int row_ctr = 0;
             float neg_refc = 0.f;
             bool alive = true, last = false;
@@ -543,6 +538,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
                 const unsigned char* base = tiles + (size_t)s * kTileBytes;
                 const int v0 = (tb + t) * kTileVecs;
                 const int nv = min(kTileVecs, rj.nvec - v0);
+                if (kLazyMax) tilemax.init();
                 if (ND > 0) {
                     // A thread takes four neighbouring vectors: one sampling group of bf16
                     // ids, half a group of fp32 ids (lane pairs share a group).  The order
@@ -577,7 +573,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
                     for (int k = 0; k < kTileVecs / kConsumers; ++k) {
                         if (kLazyMax) {
                             add_sums<DT, K>(acc, q[k], c1, neg_refc);
-                            runmax.update(q[k]);
+                            tilemax.update(q[k]);
                         } else {
                             acc.add(q[k], v0 + k * kConsumers + tid, c1, neg_refc);
                         }
@@ -592,13 +588,19 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
                         const uint4 q = lds16(base + (size_t)v * 16);
                         if (kLazyMax) {
                             add_sums<DT, K>(acc, q, c1, neg_refc);
-                            runmax.update(q);
+                            tilemax.update(q);
                         } else {
                             acc.add(q, v0 + v, c1, neg_refc);
                         }
                         if (TK) ahead.add(q, v0 + v);
                     }
                     if (TK) ahead.end_tile();
+                }
+                if (kLazyMax) {
+                    const float mt = tilemax.value();
+                    const bool up = mt > m_run;   // strict: the earliest tile stays among equals
+                    m_tile = up ? t : m_tile;
+                    m_run = up ? mt : m_run;
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sh.empty[s]);
@@ -619,7 +621,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
             u64 wk[K];
             if (kLazyMax) {
                 // (warp maximum, lanes that hold it); nothing when every logit was -inf or NaN
-                const float mt = runmax.value();
+                const float mt = m_run;
                 const float mw = warp_max_f32(mt);
                 const unsigned int holders = __ballot_sync(0xFFFFFFFFu, mt == mw);
                 wk[0] = mw > -CUDART_INF_F ? (((u64)ordered_bits(mw) << 32) | (u64)holders) : 0ull;
@@ -661,6 +663,10 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
             }
             int n_ahead = 0;
             if (TK) n_ahead = __reduce_add_sync(0xFFFFFFFFu, ahead.count);
+            if (kLazyMax) {
+                sh.max_tile[p][warp][lane] = (unsigned short)m_tile;
+                __syncwarp();
+            }
             if (lane == 0) {
                 WarpPartial& w = sh.wp[p][warp];
                 w.ahead = n_ahead;
@@ -805,6 +811,11 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
                 races[j].runner = warp_max_f32(runner);
             }
         }
+        unsigned short my_tiles[kConsumerWarps];   // lane l: the tile of lane l of every consumer warp
+        if (K == 1 && ND == 0) {
+#pragma unroll
+            for (int w = 0; w < kConsumerWarps; ++w) my_tiles[w] = sh.max_tile[p][w][lane];
+        }
         __syncwarp();
         if (lane == 0) mbar_arrive(&sh.freeb[p]);
         S = warp_sum_f64(S);
@@ -824,13 +835,15 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
                 int tb, te;
                 tile_range(job, info.row, info.chunk, tb, te);
                 int vfirst = 0x7FFFFFFF;
-                if (n_holders <= 8) {
+                if (n_holders <= 16) {
+#pragma unroll
                     for (int w = 0; w < kConsumerWarps; ++w) {
                         unsigned int lanes = __shfl_sync(0xFFFFFFFFu, mine, w);
                         while (lanes) {
                             const int l = __ffs(lanes) - 1;
                             lanes &= lanes - 1;
-                            const int v = first_vector_of_thread<DT>(rowp, rj.nvec, tb, te, w * 32 + l, m);
+                            const int t = tb + (int)__shfl_sync(0xFFFFFFFFu, (unsigned int)my_tiles[w], l);
+                            const int v = first_vector_in_tile<DT>(rowp, rj.nvec, t, w * 32 + l, m);
                             if (v >= 0 && v < vfirst) vfirst = v;
                         }
                     }
