@@ -7,6 +7,8 @@ namespace aasd {
 
 constexpr int kMaxCands = 64;   // candidates per sequence a draft call can emit
 constexpr int kExtScan = 32;    // depths per main whose extra counts are fetched in parallel
+constexpr int kDraftThreads = 1024;   // one CTA per sequence: long histories want many lanes
+constexpr int kDraftWarps = kDraftThreads / 32;
 
 struct DraftArgs {
     aasd_draft_in in;
@@ -20,13 +22,16 @@ struct DraftArgs {
 // positions that reach the best length are the lookup result of Algorithm 1's dictionary
 // for the longest key that has one (Sec. 3.1: longer keys first).  Warp ballots compact the
 // hits in descending position order.
-__global__ void __launch_bounds__(kThreads) draft_kernel(const DraftArgs a) {
+__global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs a) {
     __shared__ int s_rec[AASD_MAX_NGRAM];
     __shared__ int s_pos[kMaxCands];
-    __shared__ int s_warp[kWarps];
+    __shared__ int s_warp[kDraftWarps];
     __shared__ int s_count;
     __shared__ int s_kstar;
     __shared__ unsigned char s_next[kMaxCands * kExtScan];
+    __shared__ int s_alt[kMaxCands];         // alternatives: (main << 16) | (extra slot << 12)
+    __shared__ int s_alt_depth[kMaxCands];   // and their depth
+    __shared__ int s_total;
 
     pdl_launch_dependents();
     pdl_wait();
@@ -77,7 +82,7 @@ __global__ void __launch_bounds__(kThreads) draft_kernel(const DraftArgs a) {
 
     // pass 1: the longest key that occurs at a place with a continuation (p < len)
     int best = 0;
-    for (int p = 1 + tid; p < len; p += kThreads) best = max(best, match_len_at(p));
+    for (int p = 1 + tid; p < len; p += kDraftThreads) best = max(best, match_len_at(p));
     best = __reduce_max_sync(0xFFFFFFFFu, best);
     if (lane == 0 && best > 0) atomicMax(&s_kstar, best);
     __syncthreads();
@@ -85,22 +90,26 @@ __global__ void __launch_bounds__(kThreads) draft_kernel(const DraftArgs a) {
 
     // pass 2: its places, most recent first
     if (kstar > 0) {
-        for (int base = len - 1; base >= 1; base -= kThreads) {
+        for (int base = len - 1; base >= 1; base -= kDraftThreads) {
             const int p = base - tid;
             const bool hit = p >= 1 && match_len_at(p) == kstar;
             const unsigned int bal = __ballot_sync(0xFFFFFFFFu, hit);
             if (lane == 0) s_warp[warp] = __popc(bal);
             __syncthreads();
-            int before = s_count;
-            for (int w = 0; w < warp; ++w) before += s_warp[w];
+            // hits of the warps before this one: every warp scans the per-warp counts itself
+            const int mine = lane < kDraftWarps ? s_warp[lane] : 0;
+            int incl = mine;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                if (lane >= o) incl += up;
+            }
+            const int before = s_count + __shfl_sync(0xFFFFFFFFu, incl - mine, warp);
+            const int total = __shfl_sync(0xFFFFFFFFu, incl, 31);
             const int rank = before + __popc(bal & ((1u << lane) - 1u));
             if (hit && rank < max_cands) s_pos[rank] = p;
             __syncthreads();
-            if (tid == 0) {
-                int tot = s_count;
-                for (int w = 0; w < kWarps; ++w) tot += s_warp[w];
-                s_count = tot;
-            }
+            if (tid == 0) s_count += total;
             __syncthreads();
             if (s_count >= max_cands) break;
         }
@@ -111,7 +120,7 @@ __global__ void __launch_bounds__(kThreads) draft_kernel(const DraftArgs a) {
     uint8_t* d_fl = a.out.draft_flags + (int64_t)b * max_cands * draft_len;
     int32_t* c_len = a.out.cand_len + (int64_t)b * max_cands;
     int32_t* c_pos = a.out.cand_pos + (int64_t)b * max_cands;
-    for (int i = tid; i < max_cands * draft_len; i += kThreads) {
+    for (int i = tid; i < max_cands * draft_len; i += kDraftThreads) {
         const int c = i / draft_len, j = i % draft_len;
         int tok = AASD_NONE;
         unsigned int fl = 0;
@@ -125,7 +134,7 @@ __global__ void __launch_bounds__(kThreads) draft_kernel(const DraftArgs a) {
         d_ids[i] = tok;
         d_fl[i] = (uint8_t)fl;
     }
-    for (int c = tid; c < max_cands; c += kThreads) {
+    for (int c = tid; c < max_cands; c += kDraftThreads) {
         c_len[c] = c < n_main ? min(draft_len, len - s_pos[c]) : 0;
         c_pos[c] = c < n_main ? s_pos[c] : AASD_NONE;
     }
@@ -133,7 +142,7 @@ __global__ void __launch_bounds__(kThreads) draft_kernel(const DraftArgs a) {
     // serial walk below does not pay a trip to memory per step
     const int scan = min(draft_len, kExtScan);
     if (have_align && n_main < max_cands) {
-        for (int i = tid; i < n_main * scan; i += kThreads) {
+        for (int i = tid; i < n_main * scan; i += kDraftThreads) {
             const int c = i / scan, depth = i % scan;
             const int p = s_pos[c];
             s_next[c * kExtScan + depth] = (unsigned char)(depth < min(draft_len, len - p) ? n_ext(p + depth) : 0);
@@ -142,7 +151,8 @@ __global__ void __launch_bounds__(kThreads) draft_kernel(const DraftArgs a) {
     __syncthreads();
 
     // alternatives: a main's prefix plus one alignment-sampled token (Sec. 3.2), in
-    // (main, depth, extra slot) order while slots remain
+    // (main, depth, extra slot) order while slots remain.  One thread lays the list out from
+    // the counts in shared memory; all threads then write the tokens.
     if (tid == 0) {
         int total = n_main;
         for (int c = 0; c < n_main && total < max_cands && have_align; ++c) {
@@ -151,20 +161,31 @@ __global__ void __launch_bounds__(kThreads) draft_kernel(const DraftArgs a) {
             for (int i = 0; i < L && total < max_cands; ++i) {
                 const int ne = i < scan ? (int)s_next[c * kExtScan + i] : n_ext(p + i);
                 for (int s = 0; s < ne && total < max_cands; ++s) {
-                    const int slot = total++;
-                    for (int q = 0; q < i; ++q) {
-                        d_ids[slot * draft_len + q] = d_ids[c * draft_len + q];
-                        d_fl[slot * draft_len + q] = d_fl[c * draft_len + q];
-                    }
-                    d_ids[slot * draft_len + i] = ext(p + i, s);
-                    d_fl[slot * draft_len + i] = AASD_FLAG_CONDITIONAL | AASD_FLAG_EXTRA;
-                    c_len[slot] = i + 1;
-                    c_pos[slot] = p;
+                    s_alt[total] = (c << 16) | (s << 12) | 0;   // main and extra slot; the depth goes beside
+                    s_alt_depth[total] = i;
+                    ++total;
                 }
             }
         }
+        s_total = total;
         a.out.n_cands[b] = total;
         a.out.match_len[b] = kstar;
+    }
+    __syncthreads();
+    const int total = s_total;
+    for (int i = tid; i < (total - n_main) * draft_len; i += kDraftThreads) {
+        const int slot = n_main + i / draft_len, q = i % draft_len;
+        const int c = s_alt[slot] >> 16, es = (s_alt[slot] >> 12) & 15, depth = s_alt_depth[slot];
+        const int p = s_pos[c];
+        if (q < depth) {
+            d_ids[slot * draft_len + q] = h[p + q];
+            d_fl[slot * draft_len + q] = (uint8_t)((p + q < plen) ? AASD_FLAG_CONDITIONAL : 0u);
+        } else if (q == depth) {
+            d_ids[slot * draft_len + q] = ext(p + depth, es);
+            d_fl[slot * draft_len + q] = (uint8_t)(AASD_FLAG_CONDITIONAL | AASD_FLAG_EXTRA);
+            c_len[slot] = depth + 1;
+            c_pos[slot] = p;
+        }
     }
 }
 
