@@ -50,8 +50,9 @@ __device__ __forceinline__ void philox4x32_10(unsigned int c0, unsigned int c1, 
     constexpr unsigned int M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
 #pragma unroll
     for (int round = 0; round < 10; ++round) {
-        const unsigned int hi0 = __umulhi(M0, c0), lo0 = M0 * c0;
-        const unsigned int hi1 = __umulhi(M1, c2), lo1 = M1 * c2;
+        const u64 p0 = (u64)M0 * c0, p1 = (u64)M1 * c2;   // one wide multiply each
+        const unsigned int hi0 = (unsigned int)(p0 >> 32), lo0 = (unsigned int)p0;
+        const unsigned int hi1 = (unsigned int)(p1 >> 32), lo1 = (unsigned int)p1;
         const unsigned int n0 = hi1 ^ c1 ^ k0, n2 = hi0 ^ c3 ^ k1;
         c0 = n0;
         c1 = lo1;

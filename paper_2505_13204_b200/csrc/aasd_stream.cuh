@@ -294,17 +294,19 @@ __device__ __forceinline__ void add_sums(TileAccumulator<DT, K>& acc, const uint
 }
 
 // First vector (lowest index) with maximum m among the vectors thread `tid` of the consumers
-// read in tile t: vectors t * 1024 + k * 256 + tid.  By a whole warp; -1 if none.
-template <int DT>
+// read in tile t: vectors t * 1024 + k * 256 + tid, or, in sampling kernels (GROUPED), the four
+// neighbours t * 1024 + 4 * tid + k.  By a whole warp; -1 if none.
+template <int DT, bool GROUPED>
 __device__ int first_vector_in_tile(const char* rowp, int nvec, int t, int tid, float m) {
     constexpr int kTileVecs = kTileBytes / 16;
     constexpr int kPer = kTileVecs / kConsumers;
     const int lane = threadIdx.x & 31;
-    const int v = t * kTileVecs + lane * kConsumers + tid;
+    const int step = GROUPED ? 1 : kConsumers, first = GROUPED ? kPer * tid : tid;
+    const int v = t * kTileVecs + first + lane * step;
     bool hit = false;
     if (lane < kPer && v < nvec) hit = Clamp<DT>::vector_max(__ldg(reinterpret_cast<const uint4*>(rowp) + v)) == m;
     const unsigned int bal = __ballot_sync(0xFFFFFFFFu, hit);
-    return bal ? t * kTileVecs + (__ffs(bal) - 1) * kConsumers + tid : -1;
+    return bal ? t * kTileVecs + first + (__ffs(bal) - 1) * step : -1;
 }
 // The same over every vector of tiles [tb, te) (many lanes tie for the maximum).
 template <int DT>
@@ -395,11 +397,11 @@ template <> struct AheadCounter<AASD_F32> {
     }
 };
 
-// The same for a sampling kernel: the sum of the vector's weights goes to `gs` (the caller
-// adds a whole group's sum to S at once, and needs it for the group's ratio).
+// The sums of one vector in a sampling kernel: the sum of the vector's weights goes to `gs`
+// (the caller adds a whole group's sum to S at once, and needs it for the group's ratio).
 template <int DT, int K>
-__device__ __forceinline__ void add_to_group(TileAccumulator<DT, K>& acc, const uint4& raw, int vec_index, float c1,
-                                             float neg_refc, float2& gs) {
+__device__ __forceinline__ void add_to_group(TileAccumulator<DT, K>& acc, const uint4& raw, float c1, float neg_refc,
+                                             float2& gs) {
     constexpr int kVec = Elt<DT>::kVec;
     float x[kVec];
     Elt<DT>::unpack(Clamp<DT>::apply(raw), x);
@@ -411,21 +413,6 @@ __device__ __forceinline__ void add_to_group(TileAccumulator<DT, K>& acc, const 
         float2 e = make_float2(ex2_approx(t.x), ex2_approx(t.y));
         gs = __fadd2_rn(gs, e);
         acc.A2[i] = __ffma2_rn(e, t, acc.A2[i]);
-    }
-    float vmax = Clamp<DT>::vector_max(raw);
-    int vi = vec_index;
-#pragma unroll
-    for (int j = 0; j < K; ++j) {
-        // a thread does not meet its vectors in ascending order here: equal maxima go by index
-        const bool up = vmax > acc.best[j] || (vmax == acc.best[j] && vi < acc.best_vec[j]);
-        const float hi = fmaxf(acc.best[j], vmax);
-        const float lo = fminf(acc.best[j], vmax);
-        const int hi_i = up ? vi : acc.best_vec[j];
-        const int lo_i = up ? acc.best_vec[j] : vi;
-        acc.best[j] = hi;
-        acc.best_vec[j] = hi_i;
-        vmax = lo;
-        vi = lo_i;
     }
 }
 
@@ -507,7 +494,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
             race.init();
             AheadCounter<DT> ahead;
             ahead.count = 0;
-            constexpr bool kLazyMax = (K == 1 && ND == 0);   // maximum by value, place found later
+            constexpr bool kLazyMax = (K == 1);   // maximum by value, place found later
             RunMax<DT> tilemax;     // maximum of the current tile's logits
             float m_run = -CUDART_INF_F;   // maximum so far and the tile (within the item) that first reached it
             int m_tile = 0;
@@ -558,7 +545,10 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
                     float2 gs = make_float2(0.f, 0.f);
 #pragma unroll
                     for (int k = 0; k < kPer; ++k)
-                        if (ok[k]) add_to_group<DT, K>(acc, q[k], v0 + kPer * tid + ((k + rot) & 3), c1, neg_refc, gs);
+                        if (ok[k]) {
+                            add_to_group<DT, K>(acc, q[k], c1, neg_refc, gs);
+                            tilemax.update(q[k]);
+                        }
                     acc.S2[0] = __fadd2_rn(acc.S2[0], gs);
                     float gsum = gs.x + gs.y;
                     constexpr int kThreadsPerGroup = kGroup / (kPer * kVec);   // 1 (bf16) or 2 (fp32)
@@ -812,7 +802,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
             }
         }
         unsigned short my_tiles[kConsumerWarps];   // lane l: the tile of lane l of every consumer warp
-        if (K == 1 && ND == 0) {
+        if (K == 1) {
 #pragma unroll
             for (int w = 0; w < kConsumerWarps; ++w) my_tiles[w] = sh.max_tile[p][w][lane];
         }
@@ -822,7 +812,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
         A = warp_sum_f64(A);
         if (TK) n_ahead = warp_sum_i64(n_ahead);
         u64 mk[K];   // merged vector keys, identical in every lane
-        if (K == 1 && ND == 0) {
+        if (K == 1) {
             // the consumers reported (maximum, lanes holding it) per warp: find the first vector
             // of the item that attains the maximum
             const unsigned int top = (unsigned int)(vk[0] >> 32);
@@ -843,7 +833,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
                             const int l = __ffs(lanes) - 1;
                             lanes &= lanes - 1;
                             const int t = tb + (int)__shfl_sync(0xFFFFFFFFu, (unsigned int)my_tiles[w], l);
-                            const int v = first_vector_in_tile<DT>(rowp, rj.nvec, t, w * 32 + l, m);
+                            const int v = first_vector_in_tile<DT, (ND > 0)>(rowp, rj.nvec, t, w * 32 + l, m);
                             if (v >= 0 && v < vfirst) vfirst = v;
                         }
                     }
