@@ -364,7 +364,7 @@ int aasd_verify_tree(aasd_ctx* ctx, const void* target_logits, const int32_t* no
  * aasd_verify needs a context (aasd_create allocates its status block) and a caller-made
  * workspace; this entry point needs neither.  Its scratch - what the workspace and the
  * context's status block would hold - lives in a fixed block of device memory that is part
- * of the library image: about 0.5 MB on every GPU that loads the library, held until the
+ * of the library image: about 0.75 MB on every GPU that loads the library, held until the
  * process exits.  The call itself makes no cudaMalloc / cudaFree and calls nothing that
  * allocates.
  *
