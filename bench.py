@@ -46,8 +46,8 @@ N_BUF = 8
 # captures summarised under profiles/: (workload, kernel) -> (rows captured, bytes).  Traffic
 # is proportional to rows (each row is read once), so it is scaled to the launch's rows.
 # An entry is set to None whenever the kernel has changed since its capture.
-NCU_TRAFFIC = {("cfg5-serving-256", "verify"): (2048, 623.228672e6 + 4.375296e6),
-               ("cfg5-serving-256", "align"): (2048, 623.322880e6 + 6.061312e6)}
+NCU_TRAFFIC = {("cfg5-serving-256", "verify"): (2048, 623.236096e6 + 4.400896e6),
+               ("cfg5-serving-256", "align"): (2048, 623.325952e6 + 6.254848e6)}
 
 
 def ncu_traffic(workload: str, kernel: str, rows: int):
