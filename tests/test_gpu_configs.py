@@ -108,7 +108,7 @@ def _run_config(index, n_follow, align_mode=binding.ALIGN_TOPK, verify_mode=bind
     cap = w.steps * (w.draft_len + 1) + 8
     align = dict(align_ids=table_ids, n_extra=table_n)
     st = binding.DecodeState(ctx, prompts, cap, w.ngram, w.draft_len, w.max_cands, V, w.torch_dtype, align=align,
-                             alpha=ALPHA, beta=BETA, mode=verify_mode, seed=seed)
+                             alpha=ALPHA, beta=BETA, mode=verify_mode, seed=seed, top_k=5)
     hoffs_all = cpu(st.hist_offsets)
     F = n_follow
     hoffs = (hoffs_all[:F + 1] - hoffs_all[0]).astype(np.int32)
@@ -142,7 +142,7 @@ def _run_config(index, n_follow, align_mode=binding.ALIGN_TOPK, verify_mode=bind
         # the followed sequences, element by element
         ref = oracle.verify(to_oracle(x[:RF]), dr["draft_ids"].reshape(-1), coffs,
                             draft_flags=dr["draft_flags"].reshape(-1), alpha=ALPHA, beta=BETA, mode=verify_mode,
-                            seed=seed, step=s, threads=THREADS)
+                            seed=seed, step=s, threads=THREADS, top_k=5)
         sel = oracle.select(ref["accept_len"], ref["next_token"], dr["draft_ids"].reshape(-1), coffs, soffs,
                             w.draft_len + 1)
         oracle.append(hist, hoffs, hlen, sel["emit_ids"], sel["n_emit"])
@@ -197,6 +197,7 @@ def test_config1_pr1_reference_all_modes():
 def test_config2_single_sequence_2k():
     r = _run_config(1, 1)
     assert r["tokens_per_step"] >= 1.0
+    _run_config(1, 1, verify_mode=binding.VERIFY_TOP_K)      # the paper's ablation (k = 5)
 
 
 def test_config3_batch32_4k():

@@ -122,17 +122,21 @@ def test_verify_tree_parity(ctx, V, dtype, stride, B, Cm, Ld, mode):
         assert torch.equal(got[k], again[k]), k
 
 
-def test_tree_from_the_drafter_end_to_end(ctx):
-    """aasd_draft -> aasd_tree_build -> aasd_verify_tree -> aasd_append against the oracle on a
-    reduced configuration, closed loop."""
-    w = synth.scaled(synth.workload(2), batch=3, vocab=4096, prompt_len=300, steps=5)
+@pytest.mark.parametrize("scale", [dict(batch=3, vocab=4096, prompt_len=300, steps=5),
+                                   dict(batch=32, prompt_len=512, steps=4)])
+def test_tree_from_the_drafter_end_to_end(ctx, scale):
+    """aasd_draft -> aasd_tree_build -> aasd_verify_tree -> aasd_append against the oracle, closed
+    loop: on a reduced configuration, and on the batch-32 configuration at its full vocabulary
+    (shorter prompts, a few steps)."""
+    w = synth.scaled(synth.workload(2), **scale)
     alpha, beta = F32(0.1), F32(0.1)
     prompts = [synth.prompt_ids(w, b) for b in range(w.batch)]
     hints = torch.cat([synth.next_token_hints(p) for p in prompts])
     pre = synth.logits(hints.numel(), w.vocab, w.torch_dtype, w.recipe, hints, w.seed)
     seq_offs = np.concatenate([[0], np.cumsum([p.numel() for p in prompts])]).astype(np.int32)
     ids_all = torch.cat(prompts)
-    a_ref = oracle.align_sample(to_oracle(pre), ids_all.numpy(), seq_offs, k_extra=2)
+    import os
+    a_ref = oracle.align_sample(to_oracle(pre), ids_all.numpy(), seq_offs, k_extra=2, threads=os.cpu_count() or 1)
     a_gpu = ctx.align_sample(pre.cuda(), ids_all.cuda(), seq_offs, k_extra=2)
     st = binding.DecodeState(ctx, prompts, 64, w.ngram, w.draft_len, w.max_cands, w.vocab, w.torch_dtype,
                              align=a_gpu, alpha=alpha, beta=beta)
@@ -165,7 +169,8 @@ def test_tree_from_the_drafter_end_to_end(ctx):
             for v in range(hi - lo - 1, 0, -1):
                 hint[lo + par[lo + v]] = tok[lo + v]
         x = synth.logits(R, w.vocab, w.torch_dtype, w.recipe, torch.as_tensor(hint), w.seed * 31 + s)
-        ref = oracle.verify_tree(to_oracle(x), tok, par, offs, E, node_flags=fl, alpha=alpha, beta=beta)
+        ref = oracle.verify_tree(to_oracle(x), tok, par, offs, E, node_flags=fl, alpha=alpha, beta=beta,
+                                 threads=os.cpu_count() or 1)
         got = ctx.verify_tree(x.cuda(), _dev(tok), _dev(par), offs, E, node_flags=_dev(fl, torch.uint8),
                               alpha=alpha, beta=beta)
         assert _check_tree(got, ref, w.torch_dtype) == 0
