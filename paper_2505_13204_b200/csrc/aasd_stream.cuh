@@ -1,6 +1,6 @@
 // Persistent, warp-specialised streaming of logits rows (sm_100a).
 //
-// One CTA per SM slot runs for the whole launch.  A producer warp moves 16 KB tiles of the
+// One CTA per SM slot runs for the whole launch.  A producer warp moves 32 KB tiles of the
 // rows from HBM into a ring of shared-memory stages with bulk asynchronous copies (TMA,
 // cp.async.bulk, completion signalled on an mbarrier); eight consumer warps turn each tile
 // into running sums and best-token candidates; a finisher warp merges what the consumers
@@ -24,8 +24,8 @@
 
 namespace aasd {
 
-constexpr int kTileBytes = 16384;
-constexpr int kStages = 6;
+constexpr int kTileBytes = 32768;
+constexpr int kStages = 3;
 constexpr int kConsumerWarps = 8;
 constexpr int kConsumers = kConsumerWarps * 32;
 constexpr int kStreamThreads = kConsumers + 64;   // + producer warp + finisher warp
@@ -250,7 +250,7 @@ struct TileAccumulator {
 // which a thread met its maximum: a thread keeps the maximum of each tile's logits (one
 // packed max per word) and, once per tile, the running maximum with the tile that first
 // reached it; the warp reports the maximum and which lanes hold it, and the finisher looks
-// the first such vector up among the four vectors that lane read in that tile.
+// the first such vector up among the eight vectors that lane read in that tile.
 template <int DT> struct RunMax;
 template <> struct RunMax<AASD_BF16> {
     unsigned int m2;   // bf16x2
@@ -294,8 +294,8 @@ __device__ __forceinline__ void add_sums(TileAccumulator<DT, K>& acc, const uint
 }
 
 // First vector (lowest index) with maximum m among the vectors thread `tid` of the consumers
-// read in tile t: vectors t * 1024 + k * 256 + tid, or, in sampling kernels (GROUPED), the four
-// neighbours t * 1024 + 4 * tid + k.  By a whole warp; -1 if none.
+// read in tile t: vectors t * 2048 + k * 256 + tid, or, in sampling kernels (GROUPED), the eight
+// neighbours t * 2048 + 8 * tid + k.  By a whole warp; -1 if none.
 template <int DT, bool GROUPED>
 __device__ int first_vector_in_tile(const char* rowp, int nvec, int t, int tid, float m) {
     constexpr int kTileVecs = kTileBytes / 16;
@@ -527,34 +527,43 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
                 const int nv = min(kTileVecs, rj.nvec - v0);
                 if (kLazyMax) tilemax.init();
                 if (ND > 0) {
-                    // A thread takes four neighbouring vectors: one sampling group of bf16
-                    // ids, half a group of fp32 ids (lane pairs share a group).  The order
-                    // in which it reads them is rotated by the lane so that a quarter-warp
-                    // covers all shared-memory banks.
+                    // A thread takes the eight neighbouring vectors 8 * tid .. 8 * tid + 7 of the
+                    // tile: two sampling groups of bf16 ids, one group of fp32 ids.  The order in
+                    // which it reads them is rotated by the lane so that a quarter-warp covers
+                    // all shared-memory banks.
                     constexpr int kPer = kTileVecs / kConsumers;
-                    static_assert(kPer == 4, "four vectors per thread and tile");
-                    const int rot = (lane >> 1) & 3;
+                    constexpr int kVecsPerGroup = kGroup / kVec;           // 4 (bf16) or 8 (fp32)
+                    constexpr int kGroupsPerThread = kPer / kVecsPerGroup; // 2 or 1
+                    static_assert(kPer == 8 && kGroupsPerThread >= 1, "eight vectors per thread and tile");
+                    const int rot = lane & (kPer - 1);
                     uint4 q[kPer];
                     bool ok[kPer];
 #pragma unroll
                     for (int k = 0; k < kPer; ++k) {
-                        const int v = kPer * tid + ((k + rot) & 3);
+                        const int v = kPer * tid + ((k + rot) & (kPer - 1));
                         ok[k] = v < nv;
                         if (ok[k]) q[k] = lds16(base + (size_t)v * 16);
                     }
-                    float2 gs = make_float2(0.f, 0.f);
+                    float2 gs[kGroupsPerThread];
+#pragma unroll
+                    for (int gi = 0; gi < kGroupsPerThread; ++gi) gs[gi] = make_float2(0.f, 0.f);
 #pragma unroll
                     for (int k = 0; k < kPer; ++k)
                         if (ok[k]) {
-                            add_to_group<DT, K>(acc, q[k], c1, neg_refc, gs);
+                            float2 one = make_float2(0.f, 0.f);
+                            add_to_group<DT, K>(acc, q[k], c1, neg_refc, one);
                             tilemax.update(q[k]);
+                            const int gi = ((k + rot) & (kPer - 1)) / kVecsPerGroup;   // the group this vector belongs to
+#pragma unroll
+                            for (int j = 0; j < kGroupsPerThread; ++j)
+                                if (gi == j) gs[j] = __fadd2_rn(gs[j], one);
                         }
-                    acc.S2[0] = __fadd2_rn(acc.S2[0], gs);
-                    float gsum = gs.x + gs.y;
-                    constexpr int kThreadsPerGroup = kGroup / (kPer * kVec);   // 1 (bf16) or 2 (fp32)
-                    if (kThreadsPerGroup == 2) gsum += __shfl_xor_sync(0xFFFFFFFFu, gsum, 1);
-                    const int g = (v0 + kPer * tid) * kVec / kGroup;
-                    if (g < job.full_groups && (tid % kThreadsPerGroup) == 0) race.offer(gsum, g, row_ctr, job.smp);
+                    const int g0 = (v0 + kPer * tid) * kVec / kGroup;
+#pragma unroll
+                    for (int gi = 0; gi < kGroupsPerThread; ++gi) {
+                        acc.S2[0] = __fadd2_rn(acc.S2[0], gs[gi]);
+                        if (g0 + gi < job.full_groups) race.offer(gs[gi].x + gs[gi].y, g0 + gi, row_ctr, job.smp);
+                    }
                 } else if (nv == kTileVecs) {
                     uint4 q[kTileVecs / kConsumers];
 #pragma unroll
