@@ -2,6 +2,7 @@
 // launch geometry.  Every step of the path runs in the kernels of aasd_rows.cuh and
 // aasd_tokens.cuh; nothing here computes on the host.
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
 
 #include <cstdio>
 #include <cstdlib>
@@ -17,6 +18,14 @@
 #include "aasd_tree.cuh"
 
 using namespace aasd;
+
+namespace {
+// Named range around an entry point, visible to tools that collect NVTX (no cost without one).
+struct TraceRange {
+    explicit TraceRange(const char* name) { nvtxRangePushA(name); }
+    ~TraceRange() { nvtxRangePop(); }
+};
+}  // namespace
 
 namespace {
 
@@ -374,6 +383,7 @@ int aasd_align_sample(aasd_ctx* ctx, const void* prefill_logits, const int32_t* 
                       const int32_t* seq_offsets, int32_t n_seqs, int64_t n_rows,
                       const aasd_align_params* p, void* workspace, size_t workspace_bytes,
                       const aasd_align_out* out) {
+    TraceRange trace("aasd_align_sample");
     if (ctx == nullptr || p == nullptr || out == nullptr) return AASD_ERR_INVALID_ARG;
     if (n_seqs < 0 || n_rows < 0) return AASD_ERR_BAD_SHAPE;
     if (p->k_extra < 0 || p->k_extra > AASD_MAX_EXTRA) return AASD_ERR_INVALID_ARG;
@@ -425,6 +435,7 @@ int aasd_align_sample(aasd_ctx* ctx, const void* prefill_logits, const int32_t* 
 }
 
 int aasd_draft(aasd_ctx* ctx, const aasd_draft_in* in, const aasd_draft_params* p, const aasd_draft_out* out) {
+    TraceRange trace("aasd_draft");
     if (ctx == nullptr || in == nullptr || p == nullptr || out == nullptr) return AASD_ERR_INVALID_ARG;
     if (p->n_seqs < 0) return AASD_ERR_BAD_SHAPE;
     if (p->n < 1 || p->n > AASD_MAX_NGRAM || p->draft_len < 1 || p->max_cands < 1 || p->max_cands > kMaxCands)
@@ -516,6 +527,7 @@ int aasd_verify(aasd_ctx* ctx, const void* target_logits, const int32_t* draft_i
                 const uint8_t* draft_flags, const int32_t* cand_offsets, int32_t n_cands,
                 int64_t n_rows, const aasd_verify_params* p, void* workspace, size_t workspace_bytes,
                 const aasd_verify_out* out) {
+    TraceRange trace("aasd_verify");
     return verify_impl(ctx, target_logits, draft_ids, draft_flags, cand_offsets, n_cands, n_rows, p, workspace,
                        workspace_bytes, out, nullptr);
 }
@@ -524,6 +536,7 @@ int aasd_select(aasd_ctx* ctx, const int32_t* accept_len, const int32_t* next_to
                 const int32_t* draft_ids, const int32_t* cand_offsets, int32_t rows_per_cand,
                 const int32_t* seq_cand_offsets, int32_t cands_per_seq, int32_t n_seqs,
                 int32_t emit_stride, int32_t* best_cand, int32_t* n_emit, int32_t* emit_ids) {
+    TraceRange trace("aasd_select");
     if (ctx == nullptr) return AASD_ERR_INVALID_ARG;
     if (n_seqs < 0 || emit_stride < 1) return AASD_ERR_BAD_SHAPE;
     if (n_seqs == 0) return AASD_OK;
@@ -539,6 +552,7 @@ int aasd_select(aasd_ctx* ctx, const int32_t* accept_len, const int32_t* next_to
 
 int aasd_append(aasd_ctx* ctx, int32_t* hist_ids, const int32_t* hist_offsets, int32_t* hist_len,
                 const int32_t* emit_ids, const int32_t* n_emit, int32_t n_seqs, int32_t emit_stride) {
+    TraceRange trace("aasd_append");
     if (ctx == nullptr) return AASD_ERR_INVALID_ARG;
     if (n_seqs < 0 || emit_stride < 1) return AASD_ERR_BAD_SHAPE;
     if (n_seqs == 0) return AASD_OK;
@@ -550,6 +564,7 @@ int aasd_append(aasd_ctx* ctx, int32_t* hist_ids, const int32_t* hist_offsets, i
 }
 
 int aasd_step(aasd_ctx* ctx, const aasd_step_args* s, void* workspace, size_t workspace_bytes) {
+    TraceRange trace("aasd_step");
     if (ctx == nullptr || s == nullptr) return AASD_ERR_INVALID_ARG;
     const aasd_draft_params& dp = s->draft;
     if (!s->hist_ids || !s->hist_len || !s->best_cand || !s->n_emit || !s->emit_ids) return AASD_ERR_INVALID_ARG;
@@ -607,6 +622,7 @@ extern "C" int aasd_tree_build(aasd_ctx* ctx, const int32_t* draft_ids, const ui
                                const int32_t* cand_len, const int32_t* n_cands, int32_t n_seqs, int32_t max_cands,
                                int32_t draft_len, int32_t* node_token, int32_t* node_parent, uint8_t* node_flags,
                                int32_t* node_depth, int32_t* n_nodes) {
+    TraceRange trace("aasd_tree_build");
     if (ctx == nullptr) return AASD_ERR_INVALID_ARG;
     if (n_seqs < 0 || max_cands < 1 || draft_len < 1) return AASD_ERR_BAD_SHAPE;
     if (n_seqs == 0) return AASD_OK;
@@ -627,6 +643,7 @@ extern "C" int aasd_verify_tree(aasd_ctx* ctx, const void* target_logits, const 
                                 const int32_t* node_parent, const uint8_t* node_flags, const int32_t* tree_offsets,
                                 int32_t n_trees, int64_t n_rows, const aasd_verify_params* p, int32_t emit_stride,
                                 void* workspace, size_t workspace_bytes, const aasd_tree_out* out) {
+    TraceRange trace("aasd_verify_tree");
     if (ctx == nullptr || p == nullptr || out == nullptr) return AASD_ERR_INVALID_ARG;
     if (n_trees < 0 || n_rows < 0 || emit_stride < 1) return AASD_ERR_BAD_SHAPE;
     if (p->mode < AASD_VERIFY_CONDITIONAL || p->mode > AASD_VERIFY_STRICT_SAMPLED) return AASD_ERR_UNSUPPORTED;
