@@ -251,6 +251,19 @@ def run_ours(args, rank, world, local_rank):
     verify_ms = float(np.mean([e[2].elapsed_time(e[3]) for e in evs]))
     ms = shard.max_over_ranks(ms, dev)
 
+    # what a read-only stream with no arithmetic reaches on this device, same buffers, same run
+    sink = torch.zeros(1, dtype=torch.int32, device=dev)
+    for j in range(3):
+        bench.ctx.probe_read(bench.ver_bufs[j % N_BUF], sink)
+    p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    p0.record()
+    for j in range(16):
+        bench.ctx.probe_read(bench.ver_bufs[j % N_BUF], sink)
+    p1.record()
+    torch.cuda.synchronize()
+    buf_bytes = bench.ver_bufs[0].numel() * bench.ver_bufs[0].element_size()
+    read_probe_gbs = 16 * buf_bytes / (p0.elapsed_time(p1) * 1e-3) / 1e9
+
     # end to end: the same step fed from pinned host memory through the C ABI
     e2e = run_e2e(bench, dev, min(K, 4))
     e2e["ms_per_step"] = shard.max_over_ranks(e2e["ms_per_step"], dev)
@@ -288,14 +301,17 @@ def run_ours(args, rank, world, local_rank):
                      "kernel": "stream_kernel<%s, K=1, ND=0, VerifyEpilogue> (verification with the accept scan, "
                                "selection and append fused)" % w.dtype,
                      "achieved": ver_gbs, "peak": peak, "unit": "GB/s", "frac": ver_gbs / peak,
+                     "frac_of_nominal_8000": ver_gbs / 8000.0, "frac_of_read_probe": ver_gbs / read_probe_gbs,
                      "peak_source": peak_src, "traffic": ncu_traffic(w.name, "verify", bench.R),
                      "ms_per_launch": verify_ms, "bytes_per_launch": bench.R * row_bytes},
         "roofline_align": {"bound": "hbm",
                            "kernel": "align_next_kernel + stream_kernel<%s, K=%d, ND=0, AlignEpilogue>" % (w.dtype, K_EXTRA),
                            "achieved": ali_gbs, "peak": peak, "unit": "GB/s", "frac": ali_gbs / peak,
+                           "frac_of_nominal_8000": ali_gbs / 8000.0, "frac_of_read_probe": ali_gbs / read_probe_gbs,
                            "peak_source": peak_src, "traffic": ncu_traffic(w.name, "align", bench.pre_rows),
                            "ms_per_launch": align_ms, "bytes_per_launch": bench.pre_rows * row_bytes},
         "draft_us_per_launch": draft_ms * 1e3,
+        "read_probe_gbs": read_probe_gbs,
         "logits_gbs": (bench.R + bench.pre_rows) * row_bytes * K / (ms * 1e-3) / 1e9,
         "accepted_tokens_per_s": world * bench.accepted_per_cycle / N_BUF * K / (ms * 1e-3),
         "mean_tokens_per_seq_step": bench.accepted_per_cycle / N_BUF / w.batch,

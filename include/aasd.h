@@ -350,6 +350,14 @@ int aasd_verify_tree(aasd_ctx* ctx, const void* target_logits, const int32_t* no
                      const aasd_verify_params* params, int32_t emit_stride, void* workspace,
                      size_t workspace_bytes, const aasd_tree_out* out);
 
+/* ---- measurement aid ------------------------------------------------------------------ */
+
+/* Reads `bytes` bytes at `buffer` (16-byte aligned, bytes a multiple of 16) once with plain
+ * vector loads and folds them into *sink (4 bytes, DEVICE): no arithmetic to speak of, so the
+ * time of this launch is what the device's memory system allows a read-only stream.  The
+ * benchmark reports it beside the kernels' figures; it is not part of the method. */
+int aasd_probe_read(aasd_ctx* ctx, const void* buffer, size_t bytes, uint32_t* sink);
+
 /* ---- verification for callers that cannot allocate ------------------------------- */
 
 #define AASD_STATIC_MAX_ROWS 8192   /* most logits rows per aasd_verify_static call */

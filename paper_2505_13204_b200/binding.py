@@ -27,7 +27,7 @@ EXPORTS = [
     "aasd_get_counters", "aasd_reset_counters", "aasd_launch_count", "aasd_workspace_bytes",
     "aasd_workspace_init", "aasd_workspace_release", "aasd_align_sample", "aasd_draft",
     "aasd_verify", "aasd_select", "aasd_append", "aasd_step", "aasd_verify_static",
-    "aasd_tree_build", "aasd_verify_tree",
+    "aasd_tree_build", "aasd_verify_tree", "aasd_probe_read",
 ]
 STATIC_MAX_ROWS = STATIC_MAX_CANDS = 8192
 
@@ -132,6 +132,7 @@ def load_library(path: str | None = None):
     lib.aasd_verify_tree.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, C.c_int32, C.c_int64,
                                      C.POINTER(VerifyParams), C.c_int32, _vp, C.c_size_t,
                                      C.POINTER(TreeOut)]
+    lib.aasd_probe_read.argtypes = [_vp, _vp, C.c_size_t, _vp]
     lib.aasd_verify_static.argtypes = [C.c_int, _vp, _vp, _vp, _vp, _vp, C.c_int32, C.c_int64,
                                        C.POINTER(VerifyParams), C.POINTER(VerifyOut), _vp]
     if path == _build.LIB:
@@ -420,6 +421,11 @@ class Context:
                                          int(emit_stride), _p(ws), ws.numel(), C.byref(out)),
                "aasd_verify_tree")
         return o
+
+    def probe_read(self, buffer: torch.Tensor, sink: torch.Tensor):
+        """aasd_probe_read: one read-only pass over ``buffer`` (a measurement aid)."""
+        n = buffer.numel() * buffer.element_size()
+        _check(self.lib.aasd_probe_read(self._h, _p(buffer), n - n % 16, _p(sink)), "aasd_probe_read")
 
     def select(self, accept_len, next_token, draft_ids, emit_stride, cand_offsets=None,
                rows_per_cand=0, seq_cand_offsets=None, cands_per_seq=0, n_seqs=None):

@@ -598,6 +598,16 @@ int aasd_step(aasd_ctx* ctx, const aasd_step_args* s, void* workspace, size_t wo
 
 }  // extern "C"
 
+extern "C" int aasd_probe_read(aasd_ctx* ctx, const void* buffer, size_t bytes, uint32_t* sink) {
+    if (ctx == nullptr || buffer == nullptr || sink == nullptr) return AASD_ERR_INVALID_ARG;
+    if (((uintptr_t)buffer % 16) != 0 || (bytes % 16) != 0) return AASD_ERR_INVALID_ARG;
+    if (bytes == 0) return AASD_OK;
+    AASD_CUDA(cudaSetDevice(ctx->device));
+    launch(probe_read_kernel, (unsigned int)(ctx->sm_count * 32), 256u, 0, ctx->stream,
+           static_cast<const uint4*>(buffer), bytes / 16, sink);
+    return after_launch(ctx, 1);
+}
+
 // ---- draft trees ----------------------------------------------------------------------------
 
 namespace {
