@@ -42,6 +42,9 @@ ALPHA = float(np.float32(0.1))
 BETA = float(np.float32(0.1))
 K_EXTRA = 2
 N_BUF = 8
+# The stand-in logits are a language-model head's: finite everywhere (no masked tokens), and
+# the calls say so (AASD_HINT_FINITE).  --no-finite-hint times the path that tolerates -inf.
+FINITE_HINT = True
 # DRAM bytes (read + write) per captured launch of the streaming kernels, from the ncu
 # captures summarised under profiles/: (workload, kernel) -> (rows captured, bytes).  Traffic
 # is proportional to rows (each row is read once), so it is scaled to the launch's rows.
@@ -156,7 +159,7 @@ class Bench:
                              device=device, out=buf if keep else scratch,
                              noise=self.bank.block(k), chunk_rows=1024)
             out = self._align_out(lo)
-            self.ctx.align_sample(x, ids, offs, k_extra=K_EXTRA, outputs=out)
+            self.ctx.align_sample(x, ids, offs, k_extra=K_EXTRA, outputs=out, finite_hint=FINITE_HINT)
             if keep:
                 self.pre_bufs.append(x)
                 self.pre_ids.append(ids)
@@ -168,7 +171,7 @@ class Bench:
         align = dict(align_ids=self.table["align_ids"], n_extra=self.table["n_extra"])
         self.state = binding.DecodeState(self.ctx, self.prompts, N_BUF * (w.draft_len + 1) + 8, w.ngram,
                                          w.draft_len, w.max_cands, w.vocab, w.torch_dtype, align=align,
-                                         alpha=ALPHA, beta=BETA)
+                                         alpha=ALPHA, beta=BETA, finite_hint=FINITE_HINT)
         self.hist0 = self.state.hist_ids.clone()
         self.len0 = self.state.hist_len.clone()
         self.ver_bufs = []
@@ -202,7 +205,7 @@ class Bench:
         if events is not None:
             events[0].record()
         self.ctx.align_sample(self.pre_bufs[ja], self.pre_ids[ja], self.pre_offs[ja], k_extra=K_EXTRA,
-                              outputs=self.pre_out[ja])
+                              outputs=self.pre_out[ja], finite_hint=FINITE_HINT)
         if events is not None:
             events[1].record()
         self.state.run_draft()
@@ -287,7 +290,7 @@ def run_ours(args, rank, world, local_rank):
         "config": {"workload": w.name, "sequences_per_gpu": w.batch, "vocab": w.vocab,
                    "logits_dtype": w.dtype, "verify_rows_per_step": bench.R,
                    "prefill_rows_per_step": bench.pre_rows, "ngram": w.ngram, "k_extra": K_EXTRA,
-                   "alpha": ALPHA, "beta": BETA, "parallelism": "replicas x%d (sequences sharded, no collective)" % world,
+                   "alpha": ALPHA, "beta": BETA, "finite_hint": FINITE_HINT, "parallelism": "replicas x%d (sequences sharded, no collective)" % world,
                    "l2": "inputs larger than L2: %d rotating buffers of %.2f GB" % (2 * N_BUF, bench.R * row_bytes / 1e9),
                    "noise": "one bank of normals re-used under cyclic shifts",
                    "setup_s": round(bench.setup_s, 1)},
@@ -395,7 +398,7 @@ def run_e2e(bench: Bench, dev, steps: int):
         dpre.copy_(host_pre, non_blocking=True)
         dver.copy_(host_ver, non_blocking=True)
         bench.ctx.align_sample(dpre, bench.pre_ids[0], bench.pre_offs[0], k_extra=K_EXTRA,
-                               outputs=bench.pre_out[0])
+                               outputs=bench.pre_out[0], finite_hint=FINITE_HINT)
         st.step(dver, 0)
         res_emit.copy_(st.emit_ids, non_blocking=True)
         res_n.copy_(st.n_emit, non_blocking=True)
@@ -522,7 +525,8 @@ def run_micro(args):
     def call(j):
         nonlocal outs
         if args.micro == "verify":
-            outs = ctx.verify(bufs[j], ids[j], None, alpha=ALPHA, beta=BETA, rows_per_cand=rpc, outputs=outs)
+            outs = ctx.verify(bufs[j], ids[j], None, alpha=ALPHA, beta=BETA, rows_per_cand=rpc, outputs=outs,
+                              finite_hint=FINITE_HINT)
         elif args.micro == "verify-sampled":
             outs = ctx.verify(bufs[j], ids[j], None, rows_per_cand=rpc, outputs=outs, seed=17, step=j,
                               mode=binding.VERIFY_STRICT_SAMPLED)
@@ -530,7 +534,7 @@ def run_micro(args):
             outs = ctx.align_sample(bufs[j], ids[j], offs, k_extra=K_EXTRA, outputs=outs, seed=17,
                                     mode=binding.ALIGN_GUMBEL)
         else:
-            outs = ctx.align_sample(bufs[j], ids[j], offs, k_extra=K_EXTRA, outputs=outs)
+            outs = ctx.align_sample(bufs[j], ids[j], offs, k_extra=K_EXTRA, outputs=outs, finite_hint=FINITE_HINT)
 
     for s in range(max(args.warmup, 1)):
         call(s % n_buf)
@@ -586,7 +590,11 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-latency", action="store_true", help="skip the decode-step latencies of configs 1-4")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--no-finite-hint", action="store_true",
+                    help="do not tell the library that the logits hold no -inf")
     args = ap.parse_args()
+    global FINITE_HINT
+    FINITE_HINT = not args.no_finite_hint
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))

@@ -57,6 +57,14 @@ typedef enum aasd_status {
 
 typedef enum aasd_dtype { AASD_F32 = 0, AASD_BF16 = 1 } aasd_dtype;
 
+/* aasd_align_params.hints / aasd_verify_params.hints: performance hints, never needed for
+ * correct results. */
+#define AASD_HINT_FINITE 1u /* the logits are expected to hold no -inf (no masked tokens), as a
+                               language-model head produces them: the streaming pass then skips
+                               the step that makes masked tokens harmless.  A row that holds -inf
+                               all the same is still evaluated correctly, by a much slower second
+                               pass over that row (counted in redo_rows). */
+
 /* How the extra tokens of a misaligned position are chosen. */
 typedef enum aasd_align_mode {
     AASD_ALIGN_TOPK = 0,   /* the tokens ranked above the prompt token (Fig. 2) */
@@ -141,6 +149,7 @@ typedef struct aasd_align_params {
     int32_t mode;           /* aasd_align_mode */
     uint32_t stream_tag;    /* distinguishes random streams of calls sharing a seed */
     uint64_t seed;          /* key of the counter-based generator (GUMBEL mode) */
+    uint32_t hints;         /* AASD_HINT_* */
 } aasd_align_params;
 
 typedef struct aasd_align_out {
@@ -222,6 +231,7 @@ typedef struct aasd_verify_params {
     uint32_t step;          /* decoding step, part of the sampler's counter */
     uint64_t seed;
     int32_t top_k;          /* AASD_VERIFY_TOP_K: how many of the row's best tokens pass (>= 1) */
+    uint32_t hints;         /* AASD_HINT_* */
 } aasd_verify_params;
 
 typedef struct aasd_verify_out {

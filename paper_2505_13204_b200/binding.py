@@ -20,6 +20,7 @@ VERIFY_CONDITIONAL, VERIFY_STRICT_GREEDY, VERIFY_STRICT_SAMPLED, VERIFY_TOP_K = 
 STATUS_BAD_ROW, STATUS_ID_RANGE, STATUS_HIST_OVERFLOW, STATUS_BAD_OFFSETS = 1, 2, 4, 8
 FLAG_CONDITIONAL, FLAG_EXTRA = 1, 2
 DRAFT_MATCH_ALIGN = 1
+HINT_FINITE = 1
 STEP_REUSE_DRAFT = 1
 
 EXPORTS = [
@@ -37,7 +38,7 @@ _vp = C.c_void_p
 class AlignParams(C.Structure):
     _fields_ = [("vocab", C.c_int32), ("dtype", C.c_int32), ("row_stride", C.c_int64),
                 ("inv_temperature", C.c_float), ("k_extra", C.c_int32), ("mode", C.c_int32),
-                ("stream_tag", C.c_uint32), ("seed", C.c_uint64)]
+                ("stream_tag", C.c_uint32), ("seed", C.c_uint64), ("hints", C.c_uint32)]
 
 
 class AlignOut(C.Structure):
@@ -65,7 +66,7 @@ class VerifyParams(C.Structure):
     _fields_ = [("vocab", C.c_int32), ("dtype", C.c_int32), ("row_stride", C.c_int64),
                 ("alpha", C.c_float), ("beta", C.c_float), ("inv_temperature", C.c_float),
                 ("mode", C.c_int32), ("rows_per_cand", C.c_int32), ("step", C.c_uint32),
-                ("seed", C.c_uint64), ("top_k", C.c_int32)]
+                ("seed", C.c_uint64), ("top_k", C.c_int32), ("hints", C.c_uint32)]
 
 
 class VerifyOut(C.Structure):
@@ -291,8 +292,9 @@ class Context:
 
     # ---- the path -----------------------------------------------------------------------
     def align_sample(self, prefill_logits, prompt_ids, seq_offsets, k_extra=2, mode=ALIGN_TOPK,
-                     seed=0, stream_tag=0, inv_temperature=1.0, outputs=None):
-        """aasd_align_sample.  Returns a dict of device tensors (see include/aasd.h)."""
+                     seed=0, stream_tag=0, inv_temperature=1.0, outputs=None, finite_hint=False):
+        """aasd_align_sample.  Returns a dict of device tensors (see include/aasd.h).
+        ``finite_hint``: the logits are expected to hold no -inf (AASD_HINT_FINITE)."""
         x = prefill_logits
         assert x.is_cuda and x.dim() == 2 and x.stride(1) == 1
         R, V = x.shape
@@ -311,7 +313,7 @@ class Context:
             pmax=torch.empty(R, dtype=torch.float32, device=dev),
             aligned=torch.empty(R, dtype=torch.uint8, device=dev))
         prm = AlignParams(V, _dtype_code(x), x.stride(0), float(inv_temperature), K, int(mode),
-                          int(stream_tag), int(seed))
+                          int(stream_tag), int(seed), HINT_FINITE if finite_hint else 0)
         out = AlignOut(*[_p(o.get(n)) for n, _ in AlignOut._fields_])
         ws = self.workspace(R, 1)
         _check(self.lib.aasd_align_sample(self._h, _p(x), _p(ids), _p(offs), B, R, C.byref(prm),
@@ -342,7 +344,7 @@ class Context:
 
     def verify(self, target_logits, draft_ids, cand_offsets=None, draft_flags=None, alpha=0.1,
                beta=0.1, mode=VERIFY_CONDITIONAL, seed=0, step=0, inv_temperature=1.0,
-               rows_per_cand=0, outputs=None, top_k=5):
+               rows_per_cand=0, outputs=None, top_k=5, finite_hint=False):
         """aasd_verify.  ``cand_offsets=None`` means regular candidates of ``rows_per_cand``."""
         x = target_logits
         assert x.is_cuda and x.dim() == 2 and x.stride(1) == 1
@@ -364,7 +366,7 @@ class Context:
             n_greater=torch.empty(R, dtype=torch.int32, device=dev))
         prm = VerifyParams(V, _dtype_code(x), x.stride(0), float(alpha), float(beta),
                            float(inv_temperature), int(mode), int(rows_per_cand), int(step),
-                           int(seed), int(top_k))
+                           int(seed), int(top_k), HINT_FINITE if finite_hint else 0)
         out = VerifyOut(*[_p(o.get(n)) for n, _ in VerifyOut._fields_])
         ws = self.workspace(R, Cn)
         fl = None if draft_flags is None else draft_flags.reshape(-1)
@@ -455,7 +457,8 @@ class DecodeState:
 
     def __init__(self, ctx: Context, prompts, capacity_extra: int, n: int, draft_len: int,
                  max_cands: int, vocab: int, dtype: torch.dtype, align=None, alpha=0.1, beta=0.1,
-                 mode=VERIFY_CONDITIONAL, inv_temperature=1.0, seed=0, match_align=False, top_k=5):
+                 mode=VERIFY_CONDITIONAL, inv_temperature=1.0, seed=0, match_align=False, top_k=5,
+                 finite_hint=False):
         dev = ctx.device
         self.ctx = ctx
         B = len(prompts)
@@ -513,7 +516,7 @@ class DecodeState:
         a.draft_out = DraftOut(*[_p(self.draft_out[k]) for k, _ in DraftOut._fields_])
         a.verify = VerifyParams(vocab, F32 if dtype == torch.float32 else BF16, vocab, float(alpha),
                                 float(beta), float(inv_temperature), int(mode), draft_len, 0,
-                                int(seed), int(top_k))
+                                int(seed), int(top_k), HINT_FINITE if finite_hint else 0)
         a.verify_out = VerifyOut(*[_p(self.verify_out[k]) for k, _ in VerifyOut._fields_])
         a.hist_ids, a.hist_len = _p(self.hist_ids), _p(self.hist_len)
         a.best_cand, a.n_emit, a.emit_ids = _p(self.best_cand), _p(self.n_emit), _p(self.emit_ids)

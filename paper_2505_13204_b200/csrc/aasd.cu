@@ -222,9 +222,9 @@ int enable_stream_smem(Kernel kernel) {
                : AASD_ERR_CUDA;
 }
 
-template <int DT, int K, int ND>
+template <int DT, int K, int ND, bool FIN = false>
 int launch_align_stream(aasd_ctx* ctx, const StreamJob& sj, const AlignArgs& a, unsigned int grid) {
-    auto kernel = stream_kernel<DT, K, ND, false, AlignEpilogue<DT>>;
+    auto kernel = stream_kernel<DT, K, ND, false, FIN, AlignEpilogue<DT>>;
     if (enable_stream_smem(kernel) != AASD_OK) return AASD_ERR_CUDA;
     launch(kernel, grid, kStreamThreads, kStreamSmemBytes, ctx->stream, sj, a);
     return AASD_OK;
@@ -240,14 +240,19 @@ int dispatch_align_stream(aasd_ctx* ctx, const StreamJob& sj, const AlignArgs& a
         if (k == 2) return launch_align_stream<DT, 1, 2>(ctx, sj, a, grid);
         return launch_align_stream<DT, 1, 4>(ctx, sj, a, grid);
     }
+    if (a.hints & AASD_HINT_FINITE) {
+        if (k == 1) return launch_align_stream<DT, 1, 0, true>(ctx, sj, a, grid);
+        if (k == 2) return launch_align_stream<DT, 2, 0, true>(ctx, sj, a, grid);
+        return launch_align_stream<DT, 4, 0, true>(ctx, sj, a, grid);
+    }
     if (k == 1) return launch_align_stream<DT, 1, 0>(ctx, sj, a, grid);
     if (k == 2) return launch_align_stream<DT, 2, 0>(ctx, sj, a, grid);
     return launch_align_stream<DT, 4, 0>(ctx, sj, a, grid);
 }
 
-template <int DT, int ND, bool TK>
+template <int DT, int ND, bool TK, bool FIN = false>
 int launch_verify_stream(aasd_ctx* ctx, const StreamJob& sj, const VerifyArgs& a, unsigned int grid) {
-    auto kernel = stream_kernel<DT, 1, ND, TK, VerifyEpilogue<DT>>;
+    auto kernel = stream_kernel<DT, 1, ND, TK, FIN, VerifyEpilogue<DT>>;
     if (enable_stream_smem(kernel) != AASD_OK) return AASD_ERR_CUDA;
     launch(kernel, grid, kStreamThreads, kStreamSmemBytes, ctx->stream, sj, a);
     return AASD_OK;
@@ -257,6 +262,7 @@ template <int DT>
 int dispatch_verify_stream(aasd_ctx* ctx, const StreamJob& sj, const VerifyArgs& a, unsigned int grid) {
     if (a.mode == AASD_VERIFY_STRICT_SAMPLED) return launch_verify_stream<DT, 1, false>(ctx, sj, a, grid);
     if (a.mode == AASD_VERIFY_TOP_K) return launch_verify_stream<DT, 0, true>(ctx, sj, a, grid);
+    if (a.hints & AASD_HINT_FINITE) return launch_verify_stream<DT, 0, false, true>(ctx, sj, a, grid);
     return launch_verify_stream<DT, 0, false>(ctx, sj, a, grid);
 }
 
@@ -403,6 +409,7 @@ int aasd_align_sample(aasd_ctx* ctx, const void* prefill_logits, const int32_t* 
     a.n_seqs = n_seqs;
     a.k_extra = p->k_extra;
     a.mode = p->mode;
+    a.hints = p->hints;
     a.next_ids = reinterpret_cast<int32_t*>(ws + L->off_next);
     a.smp = make_sample_job(p->seed, p->stream_tag, true, p->inv_temperature);
     a.out = *out;
@@ -488,6 +495,7 @@ int verify_impl(aasd_ctx* ctx, const void* target_logits, const int32_t* draft_i
     a.beta = p->beta;
     a.mode = p->mode;
     a.top_k = p->top_k;
+    a.hints = p->hints;
     a.cand_tickets = reinterpret_cast<unsigned int*>(ws + L->off_cand_tickets);
     a.row_accept = reinterpret_cast<uint8_t*>(ws + L->off_row_accept);
     a.row_own = reinterpret_cast<int32_t*>(ws + L->off_row_own);
@@ -614,7 +622,7 @@ namespace {
 
 template <int DT, int ND>
 int launch_tree_stream(aasd_ctx* ctx, const StreamJob& sj, const TreeArgs& a, unsigned int grid) {
-    auto kernel = stream_kernel<DT, 1, ND, false, TreeEpilogue<DT>>;
+    auto kernel = stream_kernel<DT, 1, ND, false, false, TreeEpilogue<DT>>;
     if (enable_stream_smem(kernel) != AASD_OK) return AASD_ERR_CUDA;
     launch(kernel, grid, kStreamThreads, kStreamSmemBytes, ctx->stream, sj, a);
     return AASD_OK;
@@ -806,6 +814,7 @@ extern "C" int aasd_verify_static(int device, void* stream, const void* target_l
     a.beta = p->beta;
     a.mode = p->mode;
     a.top_k = p->top_k;
+    a.hints = p->hints;
     a.cand_tickets = reinterpret_cast<unsigned int*>(ws + L.off_cand_tickets);
     a.row_accept = reinterpret_cast<uint8_t*>(ws + L.off_row_accept);
     a.row_own = reinterpret_cast<int32_t*>(ws + L.off_row_own);

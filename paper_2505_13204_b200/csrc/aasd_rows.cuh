@@ -324,6 +324,7 @@ struct VerifyArgs {
     int32_t* row_own;              // scratch [n_rows]
     SampleJob smp;                 // STRICT_SAMPLED: the row's own token is a keyed draw
     int top_k;                     // TOP_K mode
+    unsigned int hints;            // AASD_HINT_*
     SeqTail seq;
     aasd_verify_out out;
 };
@@ -578,6 +579,7 @@ struct AlignArgs {
     int n_seqs;
     int k_extra;
     int mode;
+    unsigned int hints;   // AASD_HINT_*
     int32_t* next_ids;   // scratch [n_rows]: the prompt's next token of every row
     SampleJob smp;       // GUMBEL mode: the extras are keyed draws
     aasd_align_out out;

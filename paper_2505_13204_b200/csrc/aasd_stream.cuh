@@ -216,9 +216,10 @@ struct TileAccumulator {
             best_vec[j] = -1;
         }
     }
+    template <bool FIN>
     __device__ __forceinline__ void add(const uint4& raw, int vec_index, float c1, float neg_refc) {
         float x[kVec];
-        Elt<DT>::unpack(Clamp<DT>::apply(raw), x);
+        Elt<DT>::unpack(FIN ? raw : Clamp<DT>::apply(raw), x);
         const float2 cc = make_float2(c1, c1);
         const float2 rr = make_float2(neg_refc, neg_refc);
 #pragma unroll
@@ -277,11 +278,11 @@ template <> struct RunMax<AASD_F32> {
 };
 
 // The sums of one vector without any maximum tracking.
-template <int DT, int K>
+template <int DT, int K, bool FIN>
 __device__ __forceinline__ void add_sums(TileAccumulator<DT, K>& acc, const uint4& raw, float c1, float neg_refc) {
     constexpr int kVec = Elt<DT>::kVec;
     float x[kVec];
-    Elt<DT>::unpack(Clamp<DT>::apply(raw), x);
+    Elt<DT>::unpack(FIN ? raw : Clamp<DT>::apply(raw), x);
     const float2 cc = make_float2(c1, c1);
     const float2 rr = make_float2(neg_refc, neg_refc);
 #pragma unroll
@@ -455,7 +456,9 @@ struct FinishedRow {
 //   - entered by the whole finisher warp
 //   ND: keyed draws per row the kernel prepares (0: no sampling)
 //   TK: count the tokens ahead of the hinted token (top-k verification)
-template <int DT, int K, int ND, bool TK, class E>
+//   FIN: the logits are expected to hold no -inf: the clamp that makes masked tokens harmless
+//        is skipped, and a row that holds one is re-evaluated by the finisher (its sums are NaN)
+template <int DT, int K, int ND, bool TK, bool FIN, class E>
 __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJob job, const typename E::Args args) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* tiles = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
@@ -571,10 +574,10 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
 #pragma unroll
                     for (int k = 0; k < kTileVecs / kConsumers; ++k) {
                         if (kLazyMax) {
-                            add_sums<DT, K>(acc, q[k], c1, neg_refc);
+                            add_sums<DT, K, FIN>(acc, q[k], c1, neg_refc);
                             tilemax.update(q[k]);
                         } else {
-                            acc.add(q[k], v0 + k * kConsumers + tid, c1, neg_refc);
+                            acc.template add<FIN>(q[k], v0 + k * kConsumers + tid, c1, neg_refc);
                         }
                     }
                     if (TK) {
@@ -586,10 +589,10 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
                     for (int v = tid; v < nv; v += kConsumers) {
                         const uint4 q = lds16(base + (size_t)v * 16);
                         if (kLazyMax) {
-                            add_sums<DT, K>(acc, q, c1, neg_refc);
+                            add_sums<DT, K, FIN>(acc, q, c1, neg_refc);
                             tilemax.update(q);
                         } else {
-                            acc.add(q, v0 + v, c1, neg_refc);
+                            acc.template add<FIN>(q, v0 + v, c1, neg_refc);
                         }
                         if (TK) ahead.add(q, v0 + v);
                     }

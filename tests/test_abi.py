@@ -44,7 +44,7 @@ def test_status_strings_and_workspace_size_without_gpu():
 
 def test_struct_sizes_match_the_header_layout():
     # natural alignment of the C structs in include/aasd.h
-    assert ctypes.sizeof(binding.AlignParams) == 40
+    assert ctypes.sizeof(binding.AlignParams) == 48
     assert ctypes.sizeof(binding.VerifyParams) == 56
     assert ctypes.sizeof(binding.DraftParams) == 24
     assert ctypes.sizeof(binding.Counters) == 64

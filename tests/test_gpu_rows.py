@@ -260,6 +260,34 @@ def test_rows_with_masked_entries_far_maxima_and_bad_rows(ctx):
     assert ctx.counters()["redo_rows"] > 0
 
 
+@pytest.mark.parametrize("V,dtype,stride,rows", [c for c in CASES if c[0] >= 1000])
+def test_finite_hint_gives_the_same_results(ctx, V, dtype, stride, rows):
+    """AASD_HINT_FINITE only changes how the streaming pass treats masked tokens; results are
+    the oracle's with and without it, also on rows that do hold -inf (those take the slow
+    second pass)."""
+    rng = np.random.default_rng(V + 3 * rows)
+    d = rng.integers(0, V, rows).astype(np.int32)
+    x = _make_logits(rows, V, dtype, 700 + V, torch.as_tensor(d, dtype=torch.int64), stride=stride)
+    x[1, 5:V // 2] = -float("inf")                  # a masked row in spite of the hint
+    x[2, :] = -float("inf"); x[2, 7] = 0.25
+    offs = _random_csr(rng, rows)
+    alpha, beta = F32(0.1), F32(0.05)
+    ref = oracle.verify(to_oracle(x), d, offs, alpha=alpha, beta=beta)
+    ctx.reset_counters()
+    got = ctx.verify(_to_dev(x), torch.as_tensor(d).cuda(), torch.as_tensor(offs).cuda(), alpha=alpha, beta=beta,
+                     finite_hint=True)
+    check_verify(got, ref, offs, dtype)
+    prompt = rng.integers(0, V, rows).astype(np.int32)
+    refa = oracle.align_sample(to_oracle(x), prompt, [0, rows], k_extra=2)
+    gota = ctx.align_sample(_to_dev(x), torch.as_tensor(prompt).cuda(), [0, rows], k_extra=2, finite_hint=True)
+    check_align(gota, refa, dtype)
+    assert ctx.poll_status() == 0
+    c = ctx.counters()
+    vector_path = (stride is not None) or (V * (4 if dtype == torch.float32 else 2)) % 16 == 0
+    if vector_path:
+        assert c["redo_rows"] >= 2          # the masked rows were noticed and re-evaluated
+
+
 def test_temperature_and_thresholds(ctx):
     V, rows = 2048, 64
     rng = np.random.default_rng(11)
