@@ -154,10 +154,12 @@ def _run_config(index, n_follow, align_mode=binding.ALIGN_TOPK, verify_mode=bind
             assert np.array_equal(cpu(st.emit_ids[:F]), sel["emit_ids"])
             assert np.array_equal(cpu(st.hist_len[:F]), hlen)
             assert np.array_equal(cpu(st.hist_ids)[:hoffs_all[F]], hist)
-        else:   # a decision inside the 1e-6 band may differ: resynchronise the oracle's state
-            hist[:] = cpu(st.hist_ids)[:hoffs_all[F]]
-            hlen[:] = cpu(st.hist_len)[:F]
         emitted += int(sel["n_emit"].sum())
+        if near:
+            # a decision inside the 1e-6 band may legitimately differ, after which the two
+            # histories need not agree any more: the closed-loop comparison ends here (the
+            # oracle is never fed from the GPU's state)
+            break
         # every sequence: the outputs are consistent with one another
         vo = st.verify_out
         acc = vo["accept"].view(B, w.max_cands, w.draft_len).to(torch.int32)
@@ -183,7 +185,7 @@ def _run_config(index, n_follow, align_mode=binding.ALIGN_TOPK, verify_mode=bind
     assert ctx.poll_status() == 0
     c = ctx.counters()
     ctx.close()
-    assert emitted >= w.steps * F       # every step emits at least the target's own token
+    assert near_total or emitted >= w.steps * F   # every step emits at least the target's own token
     return dict(misaligned=misaligned, tokens_per_step=emitted / (w.steps * F), near=near_total, counters=c)
 
 
