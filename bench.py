@@ -451,7 +451,9 @@ def cpu_baseline(w: synth.Workload, seconds: float = 12.0):
         t += dt
         done += r
         reps += 1
+    t1, r1 = oracle_sample(w, 16, 1)          # the same program on one core, for scale
     return {"value": done / t, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "single_core_value": r1 / t1,
             "sample": "%d x (%d prefill rows through alignment sampling + %d verification rows) of %s, "
                       "OpenMP over rows, %.1f s of oracle time" % (reps, rows, rows, w.name, t)}
 
