@@ -45,6 +45,9 @@ N_BUF = 8
 # The stand-in logits are a language-model head's: finite everywhere (no masked tokens), and
 # the calls say so (AASD_HINT_FINITE).  --no-finite-hint times the path that tolerates -inf.
 FINITE_HINT = True
+# --extend-table: the step also enters the emitted tokens into the alignment table (alignment
+# sampling on generated context), which makes verification keep two best tokens per row.
+EXTEND_TABLE = False
 # DRAM bytes (read + write) per captured launch of the streaming kernels, from the ncu
 # captures summarised under profiles/: (workload, kernel) -> (rows captured, bytes).  Traffic
 # is proportional to rows (each row is read once), so it is scaled to the launch's rows.
@@ -171,9 +174,11 @@ class Bench:
         align = dict(align_ids=self.table["align_ids"], n_extra=self.table["n_extra"])
         self.state = binding.DecodeState(self.ctx, self.prompts, N_BUF * (w.draft_len + 1) + 8, w.ngram,
                                          w.draft_len, w.max_cands, w.vocab, w.torch_dtype, align=align,
-                                         alpha=ALPHA, beta=BETA, finite_hint=FINITE_HINT)
+                                         alpha=ALPHA, beta=BETA, finite_hint=FINITE_HINT,
+                                         extend_table=EXTEND_TABLE)
         self.hist0 = self.state.hist_ids.clone()
         self.len0 = self.state.hist_len.clone()
+        self.tab0 = (self.state.align["align_ids"].clone(), self.state.align["n_extra"].clone()) if EXTEND_TABLE else None
         self.ver_bufs = []
         for j in range(N_BUF):
             d = self.state.run_draft()["draft_ids"].reshape(-1).to(torch.int64)
@@ -196,6 +201,9 @@ class Bench:
     def restore(self):
         self.state.hist_ids.copy_(self.hist0)
         self.state.hist_len.copy_(self.len0)
+        if self.tab0 is not None:
+            self.state.align["align_ids"].copy_(self.tab0[0])
+            self.state.align["n_extra"].copy_(self.tab0[1])
 
     def step(self, s: int, events=None):
         j = s % N_BUF
@@ -290,7 +298,7 @@ def run_ours(args, rank, world, local_rank):
         "config": {"workload": w.name, "sequences_per_gpu": w.batch, "vocab": w.vocab,
                    "logits_dtype": w.dtype, "verify_rows_per_step": bench.R,
                    "prefill_rows_per_step": bench.pre_rows, "ngram": w.ngram, "k_extra": K_EXTRA,
-                   "alpha": ALPHA, "beta": BETA, "finite_hint": FINITE_HINT, "parallelism": "replicas x%d (sequences sharded, no collective)" % world,
+                   "alpha": ALPHA, "beta": BETA, "finite_hint": FINITE_HINT, "extend_table": EXTEND_TABLE, "parallelism": "replicas x%d (sequences sharded, no collective)" % world,
                    "l2": "inputs larger than L2: %d rotating buffers of %.2f GB" % (2 * N_BUF, bench.R * row_bytes / 1e9),
                    "noise": "one bank of normals re-used under cyclic shifts",
                    "setup_s": round(bench.setup_s, 1)},
@@ -594,9 +602,12 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--no-finite-hint", action="store_true",
                     help="do not tell the library that the logits hold no -inf")
+    ap.add_argument("--extend-table", action="store_true",
+                    help="alignment sampling on generated context inside the step")
     args = ap.parse_args()
-    global FINITE_HINT
+    global FINITE_HINT, EXTEND_TABLE
     FINITE_HINT = not args.no_finite_hint
+    EXTEND_TABLE = args.extend_table
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))

@@ -289,6 +289,8 @@ int aasd_append(aasd_ctx* ctx, int32_t* hist_ids, const int32_t* hist_offsets,
 #define AASD_STEP_REUSE_DRAFT 1u /* draft_out already holds this state's candidates (the caller
                                     ran aasd_draft, e.g. to feed the model): do not draft again */
 
+#define AASD_STEP_EXTEND_TABLE 2u /* also enter the emitted tokens into the alignment table (below) */
+
 typedef struct aasd_step_args {
     aasd_draft_in draft_in;        /* recent_ids == NULL: the key is the history's own tail */
     aasd_draft_params draft;
@@ -302,6 +304,8 @@ typedef struct aasd_step_args {
     int32_t* n_emit;               /* [n_seqs] */
     int32_t* emit_ids;             /* [n_seqs x (draft_len+1)] */
     uint32_t flags;                /* AASD_STEP_* */
+    int32_t* table_ids;            /* AASD_STEP_EXTEND_TABLE: the alignment table, writable */
+    int32_t* table_n;              /*   (normally the arrays draft_in.align_ids / align_n name) */
 } aasd_step_args;
 
 /* draft -> verify -> select -> append on the context's stream (Algorithm 1, loop body), in
@@ -312,6 +316,22 @@ typedef struct aasd_step_args {
  * made that call passes AASD_STEP_REUSE_DRAFT and the step is the second launch alone. */
 int aasd_step(aasd_ctx* ctx, const aasd_step_args* args, void* workspace,
               size_t workspace_bytes);
+
+/* Alignment sampling on generated context (AASD_STEP_EXTEND_TABLE).  The paper samples
+ * extras for the input context only and names the generated context as an extension
+ * (Limitations) without defining it; this is Fig. 2's rule applied to the rows the step has
+ * at hand.  Row i of the winning candidate is the distribution its token i was judged
+ * under, so for every emitted draft token d the extras are those of that row's
+ * draft.k_extra best tokens (logit descending, ties by lower id) that rank above d - what
+ * aasd_align_sample (TOPK) gives for a row whose next token is d - and the target's own
+ * token that ends the emission gets none.  They go to the table row of the token's position
+ * q, draft_in.align_row_offsets[b] + q - 1 (table_n, and table_ids padded with NONE), in the
+ * launch that appends the token; positions beyond the history's capacity are dropped like
+ * their tokens.  The table must therefore have a row for every position of every history
+ * buffer (rows laid out like hist_offsets), and a caller who wants drafts to use the new
+ * rows passes prompt_len = hist_len to aasd_draft.  CONDITIONAL and STRICT_GREEDY modes,
+ * draft.k_extra 1 or 2, rows the streaming kernel takes (16-byte aligned, vocab * element
+ * size >= 16); AASD_ERR_UNSUPPORTED otherwise. */
 
 /* ---- draft trees (Eq. 2, Sec. 3.2) and their verification (Sec. 3.3) ---------------- */
 

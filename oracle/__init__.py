@@ -252,3 +252,37 @@ def append(hist_ids, hist_offsets, hist_len, emit_ids, n_emit):
                              _ptr(n_emit), B, int(emit_ids.shape[1]), _ptr(overflow))
     assert rc == 0
     return overflow
+
+
+def extend_table(logits, cand_offsets, accept_len, best_cand, emit_ids, n_emit, hist_offsets,
+                 hist_len_before, table_ids, table_n, table_row_offsets, inv_temperature=1.0):
+    """Alignment sampling on generated context, in place on ``table_ids`` [rows x K] and
+    ``table_n`` [rows] (int32 numpy arrays).  The paper samples extras for the input context
+    (Sec. 2.3, Fig. 2) and names generated context as an extension (Limitations) without
+    defining it; here Fig. 2's rule is applied to the rows a decoding step has at hand.  Row
+    i of the winning candidate is the distribution its token i was judged under, so the
+    extras of an emitted draft token are what ``align_sample`` (TOPK) gives for that row
+    with the token as the row's next token; the target's own token that ends the emission
+    gets none.  They go to the table row of the token's position q, row offset + q - 1;
+    positions beyond the buffer's capacity are dropped like their tokens.  ``hist_len_before``
+    is the length before the step's tokens were appended."""
+    assert table_ids.dtype == np.int32 and table_n.dtype == np.int32
+    x, _, _ = _logits(logits)
+    K = table_ids.shape[1]
+    cand_offsets, hist_offsets = _i32(cand_offsets), _i32(hist_offsets)
+    for b in range(len(best_cand)):
+        cap = hist_offsets[b + 1] - hist_offsets[b]
+        c = int(best_cand[b])
+        for i in range(int(n_emit[b])):
+            q = int(hist_len_before[b]) + i
+            if q >= cap or q < 1:
+                continue
+            ids, n = np.full(K, NONE, np.int32), 0
+            if c != NONE and i < int(accept_len[c]):
+                r = int(cand_offsets[c]) + i
+                pair = align_sample(x[[r, r]], [0, int(emit_ids[b][i])], [0, 2], k_extra=K,
+                                    mode=ALIGN_TOPK, inv_temperature=inv_temperature)
+                ids, n = pair["align_ids"][0], int(pair["n_extra"][0])
+            row = int(table_row_offsets[b]) + q - 1
+            table_ids[row] = ids
+            table_n[row] = n

@@ -22,6 +22,8 @@ FLAG_CONDITIONAL, FLAG_EXTRA = 1, 2
 DRAFT_MATCH_ALIGN = 1
 HINT_FINITE = 1
 STEP_REUSE_DRAFT = 1
+STEP_EXTEND_TABLE = 2
+ERR_UNSUPPORTED = 7
 
 EXPORTS = [
     "aasd_create", "aasd_destroy", "aasd_set_stream", "aasd_status_str", "aasd_poll_status",
@@ -83,7 +85,7 @@ class StepArgs(C.Structure):
     _fields_ = [("draft_in", DraftIn), ("draft", DraftParams), ("draft_out", DraftOut),
                 ("target_logits", _vp), ("verify", VerifyParams), ("verify_out", VerifyOut),
                 ("hist_ids", _vp), ("hist_len", _vp), ("best_cand", _vp), ("n_emit", _vp),
-                ("emit_ids", _vp), ("flags", C.c_uint32)]
+                ("emit_ids", _vp), ("flags", C.c_uint32), ("table_ids", _vp), ("table_n", _vp)]
 
 
 class Counters(C.Structure):
@@ -458,7 +460,11 @@ class DecodeState:
     def __init__(self, ctx: Context, prompts, capacity_extra: int, n: int, draft_len: int,
                  max_cands: int, vocab: int, dtype: torch.dtype, align=None, alpha=0.1, beta=0.1,
                  mode=VERIFY_CONDITIONAL, inv_temperature=1.0, seed=0, match_align=False, top_k=5,
-                 finite_hint=False):
+                 finite_hint=False, extend_table=False):
+        """``extend_table``: alignment sampling on generated context.  The table given in
+        ``align`` (rows of the prompts, back to back) is copied into one with a row for every
+        position of every history buffer; each step enters the extras of the tokens it emits,
+        and drafting looks extras up at generated positions too."""
         dev = ctx.device
         self.ctx = ctx
         B = len(prompts)
@@ -480,6 +486,19 @@ class DecodeState:
             for L in lens:
                 ro.append(ro[-1] + L)
             self.align_row_offsets = torch.tensor(ro[:-1], dtype=torch.int32, device=dev)
+        self.extend_table = bool(extend_table)
+        if extend_table:
+            if align is None:
+                raise ValueError("extend_table needs an alignment table")
+            K = int(align["align_ids"].shape[1])
+            ids = torch.full((offs[-1], K), NONE, dtype=torch.int32, device=dev)
+            cnt = torch.zeros(offs[-1], dtype=torch.int32, device=dev)
+            for b, L in enumerate(lens):
+                ids[offs[b]:offs[b] + L] = align["align_ids"][ro[b]:ro[b] + L]
+                cnt[offs[b]:offs[b] + L] = align["n_extra"][ro[b]:ro[b] + L]
+            self.align = align = dict(align_ids=ids, n_extra=cnt)
+            self.align_row_offsets = self.hist_offsets[:-1].clone()
+            self.prompt_len = self.hist_len      # every position held has a table row
         R = B * max_cands * draft_len
         Cn = B * max_cands
         self.draft_out = dict(
@@ -520,6 +539,8 @@ class DecodeState:
         a.verify_out = VerifyOut(*[_p(self.verify_out[k]) for k, _ in VerifyOut._fields_])
         a.hist_ids, a.hist_len = _p(self.hist_ids), _p(self.hist_len)
         a.best_cand, a.n_emit, a.emit_ids = _p(self.best_cand), _p(self.n_emit), _p(self.emit_ids)
+        if extend_table:
+            a.table_ids, a.table_n = _p(align["align_ids"]), _p(align["n_extra"])
         self.args = a
 
     def run_draft(self):
@@ -536,7 +557,7 @@ class DecodeState:
         a = self.args
         a.target_logits = _p(target_logits)
         a.verify.row_stride = target_logits.stride(0)
-        a.flags = STEP_REUSE_DRAFT if reuse_draft else 0
+        a.flags = (STEP_REUSE_DRAFT if reuse_draft else 0) | (STEP_EXTEND_TABLE if self.extend_table else 0)
         a.verify.step = int(step_index)
         _check(self.ctx.lib.aasd_step(self.ctx._h, C.byref(a), _p(self.ws), self.ws.numel()),
                "aasd_step")

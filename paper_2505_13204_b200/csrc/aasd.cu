@@ -33,13 +33,14 @@ struct WorkspaceLayout {
     size_t bytes;
     int64_t max_rows, max_cands;
     size_t off_partials, off_row_tickets, off_cand_tickets, off_seq_tickets, off_sched, off_row_accept, off_row_own, off_next, off_race,
-        off_tree_stats;
+        off_tree_stats, off_row_extra;
+    bool full;
 };
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-// with_tree: room for the per-row statistics of tree verification (the fixed block of
-// aasd_verify_static does without).
+// with_tree: room for the per-row statistics of tree verification and for the per-row extras
+// of the table extension (the fixed block of aasd_verify_static does without both).
 WorkspaceLayout make_layout(int64_t max_rows, int64_t max_cands, bool with_tree = true) {
     WorkspaceLayout L{};
     L.max_rows = max_rows;
@@ -65,6 +66,9 @@ WorkspaceLayout make_layout(int64_t max_rows, int64_t max_cands, bool with_tree 
     o = align_up(o + sizeof(RaceSummary) * (size_t)kRaceSlots * kMaxK, 256);
     L.off_tree_stats = o;
     if (with_tree) o = align_up(o + sizeof(TreeRowStat) * (size_t)max_rows, 256);
+    L.off_row_extra = o;
+    if (with_tree) o = align_up(o + 12 * (size_t)max_rows, 256);
+    L.full = with_tree;
     L.bytes = o;
     return L;
 }
@@ -250,9 +254,9 @@ int dispatch_align_stream(aasd_ctx* ctx, const StreamJob& sj, const AlignArgs& a
     return launch_align_stream<DT, 4, 0>(ctx, sj, a, grid);
 }
 
-template <int DT, int ND, bool TK, bool FIN = false>
+template <int DT, int ND, bool TK, bool FIN = false, int K = 1>
 int launch_verify_stream(aasd_ctx* ctx, const StreamJob& sj, const VerifyArgs& a, unsigned int grid) {
-    auto kernel = stream_kernel<DT, 1, ND, TK, FIN, VerifyEpilogue<DT>>;
+    auto kernel = stream_kernel<DT, K, ND, TK, FIN, VerifyEpilogue<DT>>;
     if (enable_stream_smem(kernel) != AASD_OK) return AASD_ERR_CUDA;
     launch(kernel, grid, kStreamThreads, kStreamSmemBytes, ctx->stream, sj, a);
     return AASD_OK;
@@ -260,6 +264,11 @@ int launch_verify_stream(aasd_ctx* ctx, const StreamJob& sj, const VerifyArgs& a
 
 template <int DT>
 int dispatch_verify_stream(aasd_ctx* ctx, const StreamJob& sj, const VerifyArgs& a, unsigned int grid) {
+    if (a.row_extra) {
+        // the table extension wants the two best tokens of every row
+        if (a.hints & AASD_HINT_FINITE) return launch_verify_stream<DT, 0, false, true, 2>(ctx, sj, a, grid);
+        return launch_verify_stream<DT, 0, false, false, 2>(ctx, sj, a, grid);
+    }
     if (a.mode == AASD_VERIFY_STRICT_SAMPLED) return launch_verify_stream<DT, 1, false>(ctx, sj, a, grid);
     if (a.mode == AASD_VERIFY_TOP_K) return launch_verify_stream<DT, 0, true>(ctx, sj, a, grid);
     if (a.hints & AASD_HINT_FINITE) return launch_verify_stream<DT, 0, false, true>(ctx, sj, a, grid);
@@ -505,6 +514,10 @@ int verify_impl(aasd_ctx* ctx, const void* target_logits, const int32_t* draft_i
         a.seq = *seq;
         a.seq.enabled = 1;
         a.seq.seq_tickets = reinterpret_cast<unsigned int*>(ws + L->off_seq_tickets);
+        if (seq->table_ids) {
+            if (!L->full || !(a.job.vector_ok && a.job.nvec > 0)) return AASD_ERR_UNSUPPORTED;
+            a.row_extra = reinterpret_cast<int32_t*>(ws + L->off_row_extra);
+        }
     }
     AASD_CUDA(cudaSetDevice(ctx->device));
     if (n_rows == 0) {
@@ -577,6 +590,12 @@ int aasd_step(aasd_ctx* ctx, const aasd_step_args* s, void* workspace, size_t wo
     const aasd_draft_params& dp = s->draft;
     if (!s->hist_ids || !s->hist_len || !s->best_cand || !s->n_emit || !s->emit_ids) return AASD_ERR_INVALID_ARG;
     if (!s->verify_out.accept_len || !s->verify_out.next_token) return AASD_ERR_INVALID_ARG;
+    if (s->flags & AASD_STEP_EXTEND_TABLE) {
+        if (!s->table_ids || !s->table_n || !s->draft_in.align_row_offsets) return AASD_ERR_INVALID_ARG;
+        if (dp.k_extra < 1 || dp.k_extra > 2) return AASD_ERR_UNSUPPORTED;
+        if (s->verify.mode != AASD_VERIFY_CONDITIONAL && s->verify.mode != AASD_VERIFY_STRICT_GREEDY)
+            return AASD_ERR_UNSUPPORTED;
+    }
     int err = AASD_OK;
     if (!(s->flags & AASD_STEP_REUSE_DRAFT)) {
         err = aasd_draft(ctx, &s->draft_in, &dp, &s->draft_out);
@@ -600,6 +619,12 @@ int aasd_step(aasd_ctx* ctx, const aasd_step_args* s, void* workspace, size_t wo
     tail.hist_ids = s->hist_ids;
     tail.hist_offsets = s->draft_in.hist_offsets;
     tail.hist_len = s->hist_len;
+    if (s->flags & AASD_STEP_EXTEND_TABLE) {
+        tail.table_ids = s->table_ids;
+        tail.table_n = s->table_n;
+        tail.table_row_offsets = s->draft_in.align_row_offsets;
+        tail.table_k = dp.k_extra;
+    }
     return verify_impl(ctx, s->target_logits, s->draft_out.draft_ids, s->draft_out.draft_flags, nullptr, n_cands,
                        n_rows, &vp, workspace, workspace_bytes, &s->verify_out, &tail);
 }

@@ -308,6 +308,11 @@ struct SeqTail {
     int32_t* hist_ids;
     const int32_t* hist_offsets;
     int32_t* hist_len;
+    // alignment sampling on generated context: table rows of the emitted tokens
+    int32_t* table_ids;                 // NULL: off
+    int32_t* table_n;
+    const int32_t* table_row_offsets;   // [n_seqs] table row of each sequence's first position
+    int table_k;                        // row width of table_ids
 };
 
 struct VerifyArgs {
@@ -322,6 +327,7 @@ struct VerifyArgs {
     unsigned int* cand_tickets;
     uint8_t* row_accept;           // scratch [n_rows]
     int32_t* row_own;              // scratch [n_rows]
+    int32_t* row_extra;            // scratch [n_rows x 3] or NULL: (count, two ids) ranked above the row's draft token
     SampleJob smp;                 // STRICT_SAMPLED: the row's own token is a keyed draw
     int top_k;                     // TOP_K mode
     unsigned int hints;            // AASD_HINT_*
@@ -403,6 +409,23 @@ __device__ void verify_row(const VerifyArgs& a, const RowJob& job, int64_t row, 
     if (a.out.sampled) a.out.sampled[row] = f.bad ? AASD_NONE : sampled;
     a.row_accept[row] = acc ? 1 : 0;
     a.row_own[row] = own;
+    if (a.row_extra) {
+        // Fig. 2's rule with the draft token in the place of the prompt's next token
+        int n = 0, ids[2] = {AASD_NONE, AASD_NONE};
+        if (d_ok && !f.bad) {
+            const int width = a.seq.table_k < 2 ? a.seq.table_k : 2;
+            for (int j = 0; j < width; ++j) {
+                const u64 k = merged.key[j];
+                if (k == 0) break;
+                const float xv = key_value(k);
+                const int id = key_id(k);
+                if (xv > xd || (xv == xd && id < d)) ids[n++] = id;
+            }
+        }
+        a.row_extra[row * 3 + 0] = n;
+        a.row_extra[row * 3 + 1] = ids[0];
+        a.row_extra[row * 3 + 2] = ids[1];
+    }
     tally.rows += 1;
     tally.bad += f.bad ? 1 : 0;
     tally.near += near ? 1 : 0;
@@ -509,6 +532,23 @@ __device__ void verify_finish_warp(const VerifyArgs& a, const RowJob& job, int64
         if (i < ne) tok = (i < best_a) ? a.draft_ids[(int64_t)best * a.rows_per_cand + i] : nt;
         e[i] = tok;
         if (i < ne && len + i < cap) a.seq.hist_ids[off + len + i] = tok;
+    }
+    if (a.seq.table_ids) {
+        // table rows of the emitted tokens: position len + i has row (first row) + len + i - 1
+        const int64_t row0 = (int64_t)a.seq.table_row_offsets[b] + len - 1;
+        const int K = a.seq.table_k;
+        for (int i = lane; i < ne; i += 32) {
+            if (len + i >= cap || len + i < 1) continue;
+            int n = 0, ids[2] = {AASD_NONE, AASD_NONE};
+            if (i < best_a) {
+                const int32_t* x = a.row_extra + ((int64_t)best * a.rows_per_cand + i) * 3;
+                n = __ldcg(x);
+                ids[0] = __ldcg(x + 1);
+                ids[1] = __ldcg(x + 2);
+            }
+            a.seq.table_n[row0 + i] = n;
+            for (int j = 0; j < K; ++j) a.seq.table_ids[(row0 + i) * K + j] = j < 2 ? ids[j] : AASD_NONE;
+        }
     }
     __syncwarp();
     if (lane == 0) {

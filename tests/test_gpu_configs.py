@@ -57,7 +57,7 @@ def _check_rows_against_oracle(x, ids, L, rows, got, dtype, mode, seed, tag, row
 
 
 def _run_config(index, n_follow, align_mode=binding.ALIGN_TOPK, verify_mode=binding.VERIFY_CONDITIONAL,
-                sample_rows=6):
+                sample_rows=6, extend=False):
     w = synth.workload(index)
     dev = torch.device("cuda", 0)
     ctx = binding.Context()
@@ -108,7 +108,7 @@ def _run_config(index, n_follow, align_mode=binding.ALIGN_TOPK, verify_mode=bind
     cap = w.steps * (w.draft_len + 1) + 8
     align = dict(align_ids=table_ids, n_extra=table_n)
     st = binding.DecodeState(ctx, prompts, cap, w.ngram, w.draft_len, w.max_cands, V, w.torch_dtype, align=align,
-                             alpha=ALPHA, beta=BETA, mode=verify_mode, seed=seed, top_k=5)
+                             alpha=ALPHA, beta=BETA, mode=verify_mode, seed=seed, top_k=5, extend_table=extend)
     hoffs_all = cpu(st.hist_offsets)
     F = n_follow
     hoffs = (hoffs_all[:F + 1] - hoffs_all[0]).astype(np.int32)
@@ -116,6 +116,16 @@ def _run_config(index, n_follow, align_mode=binding.ALIGN_TOPK, verify_mode=bind
     hlen = cpu(st.hist_len)[:F].copy()
     plen = hlen.copy()
     arow = np.arange(0, F * L, L, dtype=np.int32)
+    tab_ids, tab_n = ref_tab["align_ids"], ref_tab["n_extra"]
+    if extend:
+        # alignment sampling on generated context: the oracle's table has a row per history
+        # position too, and the drafts look extras up wherever the history holds a token
+        tab_ids = np.full((hoffs[-1], K_EXTRA), oracle.NONE, np.int32)
+        tab_n = np.zeros(hoffs[-1], np.int32)
+        for b in range(F):
+            tab_ids[hoffs[b]:hoffs[b] + L] = ref_tab["align_ids"][b * L:(b + 1) * L]
+            tab_n[hoffs[b]:hoffs[b] + L] = ref_tab["n_extra"][b * L:(b + 1) * L]
+        arow = hoffs[:-1].copy()
     rows_per_seq = w.max_cands * w.draft_len
     RF = F * rows_per_seq
     coffs = np.arange(0, RF + 1, w.draft_len, dtype=np.int32)
@@ -129,9 +139,8 @@ def _run_config(index, n_follow, align_mode=binding.ALIGN_TOPK, verify_mode=bind
             rl = min(w.ngram, hlen[b])
             recent[b, :rl] = hist[hoffs[b] + hlen[b] - rl: hoffs[b] + hlen[b]]
             rlen[b] = rl
-        dr = oracle.draft(hist, hoffs, hlen, plen, recent, rlen, w.ngram, w.draft_len, w.max_cands,
-                          align_ids=ref_tab["align_ids"], align_n=ref_tab["n_extra"], align_row_offsets=arow,
-                          k_extra=K_EXTRA)
+        dr = oracle.draft(hist, hoffs, hlen, hlen if extend else plen, recent, rlen, w.ngram, w.draft_len,
+                          w.max_cands, align_ids=tab_ids, align_n=tab_n, align_row_offsets=arow, k_extra=K_EXTRA)
         dg = st.run_draft()
         check_draft({k: v[:F] for k, v in dg.items()}, dr)
         d_all = dg["draft_ids"].reshape(-1).to(torch.int64)
@@ -145,7 +154,11 @@ def _run_config(index, n_follow, align_mode=binding.ALIGN_TOPK, verify_mode=bind
                             seed=seed, step=s, threads=THREADS, top_k=5)
         sel = oracle.select(ref["accept_len"], ref["next_token"], dr["draft_ids"].reshape(-1), coffs, soffs,
                             w.draft_len + 1)
+        before = hlen.copy()
         oracle.append(hist, hoffs, hlen, sel["emit_ids"], sel["n_emit"])
+        if extend:
+            oracle.extend_table(to_oracle(x[:RF]), coffs, ref["accept_len"], sel["best_cand"], sel["emit_ids"],
+                                sel["n_emit"], hoffs, before, tab_ids, tab_n, arow)
         got = {k: (v[:RF] if v.shape[0] == st.rows else v[:F * w.max_cands]) for k, v in st.verify_out.items()}
         near = check_verify(got, ref, coffs, w.torch_dtype)
         near_total += near
@@ -154,6 +167,9 @@ def _run_config(index, n_follow, align_mode=binding.ALIGN_TOPK, verify_mode=bind
             assert np.array_equal(cpu(st.emit_ids[:F]), sel["emit_ids"])
             assert np.array_equal(cpu(st.hist_len[:F]), hlen)
             assert np.array_equal(cpu(st.hist_ids)[:hoffs_all[F]], hist)
+            if extend:
+                assert np.array_equal(cpu(st.align["n_extra"])[:hoffs_all[F]], tab_n)
+                assert np.array_equal(cpu(st.align["align_ids"])[:hoffs_all[F]], tab_ids)
         emitted += int(sel["n_emit"].sum())
         if near:
             # a decision inside the 1e-6 band may legitimately differ, after which the two
@@ -212,4 +228,10 @@ def test_config4_long_context_16k():
 
 def test_config5_serving_batch256():
     r = _run_config(4, 4)
+    assert r["counters"]["rows"] >= 64 * 4096
+
+
+def test_config5_with_table_extension():
+    # the serving batch with alignment sampling on generated context switched on
+    r = _run_config(4, 4, extend=True)
     assert r["counters"]["rows"] >= 64 * 4096
