@@ -95,20 +95,33 @@ namespace {
 // Every kernel of the library is launched with programmatic stream serialization: it may be
 // scheduled while its predecessor in the stream drains, and waits (griddepcontrol.wait,
 // first thing in each kernel) for that predecessor to complete before it touches memory.
+// cluster > 1: the grid is made of thread-block clusters of that many CTAs.
 template <class... Params, class... Args>
-void launch(void (*kernel)(Params...), unsigned int grid, unsigned int block, size_t smem, cudaStream_t stream,
-            Args&&... args) {
+void launch_clustered(void (*kernel)(Params...), unsigned int grid, unsigned int block, size_t smem,
+                      cudaStream_t stream, unsigned int cluster, Args&&... args) {
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(grid, 1, 1);
     cfg.blockDim = dim3(block, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
     cfg.numAttrs = 1;
+    if (cluster > 1) {
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = cluster;
+        attr[1].val.clusterDim.y = 1;
+        attr[1].val.clusterDim.z = 1;
+        cfg.numAttrs = 2;
+    }
+    cfg.attrs = attr;
     cudaLaunchKernelEx(&cfg, kernel, Params(args)...);   // errors surface in cudaGetLastError
+}
+template <class... Params, class... Args>
+void launch(void (*kernel)(Params...), unsigned int grid, unsigned int block, size_t smem, cudaStream_t stream,
+            Args&&... args) {
+    launch_clustered(kernel, grid, block, smem, stream, 1u, static_cast<Args&&>(args)...);
 }
 
 int after_launch(aasd_ctx* ctx, int n) {
@@ -216,6 +229,13 @@ void plan_stream(aasd_ctx* ctx, StreamJob& sj, const RowJob& job, const int32_t*
     sj.tail_chunks = (int)chunks;
     sj.n_items = (job.n_rows - tail_rows) + tail_rows * chunks;
     *grid = (unsigned int)(sj.n_items < slots ? sj.n_items : slots);
+    // Few rows, every row cut, one CTA per piece: the pieces of a row form a thread-block
+    // cluster and meet in its first CTA's shared memory.  (The sampler's per-piece records
+    // travel through global memory, so sampling launches stay as they are.)
+    sj.cluster_pieces = (chunks > 1 && chunks <= kMaxCluster && tail_rows == job.n_rows && smp == nullptr &&
+                         (int64_t)*grid == sj.n_items && getenv("AASD_NO_CLUSTER") == nullptr)
+                            ? 1
+                            : 0;
 }
 
 template <class Kernel>
@@ -230,7 +250,8 @@ template <int DT, int K, int ND, bool FIN = false>
 int launch_align_stream(aasd_ctx* ctx, const StreamJob& sj, const AlignArgs& a, unsigned int grid) {
     auto kernel = stream_kernel<DT, K, ND, false, FIN, AlignEpilogue<DT>>;
     if (enable_stream_smem(kernel) != AASD_OK) return AASD_ERR_CUDA;
-    launch(kernel, grid, kStreamThreads, kStreamSmemBytes, ctx->stream, sj, a);
+    launch_clustered(kernel, grid, kStreamThreads, kStreamSmemBytes, ctx->stream,
+                     sj.cluster_pieces ? (unsigned int)sj.tail_chunks : 1u, sj, a);
     return AASD_OK;
 }
 
@@ -258,7 +279,8 @@ template <int DT, int ND, bool TK, bool FIN = false, int K = 1>
 int launch_verify_stream(aasd_ctx* ctx, const StreamJob& sj, const VerifyArgs& a, unsigned int grid) {
     auto kernel = stream_kernel<DT, K, ND, TK, FIN, VerifyEpilogue<DT>>;
     if (enable_stream_smem(kernel) != AASD_OK) return AASD_ERR_CUDA;
-    launch(kernel, grid, kStreamThreads, kStreamSmemBytes, ctx->stream, sj, a);
+    launch_clustered(kernel, grid, kStreamThreads, kStreamSmemBytes, ctx->stream,
+                     sj.cluster_pieces ? (unsigned int)sj.tail_chunks : 1u, sj, a);
     return AASD_OK;
 }
 
@@ -649,7 +671,8 @@ template <int DT, int ND>
 int launch_tree_stream(aasd_ctx* ctx, const StreamJob& sj, const TreeArgs& a, unsigned int grid) {
     auto kernel = stream_kernel<DT, 1, ND, false, false, TreeEpilogue<DT>>;
     if (enable_stream_smem(kernel) != AASD_OK) return AASD_ERR_CUDA;
-    launch(kernel, grid, kStreamThreads, kStreamSmemBytes, ctx->stream, sj, a);
+    launch_clustered(kernel, grid, kStreamThreads, kStreamSmemBytes, ctx->stream,
+                     sj.cluster_pieces ? (unsigned int)sj.tail_chunks : 1u, sj, a);
     return AASD_OK;
 }
 

@@ -66,6 +66,42 @@ __device__ __forceinline__ bool mbar_wait(u64* bar, unsigned int parity, volatil
     }
     return false;
 }
+// ---- thread-block clusters: the pieces of a row meet in the shared memory of the cluster's
+// first CTA instead of global memory ------------------------------------------------------
+__device__ __forceinline__ void cluster_sync_all() {
+    __syncwarp();
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// address of the same shared-memory object in CTA `rank` of the cluster
+__device__ __forceinline__ unsigned int cluster_map(const void* p, unsigned int rank) {
+    unsigned int r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_u32(p)), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_store_u64(unsigned int addr, u64 v) {
+    asm volatile("st.shared::cluster.u64 [%0], %1;" ::"r"(addr), "l"(v) : "memory");
+}
+__device__ __forceinline__ void cluster_mbar_arrive(unsigned int addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(addr) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(u64* bar, unsigned int parity) {
+    unsigned int ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_cluster(u64* bar, unsigned int parity, volatile int* abort_flag) {
+    for (unsigned int it = 0; it < kWaitLimit; ++it) {
+        if (mbar_try_wait_cluster(bar, parity)) return true;
+        if ((it & 255u) == 255u && *abort_flag) return false;
+    }
+    return false;
+}
 __device__ __forceinline__ void give_up(volatile int* abort_flag, DeviceState* state) {
     *abort_flag = 1;
     atomicOr(&state->status, AASD_STATUS_TIMEOUT);
@@ -94,6 +130,7 @@ struct ItemInfo {
     int chunk;        // which piece of the row
 };
 constexpr int kNoItem = -1;
+constexpr int kMaxCluster = 8;   // portable cluster size
 struct WarpPartial {
     double S, A;
     u64 key[kMaxK];   // vector-level: (ordered vector maximum << 32) | ~vector index
@@ -109,6 +146,10 @@ struct StreamShared {
     RaceSummary race[kSlots][kConsumerWarps][kMaxK];   // sampling kernels only
     unsigned short max_tile[kSlots][kConsumerWarps][32];   // tile (within the item) where a lane met its maximum
     int abort_flag;
+    // cluster launches: the pieces of the cluster's row, written by the other CTAs of the
+    // cluster into the first CTA's copy, and the barrier they arrive on
+    RowPartial cluster_piece[kMaxCluster];
+    u64 cluster_bar;
 };
 constexpr size_t kStreamSmemBytes = (size_t)kStages * kTileBytes + sizeof(StreamShared) + 128;
 
@@ -120,6 +161,8 @@ struct StreamJob {
     int whole_rows;           // rows [0, whole_rows) are one item each
     int tail_chunks;          // every later row is cut into this many pieces
     long long n_items;        // whole_rows + (n_rows - whole_rows) * tail_chunks
+    int cluster_pieces;       // the launch is made of clusters of tail_chunks CTAs, one per row, every
+                              // row is cut (whole_rows == 0) and the grid has one CTA per piece
     // sampling kernels only
     SampleJob smp;
     RaceSummary* race_partials;   // [slots x kMaxK] beside the partial records of cut rows
@@ -481,8 +524,11 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
             mbar_init(&sh.freeb[p], 1);
         }
         sh.abort_flag = 0;
+        mbar_init(&sh.cluster_bar, job.cluster_pieces ? (unsigned int)job.tail_chunks - 1u : 1u);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    // nobody may signal a barrier of another CTA before that CTA has set it up
+    if (job.cluster_pieces) cluster_sync_all();
     pdl_launch_dependents();
     __syncthreads();
     pdl_wait();   // everything above overlapped the end of the preceding kernel
@@ -867,7 +913,63 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
                 }
             }
         }
-        if (chunks > 1) {
+        if (chunks > 1 && job.cluster_pieces) {
+            // The pieces of the row are the CTAs of this cluster (rank = piece): the others
+            // write their records into the first CTA's shared memory and signal its barrier;
+            // the first CTA waits for them and carries on.  No trip through global memory.
+            if (chunk != 0) {
+                if (lane == 0) {
+                    const unsigned int dst = cluster_map(&sh.cluster_piece[chunk], 0);
+                    cluster_store_u64(dst + (unsigned int)offsetof(RowPartial, S), (u64)__double_as_longlong(S));
+                    cluster_store_u64(dst + (unsigned int)offsetof(RowPartial, A), (u64)__double_as_longlong(A));
+#pragma unroll
+                    for (int j = 0; j < kMaxK; ++j)
+                        cluster_store_u64(dst + (unsigned int)(offsetof(RowPartial, key) + 8 * j), j < K ? mk[j] : 0ull);
+                    cluster_store_u64(dst + (unsigned int)offsetof(RowPartial, ahead), (u64)n_ahead);
+                    cluster_mbar_arrive(cluster_map(&sh.cluster_bar, 0));
+                }
+                continue;
+            }
+            if (lane == 0) {
+                RowPartial& mine = sh.cluster_piece[0];
+                mine.S = S;
+                mine.A = A;
+#pragma unroll
+                for (int j = 0; j < kMaxK; ++j) mine.key[j] = j < K ? mk[j] : 0ull;
+                mine.ahead = n_ahead;
+            }
+            if (!mbar_wait_cluster(&sh.cluster_bar, 0u, abort_flag)) {
+                if (lane == 0) give_up(abort_flag, rj.state);
+                break;
+            }
+            __syncwarp();
+            S = 0.0;
+            A = 0.0;
+            n_ahead = 0;
+#pragma unroll
+            for (int j = 0; j < K; ++j) vk[j] = 0;
+            if (lane < chunks) {
+                const RowPartial& q = sh.cluster_piece[lane];
+                S = q.S;
+                A = q.A;
+                if (TK) n_ahead = q.ahead;
+#pragma unroll
+                for (int j = 0; j < K; ++j) key_insert<K>(vk, q.key[j]);
+            }
+            S = warp_sum_f64(S);
+            A = warp_sum_f64(A);
+            if (TK) n_ahead = warp_sum_i64(n_ahead);
+#pragma unroll
+            for (int r = 0; r < K; ++r) {
+                const u64 m = warp_max_u64(vk[0]);
+                mk[r] = m;
+                if (m != 0 && vk[0] == m) {
+#pragma unroll
+                    for (int j = 0; j + 1 < K; ++j) vk[j] = vk[j + 1];
+                    vk[K - 1] = 0;
+                }
+            }
+        } else if (chunks > 1) {
             // pieces of a row meet in global memory; the last one to arrive carries on
             RowPartial* slots = rj.partials + (row - job.whole_rows) * chunks;
             int last = 0;
