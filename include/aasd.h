@@ -402,7 +402,7 @@ int aasd_probe_read(aasd_ctx* ctx, const void* buffer, size_t bytes, uint32_t* s
  * aasd_verify needs a context (aasd_create allocates its status block) and a caller-made
  * workspace; this entry point needs neither.  Its scratch - what the workspace and the
  * context's status block would hold - lives in a fixed block of device memory that is part
- * of the library image: about 0.75 MB on every GPU that loads the library, held until the
+ * of the library image: about 0.8 MB on every GPU that loads the library, held until the
  * process exits.  The call itself makes no cudaMalloc / cudaFree and calls nothing that
  * allocates.
  *

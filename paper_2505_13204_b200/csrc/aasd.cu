@@ -59,7 +59,7 @@ WorkspaceLayout make_layout(int64_t max_rows, int64_t max_cands, bool with_tree 
     L.off_row_accept = o;
     o = align_up(o + (size_t)max_rows, 256);
     L.off_row_own = o;
-    o = align_up(o + 4 * (size_t)max_rows, 256);
+    o = align_up(o + 8 * (size_t)max_rows, 256);
     L.off_next = o;
     o = align_up(o + 4 * (size_t)max_rows, 256);
     L.off_race = o;
@@ -528,8 +528,7 @@ int verify_impl(aasd_ctx* ctx, const void* target_logits, const int32_t* draft_i
     a.top_k = p->top_k;
     a.hints = p->hints;
     a.cand_tickets = reinterpret_cast<unsigned int*>(ws + L->off_cand_tickets);
-    a.row_accept = reinterpret_cast<uint8_t*>(ws + L->off_row_accept);
-    a.row_own = reinterpret_cast<int32_t*>(ws + L->off_row_own);
+    a.row_state = reinterpret_cast<u64*>(ws + L->off_row_own);
     a.smp = make_sample_job(p->seed, p->step, false, p->inv_temperature);
     a.out = *out;
     if (seq) {
@@ -779,7 +778,8 @@ constexpr size_t kStaticWorkspaceBytes =
     2 * ((4 * (size_t)kStaticMaxCands + 255) / 256 * 256) +              // candidate and sequence tickets
     256 +                                                                // work-item counters
     (((size_t)kStaticMaxRows + 255) / 256 * 256) +                       // accept bits
-    2 * ((4 * (size_t)kStaticMaxRows + 255) / 256 * 256) +               // own tokens, next ids
+    ((8 * (size_t)kStaticMaxRows + 255) / 256 * 256) +                   // row states (own token, accept bit)
+    ((4 * (size_t)kStaticMaxRows + 255) / 256 * 256) +                   // next ids
     ((sizeof(RaceSummary) * (size_t)kRaceSlots * kMaxK + 255) / 256 * 256);   // sampler records of cut rows
 constexpr size_t kStaticBytes = kStaticWorkspaceBytes + 256;
 
@@ -864,8 +864,7 @@ extern "C" int aasd_verify_static(int device, void* stream, const void* target_l
     a.top_k = p->top_k;
     a.hints = p->hints;
     a.cand_tickets = reinterpret_cast<unsigned int*>(ws + L.off_cand_tickets);
-    a.row_accept = reinterpret_cast<uint8_t*>(ws + L.off_row_accept);
-    a.row_own = reinterpret_cast<int32_t*>(ws + L.off_row_own);
+    a.row_state = reinterpret_cast<u64*>(ws + L.off_row_own);
     a.smp = make_sample_job(p->seed, p->step, false, p->inv_temperature);
     a.out = *out;
     if (n_rows == 0) {

@@ -325,8 +325,7 @@ struct VerifyArgs {
     float alpha, beta;
     int mode;
     unsigned int* cand_tickets;
-    uint8_t* row_accept;           // scratch [n_rows]
-    int32_t* row_own;              // scratch [n_rows]
+    u64* row_state;                // scratch [n_rows]: the row's own token << 32 | its accept bit
     int32_t* row_extra;            // scratch [n_rows x 3] or NULL: (count, two ids) ranked above the row's draft token
     SampleJob smp;                 // STRICT_SAMPLED: the row's own token is a keyed draw
     int top_k;                     // TOP_K mode
@@ -372,9 +371,14 @@ struct Tally {
 // draft id as given, xd its raw logit (read only when d lies inside the vocabulary), sampled
 // the row's keyed draw in STRICT_SAMPLED mode (NONE otherwise, and on a bad row).  In TOP_K
 // mode merged.ahead is the number of tokens ahead of d in the order (logit desc, id asc).
+// What the prefix rule needs of the row goes out first and the row's ticket (the counter of
+// its candidate) is taken right behind it, so that the stores of the row's outputs, which
+// nobody inside the launch reads, are under way while the ticket travels.  Returns the
+// ticket's value.
 template <int DT>
-__device__ void verify_row(const VerifyArgs& a, const RowJob& job, int64_t row, const RowPartial& merged,
-                           float neg_refc, bool centered, int d, float xd, int sampled, Tally& tally) {
+__device__ unsigned int verify_row(const VerifyArgs& a, const RowJob& job, int64_t row, const RowPartial& merged,
+                                   float neg_refc, bool centered, int d, float xd, int sampled, unsigned int* ticket,
+                                   Tally& tally) {
     const bool d_ok = d >= 0 && d < job.vocab;
     const RowFinal f = finish_row(merged, job.c1, neg_refc, centered);
     const unsigned int flag = a.draft_flags ? a.draft_flags[row] : AASD_FLAG_CONDITIONAL;
@@ -397,18 +401,7 @@ __device__ void verify_row(const VerifyArgs& a, const RowJob& job, int64_t row, 
             acc = (d == own);
         }
     }
-    if (a.out.n_greater)
-        a.out.n_greater[row] = (a.mode == AASD_VERIFY_TOP_K && d_ok && !f.bad && xd > -CUDART_INF_F)
-                                   ? (int)merged.ahead : AASD_NONE;
-    if (a.out.p_draft) a.out.p_draft[row] = (float)pd;
-    if (a.out.entropy) a.out.entropy[row] = (float)f.H;
-    if (a.out.pmax) a.out.pmax[row] = (float)f.pmax;
-    if (a.out.argmax) a.out.argmax[row] = f.top1;
-    if (a.out.threshold) a.out.threshold[row] = (float)thr;
-    if (a.out.accept) a.out.accept[row] = acc ? 1 : 0;
-    if (a.out.sampled) a.out.sampled[row] = f.bad ? AASD_NONE : sampled;
-    a.row_accept[row] = acc ? 1 : 0;
-    a.row_own[row] = own;
+    a.row_state[row] = ((u64)(unsigned int)own << 32) | (acc ? 1ull : 0ull);
     if (a.row_extra) {
         // Fig. 2's rule with the draft token in the place of the prompt's next token
         int n = 0, ids[2] = {AASD_NONE, AASD_NONE};
@@ -426,10 +419,23 @@ __device__ void verify_row(const VerifyArgs& a, const RowJob& job, int64_t row, 
         a.row_extra[row * 3 + 1] = ids[0];
         a.row_extra[row * 3 + 2] = ids[1];
     }
+    __threadfence();
+    const unsigned int t = atomicAdd(ticket, 1u);
+    if (a.out.n_greater)
+        a.out.n_greater[row] = (a.mode == AASD_VERIFY_TOP_K && d_ok && !f.bad && xd > -CUDART_INF_F)
+                                   ? (int)merged.ahead : AASD_NONE;
+    if (a.out.p_draft) a.out.p_draft[row] = (float)pd;
+    if (a.out.entropy) a.out.entropy[row] = (float)f.H;
+    if (a.out.pmax) a.out.pmax[row] = (float)f.pmax;
+    if (a.out.argmax) a.out.argmax[row] = f.top1;
+    if (a.out.threshold) a.out.threshold[row] = (float)thr;
+    if (a.out.accept) a.out.accept[row] = acc ? 1 : 0;
+    if (a.out.sampled) a.out.sampled[row] = f.bad ? AASD_NONE : sampled;
     tally.rows += 1;
     tally.bad += f.bad ? 1 : 0;
     tally.near += near ? 1 : 0;
     tally.accepted += acc ? 1 : 0;
+    return t;
 }
 
 // Candidate of a row and its row range; results of the empty candidates next to it (they
@@ -462,10 +468,9 @@ __device__ void verify_finish_warp(const VerifyArgs& a, const RowJob& job, int64
     int c = 0, last = 0;
     int64_t lo = 0, hi = 0;
     if (lane == 0) {
-        verify_row<DT>(a, job, row, merged, neg_refc, centered, d, xd, sampled, tally);
         c = candidate_of_row(a, job.n_rows, row, lo, hi);
-        __threadfence();
-        const unsigned int t = atomicAdd(&a.cand_tickets[c], 1u);
+        const unsigned int t = verify_row<DT>(a, job, row, merged, neg_refc, centered, d, xd, sampled,
+                                              &a.cand_tickets[c], tally);
         last = (t == (unsigned int)(hi - lo) - 1u);
         if (last) a.cand_tickets[c] = 0;
     }
@@ -476,18 +481,21 @@ __device__ void verify_finish_warp(const VerifyArgs& a, const RowJob& job, int64
     hi = __shfl_sync(0xFFFFFFFFu, hi, 0);
     __threadfence();
     int64_t n = hi - lo;   // leading accepted rows
+    int next = AASD_NONE;  // the own token of the first row that does not pass
     for (int64_t base = lo; base < hi; base += 32) {
         const int64_t r = base + lane;
-        const bool stop = r < hi && __ldcg(a.row_accept + r) == 0;
-        const unsigned int bal = __ballot_sync(0xFFFFFFFFu, stop);
+        const u64 st = r < hi ? __ldcg(a.row_state + r) : 1ull;
+        const unsigned int bal = __ballot_sync(0xFFFFFFFFu, (st & 1ull) == 0);
         if (bal) {
-            n = base - lo + (__ffs(bal) - 1);
+            const int first = __ffs(bal) - 1;
+            n = base - lo + first;
+            next = (int)(unsigned int)(__shfl_sync(0xFFFFFFFFu, st, first) >> 32);
             break;
         }
     }
     if (lane == 0) {
         if (a.out.accept_len) a.out.accept_len[c] = (int)n;
-        if (a.out.next_token) a.out.next_token[c] = (lo + n < hi) ? __ldcg(a.row_own + lo + n) : AASD_NONE;
+        if (a.out.next_token) a.out.next_token[c] = next;
     }
     if (!a.seq.enabled) return;
 
