@@ -353,3 +353,38 @@ def test_host_side_errors(ctx):
                              torch.tensor([0, 4], dtype=torch.int32, device="cuda").data_ptr(), 1, 4,
                              C.byref(prm), junk.data_ptr(), junk.numel(), C.byref(out))
     assert rc == 1
+
+
+@pytest.mark.parametrize("V,dtype,rows", [(32000, torch.float32, 8), (128256, torch.bfloat16, 12),
+                                          (152064, torch.bfloat16, 3), (70000, torch.bfloat16, 50),
+                                          (20000, torch.float32, 147)])
+def test_cluster_and_global_combine_agree(ctx, V, dtype, rows, monkeypatch):
+    """Scarce rows are cut into pieces; the pieces meet in a cluster's shared memory, or, with
+    the switch set, in global memory.  Both give the oracle's results and each other's bytes,
+    in verification (with the top-k count) and in alignment sampling."""
+    rng = np.random.default_rng(V + rows)
+    d = rng.integers(0, V, rows).astype(np.int32)
+    x = _make_logits(rows, V, dtype, 7 + V, torch.as_tensor(d, dtype=torch.int64))
+    offs = np.arange(0, rows + 1, 1, dtype=np.int32)
+    alpha, beta = F32(0.1), F32(0.05)
+    xd, dd, od = x.cuda(), torch.as_tensor(d).cuda(), torch.as_tensor(offs).cuda()
+    seq = np.array([0, rows], np.int32)
+    results = []
+    for no_cluster in (False, True):
+        if no_cluster:
+            monkeypatch.setenv("AASD_NO_CLUSTER", "1")
+        else:
+            monkeypatch.delenv("AASD_NO_CLUSTER", raising=False)
+        v = ctx.verify(xd, dd, od, alpha=alpha, beta=beta)
+        t = ctx.verify(xd, dd, od, mode=binding.VERIFY_TOP_K, top_k=3)
+        a = ctx.align_sample(xd, dd, seq, k_extra=2)
+        results.append({**{"v_" + k: w.clone() for k, w in v.items() if w is not None},
+                        "t_n_greater": t["n_greater"].clone(), "t_accept": t["accept"].clone(),
+                        **{"a_" + k: w.clone() for k, w in a.items() if w is not None}})
+        check_verify(v, oracle.verify(to_oracle(x), d, offs, alpha=alpha, beta=beta), offs, dtype)
+        rt = oracle.verify(to_oracle(x), d, offs, mode=binding.VERIFY_TOP_K, top_k=3)
+        assert np.array_equal(cpu(t["n_greater"]), rt["n_greater"])
+        check_align(a, oracle.align_sample(to_oracle(x), d, seq, k_extra=2), dtype)
+    for k in results[0]:
+        assert torch.equal(results[0][k], results[1][k]), k
+    assert ctx.poll_status() == 0
