@@ -129,3 +129,36 @@ def test_random_case(ctx, case):
         check_align(got, ref, dtype)
     st = ctx.poll_status()
     assert not (st & ~(binding.STATUS_BAD_ROW | binding.STATUS_ID_RANGE))
+
+
+@pytest.mark.parametrize("case", range(150))
+def test_random_draft_case(ctx, case):
+    """Drafting over random histories, keys, table widths and limits."""
+    from test_gpu_tokens import _dev as dev_i32, _draft_case
+    from parity import check_draft
+    rng = np.random.default_rng(70_000 + case)
+    B = int(rng.integers(1, 20))
+    n = int(rng.integers(1, 17))
+    draft_len = int(rng.integers(1, 17))
+    max_cands = int(rng.choice([1, 2, 3, 4, 6, 8, 16, 33, 64]))
+    K = int(rng.integers(1, 5))
+    alphabet = int(rng.choice([2, 3, 5, 11, 100]))
+    max_len = int(rng.choice([4, 40, 400, 2500]))
+    with_align = rng.random() < 0.7
+    match_align = with_align and rng.random() < 0.4
+    own_tail = rng.random() < 0.6
+    c = _draft_case(rng, B, alphabet, max_len, K, with_align, n, own_tail)
+    ref = oracle.draft(c["hist"], c["offs"], c["lens"], c["plens"], c["recent"], c["rlen"], n, draft_len, max_cands,
+                       align_ids=c["align_ids"], align_n=c["align_n"],
+                       align_row_offsets=None if c["arow"] is None else c["arow"][:-1],
+                       k_extra=K if with_align else 0, match_align=match_align)
+    kw = {}
+    if with_align:
+        kw = dict(align_ids=dev_i32(c["align_ids"]), align_n=dev_i32(c["align_n"]),
+                  align_row_offsets=dev_i32(c["arow"][:-1]))
+    use_tail = own_tail and rng.random() < 0.5      # key taken from the history itself
+    got = ctx.draft(dev_i32(c["hist"]), dev_i32(c["offs"]), dev_i32(c["lens"]), dev_i32(c["plens"]), n, draft_len,
+                    max_cands, recent_ids=None if use_tail else dev_i32(c["recent"]),
+                    recent_len=None if use_tail else dev_i32(c["rlen"]), match_align=match_align, **kw)
+    check_draft(got, ref)
+    assert ctx.poll_status() == 0
