@@ -72,6 +72,12 @@ __device__ __forceinline__ void cluster_sync_all() {
     __syncwarp();
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
+// Taken by every thread of a cluster launch on its way out: no CTA of the cluster leaves
+// (and gives its shared memory back) while another one may still write into it, whatever
+// path, a timed-out wait included, brought the threads here.
+__device__ __forceinline__ void cluster_exit_sync() {
+    asm volatile("barrier.cluster.arrive.release;\n\tbarrier.cluster.wait.acquire;" ::: "memory");
+}
 // address of the same shared-memory object in CTA `rank` of the cluster
 __device__ __forceinline__ unsigned int cluster_map(const void* p, unsigned int rank) {
     unsigned int r;
@@ -725,6 +731,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
                 mbar_arrive(&sh.done[p]);
             }
         }
+        if (job.cluster_pieces) cluster_exit_sync();
         return;
     }
 
@@ -812,6 +819,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
                 }
             }
         }
+        if (job.cluster_pieces) cluster_exit_sync();
         return;
     }
 
@@ -1121,6 +1129,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
         E::template finish<ND>(args, rj, row, rowp, fr, info, races, tail_group, tally);
     }
     if (lane == 0) tally.flush(rj.state);
+    if (job.cluster_pieces) cluster_exit_sync();
 }
 
 // Epilogues are entered by the whole finisher warp.
