@@ -246,13 +246,32 @@ int enable_stream_smem(Kernel kernel) {
                : AASD_ERR_CUDA;
 }
 
+// One launch of the streaming kernel.  Rows that stream faster than a finisher gets through
+// one (short_rows) take the variant with three finisher warps; sampling kernels, whose
+// consumers are the slower side, always run with one.
+template <int DT, int K, int ND, bool TK, bool FIN, class E>
+int launch_stream(aasd_ctx* ctx, const StreamJob& sj, const typename E::Args& a, unsigned int grid, bool short_rows) {
+    const unsigned int cluster = sj.cluster_pieces ? (unsigned int)sj.tail_chunks : 1u;
+    if (ND == 0 && short_rows) {
+        auto kernel = stream_kernel<DT, K, ND, TK, FIN, E, (ND == 0 ? kShortRowFinishers : 1)>;
+        if (enable_stream_smem(kernel) != AASD_OK) return AASD_ERR_CUDA;
+        launch_clustered(kernel, grid, stream_threads(kShortRowFinishers), kStreamSmemBytes, ctx->stream, cluster, sj, a);
+        return AASD_OK;
+    }
+    auto kernel = stream_kernel<DT, K, ND, TK, FIN, E, 1>;
+    if (enable_stream_smem(kernel) != AASD_OK) return AASD_ERR_CUDA;
+    launch_clustered(kernel, grid, stream_threads(1), kStreamSmemBytes, ctx->stream, cluster, sj, a);
+    return AASD_OK;
+}
+// bytes of a row below which the finisher, not the copy, paces a CTA (measured: a verification
+// row costs a finisher about 7 us under load, an alignment row 5 us; a CTA streams 25 GB/s)
+constexpr int64_t kShortVerifyRow = 200 * 1024;
+constexpr int64_t kShortAlignRow = 96 * 1024;
+inline int64_t row_bytes_of(const StreamJob& sj) { return (int64_t)sj.row.nvec * 16; }
+
 template <int DT, int K, int ND, bool FIN = false>
 int launch_align_stream(aasd_ctx* ctx, const StreamJob& sj, const AlignArgs& a, unsigned int grid) {
-    auto kernel = stream_kernel<DT, K, ND, false, FIN, AlignEpilogue<DT>>;
-    if (enable_stream_smem(kernel) != AASD_OK) return AASD_ERR_CUDA;
-    launch_clustered(kernel, grid, kStreamThreads, kStreamSmemBytes, ctx->stream,
-                     sj.cluster_pieces ? (unsigned int)sj.tail_chunks : 1u, sj, a);
-    return AASD_OK;
+    return launch_stream<DT, K, ND, false, FIN, AlignEpilogue<DT>>(ctx, sj, a, grid, row_bytes_of(sj) < kShortAlignRow);
 }
 
 // TOPK mode keeps the K best tokens and draws nothing; GUMBEL mode needs the best token
@@ -277,11 +296,7 @@ int dispatch_align_stream(aasd_ctx* ctx, const StreamJob& sj, const AlignArgs& a
 
 template <int DT, int ND, bool TK, bool FIN = false, int K = 1>
 int launch_verify_stream(aasd_ctx* ctx, const StreamJob& sj, const VerifyArgs& a, unsigned int grid) {
-    auto kernel = stream_kernel<DT, K, ND, TK, FIN, VerifyEpilogue<DT>>;
-    if (enable_stream_smem(kernel) != AASD_OK) return AASD_ERR_CUDA;
-    launch_clustered(kernel, grid, kStreamThreads, kStreamSmemBytes, ctx->stream,
-                     sj.cluster_pieces ? (unsigned int)sj.tail_chunks : 1u, sj, a);
-    return AASD_OK;
+    return launch_stream<DT, K, ND, TK, FIN, VerifyEpilogue<DT>>(ctx, sj, a, grid, row_bytes_of(sj) < kShortVerifyRow);
 }
 
 template <int DT>
@@ -668,11 +683,7 @@ namespace {
 
 template <int DT, int ND>
 int launch_tree_stream(aasd_ctx* ctx, const StreamJob& sj, const TreeArgs& a, unsigned int grid) {
-    auto kernel = stream_kernel<DT, 1, ND, false, false, TreeEpilogue<DT>>;
-    if (enable_stream_smem(kernel) != AASD_OK) return AASD_ERR_CUDA;
-    launch_clustered(kernel, grid, kStreamThreads, kStreamSmemBytes, ctx->stream,
-                     sj.cluster_pieces ? (unsigned int)sj.tail_chunks : 1u, sj, a);
-    return AASD_OK;
+    return launch_stream<DT, 1, ND, false, false, TreeEpilogue<DT>>(ctx, sj, a, grid, false);
 }
 
 template <int DT>

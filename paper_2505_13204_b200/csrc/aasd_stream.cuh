@@ -28,7 +28,9 @@ constexpr int kTileBytes = 32768;
 constexpr int kStages = 3;
 constexpr int kConsumerWarps = 8;
 constexpr int kConsumers = kConsumerWarps * 32;
-constexpr int kStreamThreads = kConsumers + 64;   // + producer warp + finisher warp
+// consumers + producer warp + NF finisher warps (item seq goes to finisher seq % NF)
+constexpr int stream_threads(int nf) { return kConsumers + 32 + 32 * nf; }
+constexpr int kShortRowFinishers = 3;
 constexpr int kRing = 16;
 constexpr int kSlots = 4;                         // item results in flight between consumers and finisher
 constexpr unsigned int kWaitLimit = 1u << 24;     // polls of try_wait before giving up
@@ -507,8 +509,12 @@ struct FinishedRow {
 //   TK: count the tokens ahead of the hinted token (top-k verification)
 //   FIN: the logits are expected to hold no -inf: the clamp that makes masked tokens harmless
 //        is skipped, and a row that holds one is re-evaluated by the finisher (its sums are NaN)
-template <int DT, int K, int ND, bool TK, bool FIN, class E>
-__global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJob job, const typename E::Args args) {
+//   NF: finisher warps.  A row's serial path (look-ups, fp64 evaluation, fence and ticket)
+//       takes 5-7 microseconds under load; rows that stream faster than that (below about
+//       200 KB) get three finishers, at the price of 80 instead of 94 registers per thread,
+//       which long rows, where one finisher is idle 40 % of the time, do not pay.
+template <int DT, int K, int ND, bool TK, bool FIN, class E, int NF>
+__global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const StreamJob job, const typename E::Args args) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* tiles = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
     StreamShared& sh = *reinterpret_cast<StreamShared*>(tiles + (size_t)kStages * kTileBytes);
@@ -697,7 +703,16 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
                 break;
             }
             if (last) {
-                if (lane == 0) mbar_arrive(&sh.done[p]);   // wakes the finisher, which sees the end too
+                // every finisher warp has to meet the end of the list: it stands in the records
+                // of this and the next NF - 1 items
+                bool ok = true;
+                for (int j = 0; j < NF && ok; ++j) {
+                    const unsigned int sq = seq + (unsigned int)j;
+                    const int pj = sq % kSlots;
+                    if (j > 0) ok = mbar_wait(&sh.freeb[pj], ((sq / kSlots) & 1u) ^ 1u, abort_flag);
+                    if (ok && lane == 0) mbar_arrive(&sh.done[pj]);
+                }
+                if (!ok && lane == 0) give_up(abort_flag, rj.state);
                 break;
             }
             if (ND > 0) {
@@ -751,7 +766,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
                 if (lane == 0) {
                     const int s = it % kStages;
                     if (mbar_wait(&sh.empty[s], ((it / kStages) & 1u) ^ 1u, abort_flag)) {
-                        sh.ring[seq % kRing].row = kNoItem;
+                        for (int j = 0; j < NF; ++j) sh.ring[(seq + j) % kRing].row = kNoItem;
                         mbar_arrive(&sh.full[s]);
                         // the last CTA to get here leaves the counters ready for the next launch
                         __threadfence();
@@ -823,10 +838,11 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_kernel(const StreamJ
         return;
     }
 
-    // ------------------------------------------------------------------------- finisher
-    Tally tally;   // lane 0's running counters, flushed when the CTA leaves
+    // ------------------------------------------------------------------------ finishers
+    // the items go round the NF finisher warps
+    Tally tally;   // lane 0's running counters, flushed when the warp leaves
     tally.clear();
-    for (unsigned int seq = 0;; ++seq) {
+    for (unsigned int seq = (unsigned int)(warp - kConsumerWarps - 1);; seq += NF) {
         const int p = seq % kSlots;
         if (!mbar_wait(&sh.done[p], (seq / kSlots) & 1u, abort_flag)) {
             if (lane == 0) give_up(abort_flag, rj.state);
