@@ -49,18 +49,47 @@ __device__ __forceinline__ float provisional_ref(const char* row, int vocab, int
     return r;
 }
 
-// Streams vectors [vbeg, vend) of a row plus scalar elements [sbeg, send) and leaves the
-// CTA-wide result in sc.merged (valid for every thread after the closing barrier).
+// The part of a row a CTA streams: 16-byte vectors [vbeg, vend) counted from the 16-byte
+// aligned address vbase, whose first element is token vid0 of the row, and the scalar
+// elements [s1beg, s1end) and [s2beg, s2end) in front of and behind them.  A row that starts
+// on a 16-byte boundary has vbase = row, vid0 = 0 and nothing in front; any other row is
+// peeled up to its first boundary.
+struct RowSpan {
+    const char* vbase;
+    int vid0, vbeg, vend, s1beg, s1end, s2beg, s2end;
+};
+// Elements [beg, end) of a row at an arbitrary (element-aligned) address.
+template <int DT>
+__device__ __forceinline__ RowSpan peeled_span(const char* row, int beg, int end) {
+    constexpr int kVec = Elt<DT>::kVec, kSize = Elt<DT>::kSize;
+    const uintptr_t addr = (uintptr_t)row + (uintptr_t)beg * kSize;
+    int head = (int)(((16u - (unsigned int)(addr & 15u)) & 15u) / kSize);
+    if (head > end - beg) head = end - beg;
+    const int nv = (end - beg - head) / kVec;
+    RowSpan sp;
+    sp.vbase = row + (size_t)(beg + head) * kSize;
+    sp.vid0 = beg + head;
+    sp.vbeg = 0;
+    sp.vend = nv;
+    sp.s1beg = beg;
+    sp.s1end = beg + head;
+    sp.s2beg = beg + head + nv * kVec;
+    sp.s2end = end;
+    return sp;
+}
+
+// Streams a span of a row and leaves the CTA-wide result in sc.merged (valid for every
+// thread after the closing barrier).
 template <int DT, int K, bool SAFE>
-__device__ void block_row_pass(const char* row, int vbeg, int vend, int sbeg, int send, float c1,
-                               float neg_refc, BlockScratch& sc) {
+__device__ void block_row_pass(const char* row, const RowSpan& sp, float c1, float neg_refc, BlockScratch& sc) {
     constexpr int kVec = Elt<DT>::kVec;
     const int tid = threadIdx.x;
     const int lane = tid & 31, warp = tid >> 5;
+    const int vbeg = sp.vbeg, vend = sp.vend;
     RowAccumulator<DT, K, SAFE> acc;
     acc.init();
 
-    const uint4* vrow = reinterpret_cast<const uint4*>(row);
+    const uint4* vrow = reinterpret_cast<const uint4*>(sp.vbase);
     int v = vbeg + tid;
     for (; v + 3 * kThreads < vend; v += 4 * kThreads) {
         uint4 q0 = load_stream16(vrow + v);
@@ -89,15 +118,20 @@ __device__ void block_row_pass(const char* row, int vbeg, int vend, int sbeg, in
             Elt<DT>::unpack(q, x);
 #pragma unroll
             for (int i = 0; i < kVec; ++i)
-                if (x[i] > -CUDART_INF_F) key_insert<K>(ek, make_key(x[i], acc.best_vec[j] * kVec + i));
+                if (x[i] > -CUDART_INF_F) key_insert<K>(ek, make_key(x[i], sp.vid0 + acc.best_vec[j] * kVec + i));
         }
     }
     double S, A;
     acc.totals(S, A);
-    // scalar part: the ragged tail of a vectorised row, or a whole unaligned row
+    // scalar parts: what lies in front of the first 16-byte boundary and the ragged tail
     {
         float s = 0.f, a = 0.f;
-        for (int i = sbeg + tid; i < send; i += kThreads) {
+        for (int i = sp.s1beg + tid; i < sp.s1end; i += kThreads) {
+            float xv = Elt<DT>::load(row, i);
+            acc.add_scalar(xv, c1, neg_refc, s, a);
+            if (xv > -CUDART_INF_F) key_insert<K>(ek, make_key(xv, i));
+        }
+        for (int i = sp.s2beg + tid; i < sp.s2end; i += kThreads) {
             float xv = Elt<DT>::load(row, i);
             acc.add_scalar(xv, c1, neg_refc, s, a);
             if (xv > -CUDART_INF_F) key_insert<K>(ek, make_key(xv, i));
@@ -160,22 +194,27 @@ __device__ bool row_reduce(const RowJob& job, int64_t row, int chunk, int hint, 
     const float c1 = job.c1;
     neg_refc = -(provisional_ref<DT>(rowp, V, hint) * c1);
 
-    int vbeg = 0, vend = 0, sbeg = 0, send = 0;
+    RowSpan sp;
     if (job.vector_ok) {
-        vbeg = chunk * job.vec_per_chunk;
-        vend = min(job.nvec, vbeg + job.vec_per_chunk);
-        if (vbeg > vend) vbeg = vend;
+        sp.vbase = rowp;
+        sp.vid0 = 0;
+        sp.vbeg = chunk * job.vec_per_chunk;
+        sp.vend = min(job.nvec, sp.vbeg + job.vec_per_chunk);
+        if (sp.vbeg > sp.vend) sp.vbeg = sp.vend;
+        sp.s1beg = sp.s1end = 0;
+        sp.s2beg = sp.s2end = 0;
         if (chunk == 0) {
-            sbeg = job.nvec * kVec;
-            send = V;
+            sp.s2beg = job.nvec * kVec;
+            sp.s2end = V;
         }
     } else {
-        // unaligned layout: split the elements themselves
+        // unaligned layout: split the elements themselves, then peel each share up to its
+        // first 16-byte boundary
         int per = (V + job.chunks - 1) / job.chunks;
-        sbeg = min(V, chunk * per);
-        send = min(V, sbeg + per);
+        const int beg = min(V, chunk * per);
+        sp = peeled_span<DT>(rowp, beg, min(V, beg + per));
     }
-    block_row_pass<DT, K, false>(rowp, vbeg, vend, sbeg, send, c1, neg_refc, sc);
+    block_row_pass<DT, K, false>(rowp, sp, c1, neg_refc, sc);
 
     if (job.chunks > 1) {
         RowPartial* slots = job.partials + row * job.chunks;
@@ -235,12 +274,8 @@ __device__ bool row_reduce(const RowJob& job, int64_t row, int chunk, int hint, 
     if (redo) {
         neg_refc = -m;
         centered = true;
-        int vb = 0, ve = 0, sb = 0, se = V;
-        if (job.vector_ok) {
-            ve = job.nvec;
-            sb = job.nvec * kVec;
-        }
-        block_row_pass<DT, K, true>(rowp, vb, ve, sb, se, c1, neg_refc, sc);
+        RowSpan all = peeled_span<DT>(rowp, 0, V);   // an aligned row peels nothing
+        block_row_pass<DT, K, true>(rowp, all, c1, neg_refc, sc);
         if (tid == 0) atomicAdd(&job.state->counters[kCntRedo], 1ull);
     }
     return true;
