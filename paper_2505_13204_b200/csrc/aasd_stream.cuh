@@ -3,17 +3,20 @@
 // One CTA per SM slot runs for the whole launch.  A producer warp moves 32 KB tiles of the
 // rows from HBM into a ring of shared-memory stages with bulk asynchronous copies (TMA,
 // cp.async.bulk, completion signalled on an mbarrier); eight consumer warps turn each tile
-// into running sums and best-token candidates; a finisher warp merges what the consumers
-// leave per work item, combines the pieces of rows that were split over several CTAs and
-// evaluates the row (entropy, probabilities, threshold test, accept scan).  The three roles
-// only meet at mbarriers, so the copies of the next rows are in flight while the current
-// row is being reduced and finished.
+// into running sums and best-token candidates; a finisher warp (three of them, taking the
+// items in turn, when rows are short) merges what the consumers leave per work item,
+// combines the pieces of rows that were split over several CTAs and evaluates the row
+// (entropy, probabilities, threshold test, accept scan).  The three roles only meet at
+// mbarriers, so the copies of the next rows are in flight while the current row is being
+// reduced and finished.
 //
 // Work is handed out dynamically: the producer claims the next work item from a counter in
 // global memory, so a CTA that runs on a slower path to memory simply takes fewer items.
 // An item is a whole row, or, when the host finds rows scarce, a piece of a row cut at tile
 // boundaries (rows [0, whole_rows) are whole, later rows are cut).  The pieces of a row meet
-// in global memory and the CTA that delivers the last one finishes the row.
+// in the shared memory of a thread-block cluster's first CTA when the launch is made of one
+// cluster per row, else in global memory, where the CTA that delivers the last one finishes
+// the row.
 //
 // Every wait is bounded: a role that gives up raises AASD_STATUS_TIMEOUT, tells the other
 // roles through a shared flag and leaves; the producer first waits (bounded again) for the
