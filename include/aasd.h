@@ -21,8 +21,10 @@
  *    vocabulary, NaN or +inf logit, history overflow) set bits in a device status word
  *    that aasd_poll_status returns and clears; the kernels never trap.
  *  - Logits are row-major [rows x vocab] with a row stride given in elements; dtype is
- *    AASD_F32 or AASD_BF16.  Rows whose start is 16-byte aligned take the vectorised path;
- *    other layouts are handled by a slower scalar path with identical results.
+ *    AASD_F32 or AASD_BF16.  When the buffer and the row stride in bytes are multiples of
+ *    16, so that every row starts on a 16-byte boundary, the rows are streamed at close to
+ *    memory speed; other layouts (a bf16 vocabulary of 50257 with stride = vocab, say) are
+ *    handled by a path about half as fast with identical results, so pad the stride.
  *  - Token ids are int32, AASD_NONE (-1) means "no token".  Offsets arrays are CSR.
  *  - Scratch memory comes from the caller: a workspace of aasd_workspace_bytes() bytes
  *    that was registered once with aasd_workspace_init().  A workspace must not be shared
