@@ -17,7 +17,7 @@ NONE = -1
 F32, BF16 = 0, 1
 ALIGN_TOPK, ALIGN_GUMBEL = 0, 1
 VERIFY_CONDITIONAL, VERIFY_STRICT_GREEDY, VERIFY_STRICT_SAMPLED, VERIFY_TOP_K = 0, 1, 2, 3
-STATUS_BAD_ROW, STATUS_ID_RANGE, STATUS_HIST_OVERFLOW, STATUS_BAD_OFFSETS = 1, 2, 4, 8
+STATUS_BAD_ROW, STATUS_ID_RANGE, STATUS_HIST_OVERFLOW, STATUS_BAD_OFFSETS, STATUS_TIMEOUT = 1, 2, 4, 8, 16
 FLAG_CONDITIONAL, FLAG_EXTRA = 1, 2
 DRAFT_MATCH_ALIGN = 1
 HINT_FINITE = 1

@@ -388,3 +388,51 @@ def test_cluster_and_global_combine_agree(ctx, V, dtype, rows, monkeypatch):
     for k in results[0]:
         assert torch.equal(results[0][k], results[1][k]), k
     assert ctx.poll_status() == 0
+
+
+@pytest.mark.parametrize("V,dtype", [(1000, torch.float32), (32000, torch.float32), (4096, torch.bfloat16)])
+def test_decisions_near_the_threshold_are_counted_and_excluded(ctx, V, dtype):
+    """Eq. 5 on rows whose draft probability is placed within and outside 1e-6 of
+    alpha*H + beta.  The oracle flags the rows inside the band (`near`), the device counts
+    them (`near_threshold`), and the comparison skips exactly those: outside the band the
+    accept bits must agree, at a gap of zero either decision is legitimate."""
+    rng = np.random.default_rng(V)
+    gaps = [+5e-7, -5e-7, +2e-6, -2e-6, 0.0, +3e-7, -3e-7, +4e-6]
+    rows_per_cand = 3                      # [best token, the placed token, best token]
+    alpha = F32(0.1)
+    # one row: four live tokens of probability ~ (1/2, 1/4, 1/8, 1/8) on top of a masked
+    # vocabulary (fp32) or a far-away floor (bf16), at seeded places
+    place = rng.choice(V, 4, replace=False)
+    base = torch.full((V,), -float("inf") if dtype == torch.float32 else -60.0, dtype=torch.float32)
+    base[torch.as_tensor(place)] = torch.log(torch.tensor([0.5, 0.25, 0.125, 0.125]))
+    x1 = base.to(dtype)[None, :]
+    st = oracle.verify(to_oracle(x1), [int(place[1])], [0, 1], alpha=alpha, beta=0.0)
+    pd, H = float(st["p_draft"][0]), float(st["entropy"][0])
+    xd = x1.repeat(rows_per_cand, 1).cuda()
+    d = np.asarray([place[0], place[1], place[0]], np.int32)
+    offs = np.asarray([0, rows_per_cand], np.int32)
+    n_near = 0
+    ctx.reset_counters()
+    for gap in gaps:
+        beta = F32(pd - alpha * H - gap)
+        ref = oracle.verify(to_oracle(x1.repeat(rows_per_cand, 1)), d, offs, alpha=alpha, beta=beta)
+        want_near = abs(gap) < 1e-6
+        assert ref["near"].tolist() == [0, int(want_near), 0], gap
+        if abs(gap) > 1e-7:
+            assert ref["accept"].tolist() == [1, int(gap > 0), 1], gap
+        got = ctx.verify(xd, torch.as_tensor(d).cuda(), torch.as_tensor(offs).cuda(), alpha=alpha, beta=beta)
+        assert check_verify(got, ref, offs, dtype) == int(want_near)
+        if abs(gap) >= 4e-7:
+            # the kernel's own probability is within 1e-7 of the oracle's here: same decision
+            assert cpu(got["accept"]).tolist() == ref["accept"].tolist(), gap
+        n_near += int(want_near)
+    assert ctx.poll_status() == 0
+    assert ctx.counters()["near_threshold"] == n_near
+    # the token at the row maximum is decided by the Delta clause: never counted
+    ctx.reset_counters()
+    st0 = oracle.verify(to_oracle(x1), [int(place[0])], [0, 1], alpha=alpha, beta=0.0)
+    beta = F32(float(st0["p_draft"][0]) - alpha * H + 5e-7)
+    got = ctx.verify(xd[:1], torch.as_tensor(d[:1]).cuda(), torch.as_tensor(np.asarray([0, 1], np.int32)).cuda(),
+                     alpha=alpha, beta=beta)
+    assert cpu(got["accept"]).tolist() == [1]
+    assert ctx.counters()["near_threshold"] == 0
