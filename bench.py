@@ -9,14 +9,22 @@ the longest passing candidate and history append.  Over the configuration's 64 s
 is exactly its 256 x 1024 prefill rows and 64 x 4096 verification rows.
 
 The logits of every step are resident in HBM before the timed region (8 rotating buffers
-of 1.25 GB each for prefill and for verification rows: far larger than L2).  The decoding
-state is replayed: the logits of step j were drawn for the candidates the drafter emits at
-state j, and the state is restored every 8 steps by a small device copy inside the timed
-region.
+of 1.25 GB each for prefill and for verification rows: far larger than L2).  Decoding runs
+open loop: the key of every sequence in step j is a seeded window of its prompt, chosen at
+set-up so that the drafter fills every candidate slot (all 4096 verification rows carry a
+real draft token), and the logits of step j were drawn for exactly those candidates.  The
+emitted tokens are appended as always; the state is replayed (restored every 8 steps by a
+small device copy inside the timed region).
+
+After the K timed steps the same step runs for a few seconds more (the `sustained` leg,
+clocks sampled inside it), the sampling variants of the two streaming kernels are timed on
+the same buffers, and alignment sampling runs over one whole long-context prefill block
+(16384 x 128256 bf16, 4.2 GB).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload i]
 
-prints one JSON line.  `--impl reference` times the CPU oracle on the host cores.
+prints one JSON line.  With N > 1 and no launcher around it, the program starts N ranks of
+itself (one per GPU).  `--impl reference` times the CPU oracle on the host cores.
 """
 from __future__ import annotations
 
@@ -26,6 +34,7 @@ import os
 import subprocess
 import sys
 import tempfile
+import threading
 import time
 
 import numpy as np
@@ -71,24 +80,63 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+    """SM clock and throttle reasons of one GPU, read while a timed region runs.
+
+    Reads only (NVML's clock and clocks-event-reasons queries from a thread, every
+    millisecond or so: the short timed region lasts a few milliseconds); falls back to an
+    nvidia-smi loop when the NVML binding is missing.  Changes no setting of the GPU."""
+    REASONS = {"hw_slowdown": 0x8, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20,
+               "sw_power_cap": 0x4}
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, index: int):
-        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
-        self.p = None
+    def __init__(self, index: int, period_s: float = 0.001):
+        self.sm, self.power, self.bits = [], [], 0
+        self.max_mhz = None
+        self.p = self.f = self.thread = None
+        self.stop_flag = False
         try:
-            self.p = subprocess.Popen(
-                ["nvidia-smi", "-i", str(index), "--query-gpu=" + self.Q,
-                 "--format=csv,noheader,nounits", "-lms", "50"], stdout=self.f,
-                stderr=subprocess.DEVNULL)
-        except OSError:
-            pass
+            import pynvml
+            pynvml.nvmlInit()
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+            phys = int(vis.split(",")[index]) if vis and vis.split(",")[index].isdigit() else index
+            h = pynvml.nvmlDeviceGetHandleByIndex(phys)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+
+            def loop():
+                while not self.stop_flag:
+                    try:
+                        self.sm.append(float(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)))
+                        self.bits |= int(pynvml.nvmlDeviceGetCurrentClocksEventReasons(h))
+                        self.power.append(pynvml.nvmlDeviceGetPowerUsage(h) / 1000.0)
+                    except Exception:
+                        pass
+                    time.sleep(period_s)
+            self.thread = threading.Thread(target=loop, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.thread = None
+            self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            try:
+                self.p = subprocess.Popen(
+                    ["nvidia-smi", "-i", str(index), "--query-gpu=" + self.Q,
+                     "--format=csv,noheader,nounits", "-lms", "20"], stdout=self.f,
+                    stderr=subprocess.DEVNULL)
+            except OSError:
+                pass
 
     def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "how": None}
+        if self.thread is not None:
+            self.stop_flag = True
+            self.thread.join(timeout=2)
+            if self.sm:
+                out.update(sm_mhz=float(np.median(self.sm)), sm_min_mhz=float(min(self.sm)),
+                           sm_max_mhz=self.max_mhz, samples=len(self.sm),
+                           power_w_max=max(self.power) if self.power else None,
+                           reasons=sorted(n for n, b in self.REASONS.items() if self.bits & b), how="nvml")
+            return out
         if self.p is None:
             return out
         self.p.terminate()
@@ -115,14 +163,31 @@ class ClockSampler:
         self.f.close()
         os.unlink(self.f.name)
         if sm:
-            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), samples=len(sm),
-                       reasons=sorted(reasons))
+            out.update(sm_mhz=float(np.median(sm)), sm_min_mhz=float(min(sm)), sm_max_mhz=float(max(mx)),
+                       samples=len(sm), reasons=sorted(reasons), how="nvidia-smi")
         return out
 
 
 # --------------------------------------------------------------------------------------
 # our arm
 # --------------------------------------------------------------------------------------
+def full_keys(state, prompts, n, draft_len, seed, dev, tries: int = 24):
+    """Keys of one open-loop step: a seeded prompt window per sequence, redrawn (for the
+    sequences concerned only) until the drafter fills every candidate slot at the current
+    state.  Returns (keys, rows still empty)."""
+    keys = synth.open_loop_keys(prompts, n, draft_len, seed).to(dev)
+    B = len(prompts)
+    for t in range(tries):
+        dg = state.run_draft(keys)
+        bad = (dg["draft_ids"] < 0).view(B, -1).any(dim=1)
+        if not bool(bad.any()):
+            return keys, 0
+        new = synth.open_loop_keys(prompts, n, draft_len, seed * 131 + t + 1).to(dev)
+        keys = torch.where(bad[:, None], new, keys).contiguous()
+    dg = state.run_draft(keys)
+    return keys, int((dg["draft_ids"] < 0).sum().item())
+
+
 class Bench:
     def __init__(self, w: synth.Workload, device, rank: int):
         from paper_2505_13204_b200 import binding
@@ -134,6 +199,7 @@ class Bench:
         self.pre_rows = self.seqs_per_step * w.prompt_len
         self.R = w.rows_per_step
         seed0 = shard.rank_seed(w.seed, rank)
+        self.seed0 = seed0
         t0 = time.time()
         self.prompts = [synth.prompt_ids(synth.scaled(w, seed=seed0), b) for b in range(w.batch)]
         ids_all = torch.cat(self.prompts).to(device)
@@ -170,7 +236,7 @@ class Bench:
                 self.pre_out.append(out)
         del scratch
         torch.cuda.synchronize()
-        # decoding state and the replayed verification logits
+        # decoding state and the replayed verification logits (open loop: keys from the prompts)
         align = dict(align_ids=self.table["align_ids"], n_extra=self.table["n_extra"])
         self.state = binding.DecodeState(self.ctx, self.prompts, N_BUF * (w.draft_len + 1) + 8, w.ngram,
                                          w.draft_len, w.max_cands, w.vocab, w.torch_dtype, align=align,
@@ -179,17 +245,36 @@ class Bench:
         self.hist0 = self.state.hist_ids.clone()
         self.len0 = self.state.hist_len.clone()
         self.tab0 = (self.state.align["align_ids"].clone(), self.state.align["n_extra"].clone()) if EXTEND_TABLE else None
-        self.ver_bufs = []
+        self.ver_bufs, self.keys, self.patch, self.draft_ids = [], [], [], []
+        self.empty_rows = self.below_delta = self.accepted_rows = 0
         for j in range(N_BUF):
-            d = self.state.run_draft()["draft_ids"].reshape(-1).to(torch.int64)
+            keys, empty = full_keys(self.state, self.prompts, w.ngram, w.draft_len, seed0 * 8191 + j, device)
+            dg = self.state.run_draft(keys)
+            patch = None
+            if empty:
+                # slots the drafter left empty all the same take the harness's seeded tokens
+                pad = synth.pad_ids(self.prompts, w.max_cands, w.draft_len, seed0 * 8191 + j).to(device)
+                miss = dg["draft_ids"] < 0
+                patch = (torch.where(miss, pad, dg["draft_ids"]).contiguous(),
+                         dg["draft_flags"].masked_fill(miss, 1).contiguous())
+                dg["draft_ids"].copy_(patch[0])
+                dg["draft_flags"].copy_(patch[1])
+            self.empty_rows += empty
+            d = dg["draft_ids"].reshape(-1).to(torch.int64)
             x = synth.logits(self.R, w.vocab, w.torch_dtype, w.recipe, d, seed0 + 977 * (j + 1),
                              device=device, noise=self.bank.block(100 + j), chunk_rows=1024)
             self.ver_bufs.append(x)
-            self.state.step(x, j)
+            self.keys.append(keys)
+            self.patch.append(patch)
+            self.draft_ids.append(dg["draft_ids"].reshape(-1).clone())
+            self.state.step(x, j, reuse_draft=True)
+            vo = self.state.verify_out
+            self.below_delta += int(((vo["accept"] == 1) & (vo["p_draft"] < vo["pmax"])).sum().item())
+            self.accepted_rows += int(vo["accept"].sum().item())
         torch.cuda.synchronize()
+        self.real_rows_per_step = self.R - sum(int((d < 0).sum().item()) for d in self.draft_ids) / N_BUF
         self.accepted_per_cycle = int((self.state.hist_len - self.len0).sum().item())
         self.restore()
-        self.ev_align = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
         self.setup_s = time.time() - t0
         del self.bank
 
@@ -205,6 +290,12 @@ class Bench:
             self.state.align["align_ids"].copy_(self.tab0[0])
             self.state.align["n_extra"].copy_(self.tab0[1])
 
+    def draft(self, j: int):
+        self.state.run_draft(self.keys[j])
+        if self.patch[j] is not None:
+            self.state.draft_out["draft_ids"].copy_(self.patch[j][0])
+            self.state.draft_out["draft_flags"].copy_(self.patch[j][1])
+
     def step(self, s: int, events=None):
         j = s % N_BUF
         if j == 0 and s > 0:
@@ -216,12 +307,82 @@ class Bench:
                               outputs=self.pre_out[ja], finite_hint=FINITE_HINT)
         if events is not None:
             events[1].record()
-        self.state.run_draft()
+        self.draft(j)
         if events is not None:
             events[2].record()
         self.state.step(self.ver_bufs[j], j, reuse_draft=True)
         if events is not None:
             events[3].record()
+
+
+def kernel_leg(call, n_bufs: int, bytes_per_launch: int, peak: float, reps: int = 16, warm: int = 3):
+    """One kernel alone over rotating resident buffers: CUDA events around `reps` launches."""
+    for j in range(warm):
+        call(j % n_bufs)
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    t0.record()
+    for j in range(reps):
+        call(j % n_bufs)
+    t1.record()
+    torch.cuda.synchronize()
+    ms = t0.elapsed_time(t1) / reps
+    gbs = bytes_per_launch / (ms * 1e-3) / 1e9
+    return {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
+            "frac_of_nominal_8000": gbs / 8000.0, "ms_per_launch": ms, "bytes_per_launch": int(bytes_per_launch),
+            "launches_timed": reps, "traffic": None}
+
+
+def sampled_legs(bench: "Bench", peak: float):
+    """The keyed-sampler variants of the two streaming kernels on the step's own buffers:
+    STRICT_SAMPLED verification (one draw per row, Eq. 1) and GUMBEL alignment sampling
+    (k_extra draws per misaligned row, Sec. 2.3)."""
+    w, b = bench.w, bench.binding
+    esize = 2 if w.dtype == "bf16" else 4
+    vout = dict(bench.state.verify_out)
+    aout = None
+
+    def verify(j):
+        bench.ctx.verify(bench.ver_bufs[j], bench.draft_ids[j], None, rows_per_cand=w.draft_len, outputs=vout,
+                         seed=17, step=j, mode=b.VERIFY_STRICT_SAMPLED, finite_hint=FINITE_HINT)
+
+    def align(j):
+        nonlocal aout
+        aout = bench.ctx.align_sample(bench.pre_bufs[j], bench.pre_ids[j], bench.pre_offs[j], k_extra=K_EXTRA,
+                                      outputs=aout, seed=17, mode=b.ALIGN_GUMBEL, finite_hint=FINITE_HINT)
+
+    v = kernel_leg(verify, N_BUF, bench.R * w.vocab * esize, peak)
+    v["kernel"] = "stream_kernel<%s, K=1, ND=1, VerifyEpilogue> (STRICT_SAMPLED, %d rows)" % (w.dtype, bench.R)
+    a = kernel_leg(align, len(bench.pre_bufs), bench.pre_rows * w.vocab * esize, peak)
+    a["kernel"] = "align_next_kernel + stream_kernel<%s, K=1, ND=%d, AlignEpilogue> (GUMBEL, %d rows)" % (
+        w.dtype, K_EXTRA, bench.pre_rows)
+    return {"verify": v, "align": a}
+
+
+def align_long_context_leg(dev, peak: float):
+    """Alignment sampling over the whole prefill block of the long-context configuration
+    (one sequence, 16384 positions, vocabulary 128256, bf16: 4.2 GB), alone."""
+    from paper_2505_13204_b200 import binding
+    w = synth.workload(3)
+    ctx = binding.Context()
+    ids = synth.prompt_ids(w, 0).to(dev)
+    hints = synth.next_token_hints(ids)
+    x = synth.logits(w.prompt_len, w.vocab, w.torch_dtype, w.recipe, hints, w.seed, device=dev, chunk_rows=1024)
+    offs = torch.tensor([0, w.prompt_len], dtype=torch.int32, device=dev)
+    out = None
+
+    def call(_):
+        nonlocal out
+        out = ctx.align_sample(x, ids, offs, k_extra=K_EXTRA, outputs=out, finite_hint=FINITE_HINT)
+
+    leg = kernel_leg(call, 1, w.prompt_len * w.vocab * 2, peak, reps=8)
+    leg["kernel"] = "align_next_kernel + stream_kernel<bf16, K=%d, ND=0, AlignEpilogue>" % K_EXTRA
+    leg["workload"] = "%s prefill: %d x %d bf16, one buffer of %.2f GB (larger than L2)" % (
+        w.name, w.prompt_len, w.vocab, w.prompt_len * w.vocab * 2 / 1e9)
+    ctx.close()
+    del x
+    torch.cuda.empty_cache()
+    return leg
 
 
 def run_ours(args, rank, world, local_rank):
@@ -233,10 +394,6 @@ def run_ours(args, rank, world, local_rank):
     w = synth.workload(args.workload)
     bench = Bench(w, dev, rank)
     K, W = args.steps, max(args.warmup, 3)
-    for s in range(W):
-        bench.step(s)
-    torch.cuda.synchronize()
-    bench.restore()
 
     def barrier():
         if world > 1:
@@ -246,12 +403,16 @@ def run_ours(args, rank, world, local_rank):
     launches0 = bench.ctx.launch_count()
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K)]
     t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
+    # the warm-up steps run straight into the timed ones: step s of the timed region is step
+    # W + s of one uninterrupted sequence, and the clock sampler covers all of it
     clocks = ClockSampler(local_rank)
-    time.sleep(0.2)
+    for s in range(W):
+        bench.step(s)
+    barrier()
+    launches0 = bench.ctx.launch_count()
     t_begin.record()
     for s in range(K):
-        bench.step(s, evs[s])
+        bench.step(W + s, evs[s])
     t_end.record()
     barrier()
     clk = clocks.stop()
@@ -261,6 +422,40 @@ def run_ours(args, rank, world, local_rank):
     draft_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in evs]))
     verify_ms = float(np.mean([e[2].elapsed_time(e[3]) for e in evs]))
     ms = shard.max_over_ranks(ms, dev)
+
+    esize = 2 if w.dtype == "bf16" else 4
+    peak, peak_src = measured_peaks()
+    row_bytes = w.vocab * esize
+
+    # the same step for a few seconds more: what the path sustains under the power cap
+    sustained = None
+    if args.sustain_seconds > 0:
+        n_sus = max(64, int(args.sustain_seconds * 1e3 / (ms / K)))
+        every = 16
+        sev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(n_sus // every + 1)]
+        s_begin, s_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        sclocks = ClockSampler(local_rank, period_s=0.005)
+        s_begin.record()
+        for s in range(n_sus):
+            bench.step(W + K + s, sev[s // every] if s % every == 0 else None)
+        s_end.record()
+        barrier()
+        sclk = sclocks.stop()
+        s_ms = shard.max_over_ranks(s_begin.elapsed_time(s_end), dev)
+        used = [e for i, e in enumerate(sev) if i * every < n_sus]
+        s_align = float(np.mean([e[0].elapsed_time(e[1]) for e in used]))
+        s_verify = float(np.mean([e[2].elapsed_time(e[3]) for e in used]))
+        sustained = {"seconds": s_ms * 1e-3, "steps": n_sus, "ms_per_step": s_ms / n_sus,
+                     "value": shard.whole_job_rate(bench.R, n_sus, world, s_ms), "unit": UNIT,
+                     "verify_ms_per_launch": s_verify, "align_ms_per_launch": s_align,
+                     "verify_gbs": bench.R * row_bytes / (s_verify * 1e-3) / 1e9,
+                     "align_gbs": bench.pre_rows * row_bytes / (s_align * 1e-3) / 1e9,
+                     "verify_frac": bench.R * row_bytes / (s_verify * 1e-3) / 1e9 / peak,
+                     "align_frac": bench.pre_rows * row_bytes / (s_align * 1e-3) / 1e9 / peak,
+                     "sm_mhz_median": sclk["sm_mhz"], "sm_mhz_min": sclk.get("sm_min_mhz"),
+                     "power_w_max": sclk.get("power_w_max"), "reasons": sclk["reasons"],
+                     "clock_samples": sclk["samples"], "events": "every %dth step" % every}
 
     # what a read-only stream with no arithmetic reaches on this device, same buffers, same run
     sink = torch.zeros(1, dtype=torch.int32, device=dev)
@@ -275,6 +470,8 @@ def run_ours(args, rank, world, local_rank):
     buf_bytes = bench.ver_bufs[0].numel() * bench.ver_bufs[0].element_size()
     read_probe_gbs = 16 * buf_bytes / (p0.elapsed_time(p1) * 1e-3) / 1e9
 
+    sampled = sampled_legs(bench, peak) if (world == 1 and not args.no_extra_legs) else None
+
     # end to end: the same step fed from pinned host memory through the C ABI
     e2e = run_e2e(bench, dev, min(K, 4))
     e2e["ms_per_step"] = shard.max_over_ranks(e2e["ms_per_step"], dev)
@@ -283,27 +480,30 @@ def run_ours(args, rank, world, local_rank):
             dist.destroy_process_group()
         return
 
-    esize = 2 if w.dtype == "bf16" else 4
-    peak, peak_src = measured_peaks()
-    row_bytes = w.vocab * esize
     # events bracket the verification launch alone (selection and append ride on it) and the
     # two launches of aasd_align_sample (next-token gather, ~3 us, + streaming kernel)
     ver_gbs = bench.R * row_bytes / (verify_ms * 1e-3) / 1e9
     ali_gbs = bench.pre_rows * row_bytes / (align_ms * 1e-3) / 1e9
     value = shard.whole_job_rate(bench.R, K, world, ms)
+    cnt = bench.ctx.counters()
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name, "sequences_per_gpu": w.batch, "vocab": w.vocab,
                    "logits_dtype": w.dtype, "verify_rows_per_step": bench.R,
+                   "real_draft_rows_per_step": bench.real_rows_per_step,
+                   "rows_filled_by_the_harness_per_step": bench.empty_rows / N_BUF,
                    "prefill_rows_per_step": bench.pre_rows, "ngram": w.ngram, "k_extra": K_EXTRA,
-                   "alpha": ALPHA, "beta": BETA, "finite_hint": FINITE_HINT, "extend_table": EXTEND_TABLE, "parallelism": "replicas x%d (sequences sharded, no collective)" % world,
+                   "alpha": ALPHA, "beta": BETA, "finite_hint": FINITE_HINT, "extend_table": EXTEND_TABLE,
+                   "driver": "open loop: keys are seeded prompt windows, every candidate slot holds real tokens",
+                   "parallelism": "replicas x%d (sequences sharded, no collective)" % world,
                    "l2": "inputs larger than L2: %d rotating buffers of %.2f GB" % (2 * N_BUF, bench.R * row_bytes / 1e9),
                    "noise": "one bank of normals re-used under cyclic shifts",
                    "setup_s": round(bench.setup_s, 1)},
         "clocks": {"sm_mhz": clk["sm_mhz"], "sm_max_mhz": clk["sm_max_mhz"], "reasons": clk["reasons"],
-                   "samples": clk["samples"]},
+                   "samples": clk["samples"], "how": clk["how"],
+                   "covers": "%d warm-up + %d timed steps, run back to back" % (W, K)},
         "e2e": {"value": world * bench.R / (e2e["ms_per_step"] * 1e-3), "unit": UNIT,
                 "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
                 "ms_per_step": e2e["ms_per_step"]},
@@ -321,15 +521,24 @@ def run_ours(args, rank, world, local_rank):
                            "frac_of_nominal_8000": ali_gbs / 8000.0, "frac_of_read_probe": ali_gbs / read_probe_gbs,
                            "peak_source": peak_src, "traffic": ncu_traffic(w.name, "align", bench.pre_rows),
                            "ms_per_launch": align_ms, "bytes_per_launch": bench.pre_rows * row_bytes},
+        "sustained": sustained,
+        "roofline_sampled": sampled,
         "draft_us_per_launch": draft_ms * 1e3,
         "read_probe_gbs": read_probe_gbs,
         "logits_gbs": (bench.R + bench.pre_rows) * row_bytes * K / (ms * 1e-3) / 1e9,
-        "accepted_tokens_per_s": world * bench.accepted_per_cycle / N_BUF * K / (ms * 1e-3),
+        "emitted_tokens_per_s": world * bench.accepted_per_cycle / N_BUF * K / (ms * 1e-3),
         "mean_tokens_per_seq_step": bench.accepted_per_cycle / N_BUF / w.batch,
-        "counters": bench.ctx.counters(),
+        "accepted_rows_per_step": bench.accepted_rows / N_BUF,
+        "accepted_below_delta_per_step": bench.below_delta / N_BUF,
+        "counters": cnt,
     }
-    if world == 1 and not args.no_latency:
+    if world == 1 and not args.no_extra_legs:
         del bench
+        torch.cuda.empty_cache()
+        line["roofline_align_cfg4"] = align_long_context_leg(dev, peak)
+        line["roofline_align_cfg4"]["peak_source"] = peak_src
+    if world == 1 and not args.no_latency:
+        bench = None
         torch.cuda.empty_cache()
         line["decode_step_latency_us"] = {synth.workload(i).name: decode_step_latency(i, dev) for i in range(4)}
     if not args.no_cpu_baseline and world == 1:
@@ -344,8 +553,10 @@ def decode_step_latency(index: int, dev, n_buf: int = 4, reps: int = 50):
 
     The single-sequence configurations verify 8-12 rows per step: that is latency, not
     bandwidth, so the figure is microseconds per step, measured by replaying a CUDA graph of
-    n_buf consecutive steps (a launch from Python costs more than such a step runs).  The
-    logits of step j are drawn for the candidates the drafter emits at state j."""
+    n_buf consecutive steps (a launch from Python costs more than such a step runs).  Open
+    loop like the main benchmark: the keys are prompt windows for which the drafter fills
+    every slot, and the logits of step j are drawn for those candidates.  Also times the
+    verification launch alone (`verify_launch_us`, same graph without the drafting calls)."""
     from paper_2505_13204_b200 import binding
     w = synth.workload(index)
     side = torch.cuda.Stream()
@@ -355,32 +566,43 @@ def decode_step_latency(index: int, dev, n_buf: int = 4, reps: int = 50):
         st = binding.DecodeState(ctx, prompts, n_buf * (w.draft_len + 1) + 8, w.ngram, w.draft_len, w.max_cands,
                                  w.vocab, w.torch_dtype, alpha=ALPHA, beta=BETA)
         hist0, len0 = st.hist_ids.clone(), st.hist_len.clone()
-        bufs = []
+        bufs, keys, real = [], [], 0
         for j in range(n_buf):
-            d = st.run_draft()["draft_ids"].reshape(-1).to(torch.int64)
+            k, empty = full_keys(st, prompts, w.ngram, w.draft_len, w.seed * 8191 + j, dev)
+            d = st.run_draft(k)["draft_ids"].reshape(-1).to(torch.int64)
+            real += int((d >= 0).sum().item())
             x = synth.logits(st.rows, w.vocab, w.torch_dtype, w.recipe, d, w.seed + 977 * (j + 1), device=dev,
                              chunk_rows=1024)
             bufs.append(x)
+            keys.append(k)
             st.step(x, j, reuse_draft=True)
         side.synchronize()
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph, stream=side):
-            st.hist_ids.copy_(hist0)
-            st.hist_len.copy_(len0)
-            for j in range(n_buf):
-                st.run_draft()
-                st.step(bufs[j], j, reuse_draft=True)
-        for _ in range(3):
-            graph.replay()
-        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        t0.record()
-        for _ in range(reps):
-            graph.replay()
-        t1.record()
+
+        def timed(with_draft: bool):
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                st.hist_ids.copy_(hist0)
+                st.hist_len.copy_(len0)
+                for j in range(n_buf):
+                    if with_draft:
+                        st.run_draft(keys[j])
+                    st.step(bufs[j], j, reuse_draft=True)
+            for _ in range(3):
+                graph.replay()
+            t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            t0.record()
+            for _ in range(reps):
+                graph.replay()
+            t1.record()
+            side.synchronize()
+            return t0.elapsed_time(t1) * 1e3 / (reps * n_buf)
+
+        us = timed(True)
+        us_verify = timed(False)
     torch.cuda.synchronize()
-    us = t0.elapsed_time(t1) * 1e3 / (reps * n_buf)
     ctx.close()
-    return {"us_per_step": us, "verify_rows": st.rows, "sequences": w.batch,
+    return {"us_per_step": us, "verify_launch_us": us_verify, "verify_rows": st.rows,
+            "real_draft_rows": real / n_buf, "sequences": w.batch,
             "note": "draft + verify/select/append, graph replay; includes 1/%d of a state restore" % n_buf}
 
 
@@ -407,7 +629,8 @@ def run_e2e(bench: Bench, dev, steps: int):
         dver.copy_(host_ver, non_blocking=True)
         bench.ctx.align_sample(dpre, bench.pre_ids[0], bench.pre_offs[0], k_extra=K_EXTRA,
                                outputs=bench.pre_out[0], finite_hint=FINITE_HINT)
-        st.step(dver, 0)
+        bench.draft(0)
+        st.step(dver, 0, reuse_draft=True)
         res_emit.copy_(st.emit_ids, non_blocking=True)
         res_n.copy_(st.n_emit, non_blocking=True)
         res_tab.copy_(bench.pre_out[0]["align_ids"], non_blocking=True)
@@ -599,6 +822,10 @@ def main():
     ap.add_argument("--workload", type=int, default=4, help="0-based index of the configuration")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-latency", action="store_true", help="skip the decode-step latencies of configs 1-4")
+    ap.add_argument("--no-extra-legs", action="store_true",
+                    help="skip the sampling-kernel legs and the long-context alignment pass")
+    ap.add_argument("--sustain-seconds", type=float, default=2.5,
+                    help="length of the sustained leg after the timed steps (0: none)")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--no-finite-hint", action="store_true",
                     help="do not tell the library that the logits hold no -inf")
@@ -614,6 +841,14 @@ def main():
     if args.impl == "reference":
         run_reference(args, rank, world)
         return
+    if not args.micro:
+        try:
+            plan = shard.launch_plan(args.gpus)
+        except ValueError as e:
+            raise SystemExit("bench.py: %s" % e)
+        if plan == "spawn":
+            # started plainly with --gpus N > 1: start the N ranks (one process per GPU)
+            raise SystemExit(shard.spawn_ranks(os.path.abspath(__file__), sys.argv[1:], args.gpus))
     if args.micro:
         run_micro(args)
         return

@@ -390,6 +390,24 @@ int aasd_verify_tree(aasd_ctx* ctx, const void* target_logits, const int32_t* no
  * benchmark reports it beside the kernels' figures; it is not part of the method. */
 int aasd_probe_read(aasd_ctx* ctx, const void* buffer, size_t bytes, uint32_t* sink);
 
+/* ---- testing aid: showing that a launch whose data never arrives ends by itself -------- */
+
+/* Every wait inside the kernels is bounded: a role that waits longer than its limit raises
+ * AASD_STATUS_TIMEOUT, tells the other roles of its CTA, and all of them leave; the launch
+ * then ends like any other, with invalid results for the rows concerned and a workspace that
+ * has to be registered again.  This call lets a test see that happen without any fault: it
+ * arms, for the NEXT launch of the streaming kernel made through this context (by
+ * aasd_verify, aasd_align_sample, aasd_step or aasd_verify_tree) and for that launch only,
+ *   - a wait limit of `wait_limit` polls (>= 1024) instead of the default 2^24, and
+ *   - the CTA that handles work item `item` (a logits row when the call has at least twice
+ *     as many rows as the device has SMs, else a piece of a row) never issuing the copy of
+ *     that item's tile number `tile` (32 KB tiles, counted within the item).
+ * The consumers of that CTA run out of polls, the CTA leaves, the other CTAs finish their
+ * rows, and aasd_poll_status shows AASD_STATUS_TIMEOUT.  Afterwards: aasd_workspace_init on
+ * the workspace, and the context works as before.  Nothing is armed when `item` lies beyond
+ * the launch's items (the limit still applies).  Not for production use. */
+int aasd_debug_withhold_tile(aasd_ctx* ctx, int64_t item, int32_t tile, uint32_t wait_limit);
+
 /* ---- verification for callers that cannot allocate ------------------------------- */
 
 #define AASD_STATIC_MAX_ROWS 8192   /* most logits rows per aasd_verify_static call */

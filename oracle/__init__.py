@@ -136,12 +136,16 @@ def align_sample(logits, prompt_ids, seq_offsets, k_extra=2, mode=ALIGN_TOPK, se
 
 def draft(hist_ids, hist_offsets, hist_len, prompt_len, recent_ids, recent_len, n, draft_len,
           max_cands, align_ids=None, align_n=None, align_row_offsets=None, k_extra=0,
-          match_align=False):
+          match_align=False, pool_ids=None, pool_align_ids=None, pool_align_n=None):
+    """``pool_ids``: an external pool (one int32 token sequence shared by all sequences, NONE
+    separates documents), optionally with its own alignment table ``pool_align_ids`` [len x
+    k_extra] / ``pool_align_n`` [len]; candidates from the pool have cand_pos = -2 - place."""
     hist_ids, hist_offsets = _i32(hist_ids), _i32(hist_offsets)
     hist_len, prompt_len = _i32(hist_len), _i32(prompt_len)
     recent_ids, recent_len = _i32(recent_ids), _i32(recent_len)
     align_ids, align_n = _i32(align_ids), _i32(align_n)
     align_row_offsets = _i32(align_row_offsets)
+    pool_ids, pool_align_ids, pool_align_n = _i32(pool_ids), _i32(pool_align_ids), _i32(pool_align_n)
     B = len(hist_len)
     assert recent_ids.size == B * n
     out = dict(draft_ids=np.zeros((B, max_cands, draft_len), np.int32),
@@ -153,6 +157,7 @@ def draft(hist_ids, hist_offsets, hist_len, prompt_len, recent_ids, recent_len, 
         _ptr(hist_ids), _ptr(hist_offsets), _ptr(hist_len), _ptr(prompt_len), _ptr(align_ids),
         _ptr(align_n), _ptr(align_row_offsets), int(k_extra), _ptr(recent_ids),
         _ptr(recent_len), B, int(n), int(draft_len), int(max_cands), int(bool(match_align)),
+        _ptr(pool_ids), 0 if pool_ids is None else int(pool_ids.size), _ptr(pool_align_ids), _ptr(pool_align_n),
         _ptr(out["draft_ids"]), _ptr(out["draft_flags"]), _ptr(out["cand_len"]),
         _ptr(out["cand_pos"]), _ptr(out["n_cands"]), _ptr(out["match_len"]))
     assert rc == 0
@@ -203,7 +208,7 @@ def tree_build(draft_ids, draft_flags, cand_len, n_cands):
 
 
 def verify_tree(logits, node_token, node_parent, tree_offsets, emit_stride, node_flags=None, alpha=0.1,
-                beta=0.1, mode=VERIFY_CONDITIONAL, seed=0, step=0, inv_temperature=1.0, threads=1):
+                beta=0.1, mode=VERIFY_CONDITIONAL, seed=0, step=0, inv_temperature=1.0, threads=1, top_k=5):
     x, code, stride = _logits(logits)
     R, V = x.shape
     tok, par = _i32(node_token).reshape(-1), _i32(node_parent).reshape(-1)
@@ -213,15 +218,15 @@ def verify_tree(logits, node_token, node_parent, tree_offsets, emit_stride, node
     fl = None if node_flags is None else np.ascontiguousarray(node_flags, np.uint8).reshape(-1)
     out = dict(p_token=np.zeros(R), entropy=np.zeros(R), pmax=np.zeros(R), argmax=np.zeros(R, np.int32),
                threshold=np.zeros(R), accept=np.zeros(R, np.uint8), sampled=np.zeros(R, np.int32),
-               near=np.zeros(R, np.uint8), bad=np.zeros(R, np.uint8), best_node=np.zeros(T, np.int32),
-               n_accept=np.zeros(T, np.int32), n_emit=np.zeros(T, np.int32),
+               near=np.zeros(R, np.uint8), bad=np.zeros(R, np.uint8), n_greater=np.zeros(R, np.int32),
+               best_node=np.zeros(T, np.int32), n_accept=np.zeros(T, np.int32), n_emit=np.zeros(T, np.int32),
                emit_ids=np.zeros((T, emit_stride), np.int32))
     rc = lib().oracle_verify_tree(
         _ptr(x), code, _ptr(tok), _ptr(par), _ptr(fl), _ptr(offs), T, C.c_int64(V), C.c_int64(stride),
         C.c_double(alpha), C.c_double(beta), C.c_double(inv_temperature), int(mode), C.c_uint64(seed),
-        C.c_uint32(step), int(threads), int(emit_stride), _ptr(out["p_token"]), _ptr(out["entropy"]),
+        C.c_uint32(step), int(top_k), int(threads), int(emit_stride), _ptr(out["p_token"]), _ptr(out["entropy"]),
         _ptr(out["pmax"]), _ptr(out["argmax"]), _ptr(out["threshold"]), _ptr(out["accept"]),
-        _ptr(out["sampled"]), _ptr(out["near"]), _ptr(out["bad"]), _ptr(out["best_node"]),
+        _ptr(out["sampled"]), _ptr(out["near"]), _ptr(out["bad"]), _ptr(out["n_greater"]), _ptr(out["best_node"]),
         _ptr(out["n_accept"]), _ptr(out["n_emit"]), _ptr(out["emit_ids"]))
     assert rc == 0
     return out

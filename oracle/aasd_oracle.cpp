@@ -13,7 +13,7 @@
 // Pins (tests/test_oracle_*.py): closed forms of softmax/entropy (uniform, one spike,
 // (1/2,1/4,1/8,1/8)), hand-computed thresholds of Eq. 5, the worked alignment examples of
 // Sec. 2.3 and Fig. 2, brute-force sorts and 2^len accept patterns on tiny inputs, a
-// naive double loop for the Algorithm-1 dictionary, published Philox4x32-10 known-answer
+// dictionary of Algorithm 1 and a naive double loop for the lookup, published Philox4x32-10 known-answer
 // vectors and a chi-square test of the sampler against the exact softmax; top-k verification
 // against a full stable sort and the two extreme rows of Sec. 3.3; the draft tree against the
 // set of distinct candidate prefixes, tree verification against the longest passing flat
@@ -361,75 +361,101 @@ int oracle_align_sample(const void* logits, int dtype, const int32_t* prompt_ids
 }
 
 // ---------------------------------------------------------------------------------
-// O-D: context-aware drafting, Algorithm 1 taken literally (Sec. 3.1).
-// pool: for k = 1..n and every window hist[i:i+k], pool[key].append(i+k), i.e. the index
-// right after the key.  Lookup: keys recent[-k:] for k = min(n, recent_len) .. 1, stopping
-// at the first k that has a stored position p with a continuation (p < len).
-// With match_align != 0 the last token of a window may also be one of the alignment
+// O-D: context-aware drafting (Sec. 3.1, Algorithm 1).
+// The draft pool of Algorithm 1 holds, for every k-gram (k <= n) of the current sequence, the
+// places right after its occurrences; the lookup tries the last k tokens of the sequence as
+// the key for k = n, n-1, ..., 1 and stops at the first k that has a place (Sec. 3.1: longer
+// keys first).  Written out as a definition: the match length of a place p (an index into the
+// token sequence, 1 <= p < len, so that a continuation exists) is the largest k <= min(n, p,
+// recent_len) such that the k tokens in front of p equal the key's last k tokens; k* is the
+// largest match length of any place, and the lookup result is every place that reaches it.
+// With match_align != 0 the token right in front of p may also be one of the alignment
 // extras stored for that prompt position (extras of position q live in align row q-1).
-// Candidates: the stored positions in descending order, at most max_cands ("mains"),
-// each continued by hist[p : p+draft_len] clipped at len; then, while slots remain,
-// alternatives in (main, depth i, extra slot s) order = the main's first i tokens plus
-// extra s of position p+i.  Token flags: bit0 = eligible for conditional verification
-// (source index < prompt_len, or an alignment extra), bit1 = alignment extra.
-// Outputs per sequence b: draft_ids/draft_flags [max_cands x draft_len] (NONE / 0
-// padded), cand_len, cand_pos (match position of the main a candidate derives from; NONE
-// for unused slots) [max_cands], n_cands, match_len (k*, 0 when nothing matched).
+// An external pool (Limitations: "most existing retrieval-based speculative decoding") is a
+// second token sequence, shared by all sequences and owned by the caller, that is looked up
+// the same way: its places compete with the history's for k*, a NONE token inside it separates
+// documents (it matches nothing and ends a continuation), and its tokens are not input
+// context, so they are verified strictly (flag 0).  The pool may carry an alignment table of
+// its own (extras of pool position q in row q-1): those extras are alignment-sampled tokens
+// like any other (flags 3).
+// Candidates: the places of the history in descending order, then those of the pool in
+// descending order, at most max_cands ("mains"), each continued by up to draft_len tokens of
+// its source; then, while slots remain, alternatives in (main, depth i, extra slot s) order =
+// the main's first i tokens plus extra s of position p+i.  Token flags: bit0 = eligible for
+// conditional verification (history index < prompt_len, or an alignment extra), bit1 =
+// alignment extra.
+// Outputs per sequence b: draft_ids/draft_flags [max_cands x draft_len] (NONE / 0 padded),
+// cand_len, cand_pos (place of the main a candidate derives from: p for the history,
+// -2 - p for the pool; NONE for unused slots) [max_cands], n_cands, match_len (k*, 0 when
+// nothing matched).
 // ---------------------------------------------------------------------------------
 int oracle_draft(const int32_t* hist_ids, const int32_t* hist_offsets, const int32_t* hist_len,
                  const int32_t* prompt_len, const int32_t* align_ids, const int32_t* align_n,
                  const int32_t* align_row_offsets, int K, const int32_t* recent_ids,
                  const int32_t* recent_len, int32_t B, int n, int draft_len, int max_cands,
-                 int match_align, int32_t* draft_ids, uint8_t* draft_flags, int32_t* cand_len,
-                 int32_t* cand_pos, int32_t* n_cands, int32_t* match_len) {
-    if (n < 1 || draft_len < 1 || max_cands < 1 || B < 0) return 1;
+                 int match_align, const int32_t* pool_ids, int32_t pool_len,
+                 const int32_t* pool_align_ids, const int32_t* pool_align_n, int32_t* draft_ids,
+                 uint8_t* draft_flags, int32_t* cand_len, int32_t* cand_pos, int32_t* n_cands,
+                 int32_t* match_len) {
+    if (n < 1 || draft_len < 1 || max_cands < 1 || B < 0 || pool_len < 0) return 1;
     const bool have_align = (align_ids != nullptr && align_n != nullptr && K > 0);
+    const bool have_pool = (pool_ids != nullptr && pool_len > 0);
+    const bool have_pool_align = have_pool && pool_align_ids != nullptr && pool_align_n != nullptr && K > 0;
     for (int32_t b = 0; b < B; ++b) {
         const int32_t* h = hist_ids + hist_offsets[b];
         const int32_t len = hist_len[b];
         const int32_t plen = prompt_len[b];
         const int32_t* rec = recent_ids + (int64_t)b * n;
-        const int32_t rl = recent_len[b];
+        const int32_t rl = std::max<int32_t>(0, std::min<int32_t>(n, recent_len[b]));
         const int64_t arow0 = have_align ? (int64_t)align_row_offsets[b] : 0;
-        // extras stored for prompt position q
+        // extras stored for prompt position q / pool position q
         auto n_ext = [&](int32_t q) -> int {
             if (!have_align || q < 1 || q >= plen) return 0;
             return align_n[arow0 + q - 1];
         };
         auto ext = [&](int32_t q, int s) -> int32_t { return align_ids[(arow0 + q - 1) * K + s]; };
-
-        std::map<std::vector<int32_t>, std::vector<int32_t>> pool;
-        for (int k = 1; k <= n; ++k) {
-            for (int32_t i = 0; i + k <= len; ++i) {
-                std::vector<int32_t> key(h + i, h + i + k);
-                pool[key].push_back(i + k);
-                if (match_align) {
-                    int32_t q = i + k - 1;
-                    for (int s = 0; s < n_ext(q); ++s) {
-                        std::vector<int32_t> key2 = key;
-                        key2[k - 1] = ext(q, s);
-                        pool[key2].push_back(i + k);
-                    }
-                }
+        auto n_pool_ext = [&](int32_t q) -> int {
+            if (!have_pool_align || q < 1 || q >= pool_len) return 0;
+            return pool_align_n[q - 1];
+        };
+        auto pool_ext = [&](int32_t q, int s) -> int32_t { return pool_align_ids[(int64_t)(q - 1) * K + s]; };
+        // match length of place p of the history
+        auto hist_match = [&](int32_t p) -> int {
+            int m = 0;
+            for (int k = 1; k <= std::min<int>(std::min<int>(n, p), rl); ++k) {
+                const int32_t q = p - k, want = rec[rl - k];
+                bool same = (h[q] == want);
+                if (!same && k == 1 && match_align)
+                    for (int s = 0; s < n_ext(q); ++s) same |= (ext(q, s) == want);
+                if (!same) break;
+                m = k;
             }
-        }
-        std::vector<int32_t> found;
+            return m;
+        };
+        // and of place p of the pool (NONE separates documents: it equals no key token)
+        auto pool_match = [&](int32_t p) -> int {
+            int m = 0;
+            for (int k = 1; k <= std::min<int>(std::min<int>(n, p), rl); ++k) {
+                const int32_t t = pool_ids[p - k];
+                if (t == NONE || t != rec[rl - k]) break;
+                m = k;
+            }
+            return m;
+        };
         int kstar = 0;
-        for (int k = std::min(n, (int)rl); k >= 1; --k) {
-            std::vector<int32_t> key(rec + rl - k, rec + rl);
-            auto it = pool.find(key);
-            if (it == pool.end()) continue;
-            std::vector<int32_t> with_cont;
-            for (int32_t p : it->second)
-                if (p < len) with_cont.push_back(p);
-            if (with_cont.empty()) continue;
-            found = with_cont;
-            kstar = k;
-            break;
+        for (int32_t p = 1; p < len; ++p) kstar = std::max(kstar, hist_match(p));
+        if (have_pool)
+            for (int32_t p = 1; p < pool_len; ++p)
+                if (pool_ids[p] != NONE) kstar = std::max(kstar, pool_match(p));
+        // places that reach k*: (source, p), history first, most recent first within a source
+        std::vector<std::pair<int, int32_t>> found;
+        if (kstar > 0) {
+            for (int32_t p = len - 1; p >= 1; --p)
+                if (hist_match(p) == kstar) found.push_back({0, p});
+            if (have_pool)
+                for (int32_t p = pool_len - 1; p >= 1; --p)
+                    if (pool_ids[p] != NONE && pool_match(p) == kstar) found.push_back({1, p});
         }
-        // descending position, duplicates (possible with match_align) removed
-        std::sort(found.begin(), found.end(), [](int32_t a, int32_t c) { return a > c; });
-        found.erase(std::unique(found.begin(), found.end()), found.end());
 
         int32_t* d_ids = draft_ids + (int64_t)b * max_cands * draft_len;
         uint8_t* d_fl = draft_flags + (int64_t)b * max_cands * draft_len;
@@ -443,32 +469,44 @@ int oracle_draft(const int32_t* hist_ids, const int32_t* hist_offsets, const int
             c_len[c] = 0;
             c_pos[c] = NONE;
         }
-        int n_main = std::min<int>((int)found.size(), max_cands);
+        const int n_main = std::min<int>((int)found.size(), max_cands);
         int total = 0;
         for (int c = 0; c < n_main; ++c) {
-            int32_t p = found[c];
-            int32_t L = std::min<int32_t>(draft_len, len - p);
-            for (int32_t i = 0; i < L; ++i) {
-                d_ids[c * draft_len + i] = h[p + i];
-                d_fl[c * draft_len + i] = (p + i < plen) ? 1 : 0;
+            const bool from_pool = found[c].first == 1;
+            const int32_t p = found[c].second;
+            int32_t L = 0;
+            if (!from_pool) {
+                L = std::min<int32_t>(draft_len, len - p);
+                for (int32_t i = 0; i < L; ++i) {
+                    d_ids[c * draft_len + i] = h[p + i];
+                    d_fl[c * draft_len + i] = (p + i < plen) ? 1 : 0;
+                }
+            } else {
+                while (L < draft_len && p + L < pool_len && pool_ids[p + L] != NONE) {
+                    d_ids[c * draft_len + L] = pool_ids[p + L];
+                    d_fl[c * draft_len + L] = 0;
+                    ++L;
+                }
             }
             c_len[c] = L;
-            c_pos[c] = p;
+            c_pos[c] = from_pool ? -2 - p : p;
             ++total;
         }
         for (int c = 0; c < n_main && total < max_cands; ++c) {
-            int32_t p = found[c];
+            const bool from_pool = found[c].first == 1;
+            const int32_t p = found[c].second;
             for (int32_t i = 0; i < c_len[c] && total < max_cands; ++i) {
-                for (int s = 0; s < n_ext(p + i) && total < max_cands; ++s) {
+                const int ne = from_pool ? n_pool_ext(p + i) : n_ext(p + i);
+                for (int s = 0; s < ne && total < max_cands; ++s) {
                     int slot = total++;
                     for (int32_t q = 0; q < i; ++q) {
                         d_ids[slot * draft_len + q] = d_ids[c * draft_len + q];
                         d_fl[slot * draft_len + q] = d_fl[c * draft_len + q];
                     }
-                    d_ids[slot * draft_len + i] = ext(p + i, s);
+                    d_ids[slot * draft_len + i] = from_pool ? pool_ext(p + i, s) : ext(p + i, s);
                     d_fl[slot * draft_len + i] = 3;
                     c_len[slot] = i + 1;
-                    c_pos[slot] = p;
+                    c_pos[slot] = c_pos[c];
                 }
             }
         }
@@ -631,7 +669,10 @@ int oracle_tree_build(const int32_t* draft_ids, const uint8_t* draft_flags, cons
 // so the token of node v is judged by the row of its parent, with the rules of O-V (modes
 // 0-2).  A node passes when it and all its ancestors are accepted (prefix rule, Sec. 2.1);
 // the result of a tree is its deepest passing node (ties: lowest node index; the root when
-// nothing passes): "the longest draft candidate that passes verification".  Emitted: the
+// nothing passes): "the longest draft candidate that passes verification".  Mode 3 (TOP_K,
+// the alternative of Sec. 3.3): an eligible node passes iff fewer than top_k tokens of its
+// parent's row are ahead of its token in the order (logit desc, id asc) and the token is not
+// masked; n_greater[node] is that count (NONE for roots, NONE / masked tokens, bad rows).  Emitted: the
 // tokens on the path to that node, followed by the target's own token of that node's row.
 // Trees are CSR ranges of nodes (tree_offsets[T+1]); node_parent holds indices inside the
 // tree (NONE for the root, which is node 0 of its tree); parents precede children.
@@ -643,11 +684,11 @@ int oracle_verify_tree(const void* logits, int dtype, const int32_t* node_token,
                        const int32_t* node_parent, const uint8_t* node_flags,
                        const int32_t* tree_offsets, int32_t T, int64_t V, int64_t row_stride,
                        double alpha, double beta, double invT, int mode, uint64_t seed, uint32_t step,
-                       int threads, int emit_stride, double* p_token, double* entropy, double* pmax,
+                       int top_k, int threads, int emit_stride, double* p_token, double* entropy, double* pmax,
                        int32_t* argmax, double* threshold, uint8_t* accept, int32_t* sampled,
-                       uint8_t* near, uint8_t* bad, int32_t* best_node, int32_t* n_accept,
+                       uint8_t* near, uint8_t* bad, int32_t* n_greater, int32_t* best_node, int32_t* n_accept,
                        int32_t* n_emit, int32_t* emit_ids) {
-    if (T < 0 || V <= 0 || mode < 0 || mode > 2 || emit_stride < 1) return 1;
+    if (T < 0 || V <= 0 || mode < 0 || mode > 3 || emit_stride < 1) return 1;
     Rows X{logits, dtype, row_stride};
     const int64_t R = tree_offsets[T];
     std::vector<RowStats> st(R);
@@ -677,6 +718,7 @@ int oracle_verify_tree(const void* logits, int dtype, const int32_t* node_token,
             const int32_t par = node_parent[g];
             double pt = 0.0;
             bool a = false, is_near = false;
+            int32_t ahead_of_d = NONE;
             if (v == 0 || par < 0 || par >= v) {   // the root (or a malformed node: never passes)
                 ok[v] = (v == 0);
             } else {
@@ -686,11 +728,19 @@ int oracle_verify_tree(const void* logits, int dtype, const int32_t* node_token,
                 const uint8_t f = node_flags ? node_flags[g] : 1;
                 if (!ps.bad && d != NONE) {
                     pt = prob_of(X, lo + par, d, invT, ps);
+                    const double yd = X.at(lo + par, d) * invT;
+                    if (yd != -std::numeric_limits<double>::infinity()) {   // a masked token has no rank
+                        ahead_of_d = 0;
+                        for (int64_t i = 0; i < V; ++i)
+                            if (i != d && ahead(X.at(lo + par, i) * invT, i, yd, d)) ++ahead_of_d;
+                    }
                     if (mode == 0 && (f & 1)) {
                         const double lin = alpha * ps.H + beta;
                         const bool at_max = (X.at(lo + par, d) * invT == ps.m);
                         a = at_max || (pt >= lin);
                         is_near = !at_max && std::fabs(pt - lin) <= 1e-6;
+                    } else if (mode == 3 && (f & 1)) {
+                        a = ahead_of_d != NONE && ahead_of_d < top_k;
                     } else {
                         a = (d == own[lo + par]);
                     }
@@ -702,6 +752,7 @@ int oracle_verify_tree(const void* logits, int dtype, const int32_t* node_token,
             if (p_token) p_token[g] = pt;
             if (accept) accept[g] = a ? 1 : 0;
             if (near) near[g] = is_near ? 1 : 0;
+            if (n_greater) n_greater[g] = ahead_of_d;
         }
         if (n == 0) {
             if (best_node) best_node[t] = NONE;

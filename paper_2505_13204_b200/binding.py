@@ -30,7 +30,7 @@ EXPORTS = [
     "aasd_get_counters", "aasd_reset_counters", "aasd_launch_count", "aasd_workspace_bytes",
     "aasd_workspace_init", "aasd_workspace_release", "aasd_align_sample", "aasd_draft",
     "aasd_verify", "aasd_select", "aasd_append", "aasd_step", "aasd_verify_static",
-    "aasd_tree_build", "aasd_verify_tree", "aasd_probe_read",
+    "aasd_tree_build", "aasd_verify_tree", "aasd_probe_read", "aasd_debug_withhold_tile",
 ]
 STATIC_MAX_ROWS = STATIC_MAX_CANDS = 8192
 
@@ -136,6 +136,7 @@ def load_library(path: str | None = None):
                                      C.POINTER(VerifyParams), C.c_int32, _vp, C.c_size_t,
                                      C.POINTER(TreeOut)]
     lib.aasd_probe_read.argtypes = [_vp, _vp, C.c_size_t, _vp]
+    lib.aasd_debug_withhold_tile.argtypes = [_vp, C.c_int64, C.c_int32, C.c_uint32]
     lib.aasd_verify_static.argtypes = [C.c_int, _vp, _vp, _vp, _vp, _vp, C.c_int32, C.c_int64,
                                        C.POINTER(VerifyParams), C.POINTER(VerifyOut), _vp]
     if path == _build.LIB:
@@ -268,6 +269,19 @@ class Context:
 
     def launch_count(self) -> int:
         return int(self.lib.aasd_launch_count(self._h))
+
+    def debug_withhold_tile(self, item: int, tile: int, wait_limit: int):
+        """aasd_debug_withhold_tile: the next streaming launch never copies one tile and gives
+        up its waits after ``wait_limit`` polls (a testing aid, see include/aasd.h)."""
+        _check(self.lib.aasd_debug_withhold_tile(self._h, int(item), int(tile), int(wait_limit)),
+               "aasd_debug_withhold_tile")
+
+    def reinit_workspace(self):
+        """Registers the context's own workspace again (clears it): required after a launch
+        that ended with STATUS_TIMEOUT."""
+        if self._ws is not None:
+            _check(self.lib.aasd_workspace_init(self._h, _vp(self._ws.data_ptr()), self._ws.numel(),
+                                                self._ws_rows, self._ws_cands), "aasd_workspace_init")
 
     def new_workspace(self, rows: int, cands: int) -> torch.Tensor:
         """Allocates and registers a workspace for ``rows`` logits rows and ``cands`` candidates."""
@@ -543,9 +557,22 @@ class DecodeState:
             a.table_ids, a.table_n = _p(align["align_ids"]), _p(align["n_extra"])
         self.args = a
 
-    def run_draft(self):
-        """Only the drafting part of a step (so that a stand-in model can be run on it)."""
+    def run_draft(self, recent_ids=None, recent_len=None):
+        """Only the drafting part of a step (so that a stand-in model can be run on it).
+        ``recent_ids`` (int32 [B x n] on the device, with ``recent_len`` [B]) gives the keys
+        explicitly; None: every history's own tail is the key."""
         a = self.args
+        if recent_ids is not None:
+            assert recent_ids.dtype == torch.int32 and recent_ids.is_cuda and recent_ids.is_contiguous()
+            assert tuple(recent_ids.shape) == (self.B, self.n)
+            if recent_len is None:
+                recent_len = torch.full((self.B,), self.n, dtype=torch.int32, device=recent_ids.device)
+            assert recent_len.dtype == torch.int32 and recent_len.is_cuda
+            self._recent = (recent_ids, recent_len)     # kept alive until the next call
+        else:
+            self._recent = (None, None)
+        a.draft_in.recent_ids = _p(self._recent[0])
+        a.draft_in.recent_len = _p(self._recent[1])
         _check(self.ctx.lib.aasd_draft(self.ctx._h, C.byref(a.draft_in), C.byref(a.draft),
                                        C.byref(a.draft_out)), "aasd_draft")
         return self.draft_out

@@ -11,11 +11,10 @@
 #include <mutex>
 #include <new>
 
-#include "../../include/aasd.h"
-#include "aasd_rows.cuh"
-#include "aasd_stream.cuh"
+// this translation unit holds the kernels that are not templates (see AASD_HOST_TU in the headers)
+#define AASD_HOST_TU 1
+#include "aasd_host.h"
 #include "aasd_tokens.cuh"
-#include "aasd_tree.cuh"
 
 using namespace aasd;
 
@@ -25,54 +24,23 @@ struct TraceRange {
     explicit TraceRange(const char* name) { nvtxRangePushA(name); }
     ~TraceRange() { nvtxRangePop(); }
 };
-}  // namespace
 
-namespace {
-
-struct WorkspaceLayout {
-    size_t bytes;
-    int64_t max_rows, max_cands;
-    size_t off_partials, off_row_tickets, off_cand_tickets, off_seq_tickets, off_sched, off_row_accept, off_row_own, off_next, off_race,
-        off_tree_stats, off_row_extra;
-    bool full;
+// Two environment switches for measurements and tests, read once per context:
+// AASD_NO_CLUSTER=1 sends the pieces of cut rows through global memory instead of a cluster's
+// shared memory, AASD_STREAM_CHUNKS=n sets the piece count of scarce rows.
+struct Tuning {
+    bool no_cluster;
+    long stream_chunks;   // 0: the library's own choice
 };
-
-size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
-
-// with_tree: room for the per-row statistics of tree verification and for the per-row extras
-// of the table extension (the fixed block of aasd_verify_static does without both).
-WorkspaceLayout make_layout(int64_t max_rows, int64_t max_cands, bool with_tree = true) {
-    WorkspaceLayout L{};
-    L.max_rows = max_rows;
-    L.max_cands = max_cands;
-    size_t o = 0;
-    L.off_partials = o;
-    o = align_up(o + sizeof(RowPartial) * (size_t)kPartialSlots, 256);
-    L.off_row_tickets = o;
-    o = align_up(o + 4 * (size_t)max_rows, 256);
-    L.off_cand_tickets = o;
-    o = align_up(o + 4 * (size_t)max_cands, 256);
-    L.off_seq_tickets = o;
-    o = align_up(o + 4 * (size_t)max_cands, 256);
-    L.off_sched = o;
-    o = align_up(o + 2 * sizeof(unsigned int), 256);
-    L.off_row_accept = o;
-    o = align_up(o + (size_t)max_rows, 256);
-    L.off_row_own = o;
-    o = align_up(o + 8 * (size_t)max_rows, 256);
-    L.off_next = o;
-    o = align_up(o + 4 * (size_t)max_rows, 256);
-    L.off_race = o;
-    o = align_up(o + sizeof(RaceSummary) * (size_t)kRaceSlots * kMaxK, 256);
-    L.off_tree_stats = o;
-    if (with_tree) o = align_up(o + sizeof(TreeRowStat) * (size_t)max_rows, 256);
-    L.off_row_extra = o;
-    if (with_tree) o = align_up(o + 12 * (size_t)max_rows, 256);
-    L.full = with_tree;
-    L.bytes = o;
-    return L;
+Tuning read_tuning() {
+    Tuning t{};
+    t.no_cluster = getenv("AASD_NO_CLUSTER") != nullptr;
+    if (const char* e = getenv("AASD_STREAM_CHUNKS")) {
+        const long v = atol(e);
+        if (v >= 1) t.stream_chunks = v;
+    }
+    return t;
 }
-
 }  // namespace
 
 struct aasd_ctx {
@@ -81,48 +49,15 @@ struct aasd_ctx {
     int sm_count;
     DeviceState* state;
     uint64_t launches;
+    Tuning tuning;
     std::map<void*, WorkspaceLayout> workspaces;
+    // testing aid, armed by aasd_debug_withhold_tile and used up by the next streaming launch
+    long long withhold_item = -1;
+    int withhold_tile = 0;
+    unsigned int test_wait_limit = 0;
 };
 
 namespace {
-
-#define AASD_CUDA(call)                                   \
-    do {                                                  \
-        cudaError_t e__ = (call);                         \
-        if (e__ != cudaSuccess) return AASD_ERR_CUDA;     \
-    } while (0)
-
-// Every kernel of the library is launched with programmatic stream serialization: it may be
-// scheduled while its predecessor in the stream drains, and waits (griddepcontrol.wait,
-// first thing in each kernel) for that predecessor to complete before it touches memory.
-// cluster > 1: the grid is made of thread-block clusters of that many CTAs.
-template <class... Params, class... Args>
-void launch_clustered(void (*kernel)(Params...), unsigned int grid, unsigned int block, size_t smem,
-                      cudaStream_t stream, unsigned int cluster, Args&&... args) {
-    cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3(grid, 1, 1);
-    cfg.blockDim = dim3(block, 1, 1);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[2];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.numAttrs = 1;
-    if (cluster > 1) {
-        attr[1].id = cudaLaunchAttributeClusterDimension;
-        attr[1].val.clusterDim.x = cluster;
-        attr[1].val.clusterDim.y = 1;
-        attr[1].val.clusterDim.z = 1;
-        cfg.numAttrs = 2;
-    }
-    cfg.attrs = attr;
-    cudaLaunchKernelEx(&cfg, kernel, Params(args)...);   // errors surface in cudaGetLastError
-}
-template <class... Params, class... Args>
-void launch(void (*kernel)(Params...), unsigned int grid, unsigned int block, size_t smem, cudaStream_t stream,
-            Args&&... args) {
-    launch_clustered(kernel, grid, block, smem, stream, 1u, static_cast<Args&&>(args)...);
-}
 
 int after_launch(aasd_ctx* ctx, int n) {
     ctx->launches += (uint64_t)n;
@@ -160,6 +95,8 @@ int plan_rows(aasd_ctx* ctx, RowJob& job, const void* logits, int dtype, int voc
     job.vocab = vocab;
     job.vector_ok = ((uintptr_t)logits % 16 == 0) && ((row_stride * esize) % 16 == 0);
     job.nvec = job.vector_ok ? vocab / vec : 0;
+    // a row that starts anywhere has at most vec - 1 tokens in front of its first 16-byte boundary
+    job.stream_nvec = job.vector_ok ? job.nvec : ((int64_t)vocab * esize >= 256 ? (vocab - (vec - 1)) / vec : 0);
     job.vec_elts = vec;
     job.c1 = inv_temperature * kLog2e;
     // Fill the machine: aim at eight CTAs per SM, but keep at least one sweep of the CTA
@@ -186,7 +123,14 @@ int plan_rows(aasd_ctx* ctx, RowJob& job, const void* logits, int dtype, int voc
     return AASD_OK;
 }
 
-// Geometry of the persistent streaming launch over 16-byte aligned rows: a grid of two CTAs
+// Which rows the persistent streaming kernel takes: 16-byte aligned layouts always; any other
+// element-aligned layout too (every row is then streamed from its own first 16-byte boundary)
+// unless the launch samples, since the sampler's groups of 32 ids are tied to the vectors.
+bool stream_path(const RowJob& job, bool sampling) {
+    return job.vector_ok ? job.nvec > 0 : (!sampling && job.stream_nvec > 0);
+}
+
+// Geometry of the persistent streaming launch: a grid of two CTAs
 // per SM that claim work items from a counter.  An item is a whole row unless there are
 // fewer rows than CTA slots; then every row is cut into pieces at tile boundaries.
 void plan_stream(aasd_ctx* ctx, StreamJob& sj, const RowJob& job, const int32_t* hint_ids, char* ws,
@@ -197,7 +141,9 @@ void plan_stream(aasd_ctx* ctx, StreamJob& sj, const RowJob& job, const int32_t*
     sj.race_partials = reinterpret_cast<RaceSummary*>(ws + L.off_race);
     sj.full_groups = (int)(((int64_t)job.nvec * job.vec_elts) / kGroup);
     if (smp) sj.smp = *smp;
-    const int64_t row_bytes = (int64_t)job.nvec * 16;
+    // (rows that are not aligned may hold one vector more than this: a piece count that suits
+    // the smaller figure suits them too)
+    const int64_t row_bytes = (int64_t)job.stream_nvec * 16;
     const int tiles = (int)((row_bytes + kTileBytes - 1) / kTileBytes);
     const int64_t slots = (int64_t)ctx->sm_count * 2;
     // Cutting a row costs its pieces a trip through global memory (partial record, fence,
@@ -209,10 +155,7 @@ void plan_stream(aasd_ctx* ctx, StreamJob& sj, const RowJob& job, const int32_t*
         tail_rows = job.n_rows;
         chunks = slots / (2 * job.n_rows);
         if (chunks > 8) chunks = 8;
-        if (const char* e = getenv("AASD_STREAM_CHUNKS")) {   // tuning override
-            const long v = atol(e);
-            if (v >= 1) chunks = v;
-        }
+        if (ctx->tuning.stream_chunks >= 1) chunks = ctx->tuning.stream_chunks;   // tuning override
     }
     if (chunks > tiles) chunks = tiles;
     if (chunks <= 1) {
@@ -224,6 +167,17 @@ void plan_stream(aasd_ctx* ctx, StreamJob& sj, const RowJob& job, const int32_t*
         chunks = 1;
         tail_rows = 0;
     }
+    sj.wait_limit = kWaitLimit;
+    sj.withhold_item = -1;
+    sj.withhold_tile = 0;
+    if (ctx->withhold_item >= 0) {
+        sj.wait_limit = ctx->test_wait_limit;
+        sj.withhold_item = ctx->withhold_item;
+        sj.withhold_tile = ctx->withhold_tile;
+        ctx->withhold_item = -1;
+        // one CTA per piece of a row would wait for the withheld piece at a cluster barrier
+        // as well; the aid is about the waits of one CTA, so such a launch goes without clusters
+    }
     sj.tiles_per_row = tiles;
     sj.whole_rows = (int)(job.n_rows - tail_rows);
     sj.tail_chunks = (int)chunks;
@@ -233,84 +187,12 @@ void plan_stream(aasd_ctx* ctx, StreamJob& sj, const RowJob& job, const int32_t*
     // cluster and meet in its first CTA's shared memory.  (The sampler's per-piece records
     // travel through global memory, so sampling launches stay as they are.)
     sj.cluster_pieces = (chunks > 1 && chunks <= kMaxCluster && tail_rows == job.n_rows && smp == nullptr &&
-                         (int64_t)*grid == sj.n_items && getenv("AASD_NO_CLUSTER") == nullptr)
+                         (int64_t)*grid == sj.n_items && sj.withhold_item < 0 && !ctx->tuning.no_cluster)
                             ? 1
                             : 0;
 }
 
-template <class Kernel>
-int enable_stream_smem(Kernel kernel) {
-    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStreamSmemBytes) ==
-                   cudaSuccess
-               ? AASD_OK
-               : AASD_ERR_CUDA;
-}
-
-// One launch of the streaming kernel.  Rows that stream faster than a finisher gets through
-// one (short_rows) take the variant with three finisher warps; sampling kernels, whose
-// consumers are the slower side, always run with one.
-template <int DT, int K, int ND, bool TK, bool FIN, class E>
-int launch_stream(aasd_ctx* ctx, const StreamJob& sj, const typename E::Args& a, unsigned int grid, bool short_rows) {
-    const unsigned int cluster = sj.cluster_pieces ? (unsigned int)sj.tail_chunks : 1u;
-    if (ND == 0 && short_rows) {
-        auto kernel = stream_kernel<DT, K, ND, TK, FIN, E, (ND == 0 ? kShortRowFinishers : 1)>;
-        if (enable_stream_smem(kernel) != AASD_OK) return AASD_ERR_CUDA;
-        launch_clustered(kernel, grid, stream_threads(kShortRowFinishers), kStreamSmemBytes, ctx->stream, cluster, sj, a);
-        return AASD_OK;
-    }
-    auto kernel = stream_kernel<DT, K, ND, TK, FIN, E, 1>;
-    if (enable_stream_smem(kernel) != AASD_OK) return AASD_ERR_CUDA;
-    launch_clustered(kernel, grid, stream_threads(1), kStreamSmemBytes, ctx->stream, cluster, sj, a);
-    return AASD_OK;
-}
-// bytes of a row below which the finisher, not the copy, paces a CTA (measured: a verification
-// row costs a finisher about 7 us under load, an alignment row 5 us; a CTA streams 25 GB/s)
-constexpr int64_t kShortVerifyRow = 200 * 1024;
-constexpr int64_t kShortAlignRow = 96 * 1024;
-inline int64_t row_bytes_of(const StreamJob& sj) { return (int64_t)sj.row.nvec * 16; }
-
-template <int DT, int K, int ND, bool FIN = false>
-int launch_align_stream(aasd_ctx* ctx, const StreamJob& sj, const AlignArgs& a, unsigned int grid) {
-    return launch_stream<DT, K, ND, false, FIN, AlignEpilogue<DT>>(ctx, sj, a, grid, row_bytes_of(sj) < kShortAlignRow);
-}
-
-// TOPK mode keeps the K best tokens and draws nothing; GUMBEL mode needs the best token
-// only (for the alignment test) and prepares ND >= k_extra draws.
-template <int DT>
-int dispatch_align_stream(aasd_ctx* ctx, const StreamJob& sj, const AlignArgs& a, unsigned int grid) {
-    const int k = a.k_extra <= 1 ? 1 : (a.k_extra == 2 ? 2 : 4);
-    if (a.mode == AASD_ALIGN_GUMBEL && a.k_extra > 0) {
-        if (k == 1) return launch_align_stream<DT, 1, 1>(ctx, sj, a, grid);
-        if (k == 2) return launch_align_stream<DT, 1, 2>(ctx, sj, a, grid);
-        return launch_align_stream<DT, 1, 4>(ctx, sj, a, grid);
-    }
-    if (a.hints & AASD_HINT_FINITE) {
-        if (k == 1) return launch_align_stream<DT, 1, 0, true>(ctx, sj, a, grid);
-        if (k == 2) return launch_align_stream<DT, 2, 0, true>(ctx, sj, a, grid);
-        return launch_align_stream<DT, 4, 0, true>(ctx, sj, a, grid);
-    }
-    if (k == 1) return launch_align_stream<DT, 1, 0>(ctx, sj, a, grid);
-    if (k == 2) return launch_align_stream<DT, 2, 0>(ctx, sj, a, grid);
-    return launch_align_stream<DT, 4, 0>(ctx, sj, a, grid);
-}
-
-template <int DT, int ND, bool TK, bool FIN = false, int K = 1>
-int launch_verify_stream(aasd_ctx* ctx, const StreamJob& sj, const VerifyArgs& a, unsigned int grid) {
-    return launch_stream<DT, K, ND, TK, FIN, VerifyEpilogue<DT>>(ctx, sj, a, grid, row_bytes_of(sj) < kShortVerifyRow);
-}
-
-template <int DT>
-int dispatch_verify_stream(aasd_ctx* ctx, const StreamJob& sj, const VerifyArgs& a, unsigned int grid) {
-    if (a.row_extra) {
-        // the table extension wants the two best tokens of every row
-        if (a.hints & AASD_HINT_FINITE) return launch_verify_stream<DT, 0, false, true, 2>(ctx, sj, a, grid);
-        return launch_verify_stream<DT, 0, false, false, 2>(ctx, sj, a, grid);
-    }
-    if (a.mode == AASD_VERIFY_STRICT_SAMPLED) return launch_verify_stream<DT, 1, false>(ctx, sj, a, grid);
-    if (a.mode == AASD_VERIFY_TOP_K) return launch_verify_stream<DT, 0, true>(ctx, sj, a, grid);
-    if (a.hints & AASD_HINT_FINITE) return launch_verify_stream<DT, 0, false, true>(ctx, sj, a, grid);
-    return launch_verify_stream<DT, 0, false>(ctx, sj, a, grid);
-}
+LaunchEnv env_of(const aasd_ctx* ctx) { return LaunchEnv{ctx->stream, ctx->device}; }
 
 SampleJob make_sample_job(uint64_t seed, uint32_t step, bool align, float inv_temperature) {
     SampleJob s{};
@@ -356,6 +238,7 @@ int aasd_create(aasd_ctx** out, int device, void* stream) {
     ctx->stream = static_cast<cudaStream_t>(stream);
     ctx->sm_count = prop.multiProcessorCount;
     ctx->launches = 0;
+    ctx->tuning = read_tuning();
     if (cudaMalloc(&ctx->state, sizeof(DeviceState)) != cudaSuccess) {
         delete ctx;
         return AASD_ERR_CUDA;
@@ -461,29 +344,22 @@ int aasd_align_sample(aasd_ctx* ctx, const void* prefill_logits, const int32_t* 
     a.out = *out;
     AASD_CUDA(cudaSetDevice(ctx->device));
     launch(align_next_kernel, (unsigned int)((n_rows + 255) / 256), 256, 0, ctx->stream, a);
-    // plain kernels: the K best tokens in TOPK mode, the best token alone in GUMBEL mode
-    const int K = (p->k_extra <= 1 || p->mode == AASD_ALIGN_GUMBEL) ? 1 : (p->k_extra == 2 ? 2 : 4);
-    if (a.job.vector_ok && a.job.nvec > 0) {
-        // 16-byte aligned rows: persistent TMA-fed streaming kernel
+    const bool f32 = p->dtype == AASD_F32;
+    const bool draws = p->mode == AASD_ALIGN_GUMBEL && p->k_extra > 0;
+    const LaunchEnv env = env_of(ctx);
+    int rc = AASD_OK;
+    if (stream_path(a.job, draws)) {
+        // persistent TMA-fed streaming kernel
         StreamJob sj{};
         unsigned int grid = 0;
-        const bool draws = p->mode == AASD_ALIGN_GUMBEL && p->k_extra > 0;
         plan_stream(ctx, sj, a.job, a.next_ids, ws, *L, draws ? &a.smp : nullptr, &grid);
-        const int rc = p->dtype == AASD_F32 ? dispatch_align_stream<AASD_F32>(ctx, sj, a, grid)
-                                            : dispatch_align_stream<AASD_BF16>(ctx, sj, a, grid);
-        if (rc != AASD_OK) return rc;
-        return after_launch(ctx, 2);
-    }
-    const unsigned int grid = (unsigned int)(n_rows * a.job.chunks);
-    if (p->dtype == AASD_F32) {
-        if (K == 1) launch(align_kernel<AASD_F32, 1>, grid, kThreads, 0, ctx->stream, a);
-        else if (K == 2) launch(align_kernel<AASD_F32, 2>, grid, kThreads, 0, ctx->stream, a);
-        else launch(align_kernel<AASD_F32, 4>, grid, kThreads, 0, ctx->stream, a);
+        if (draws) rc = f32 ? launch_align_gumbel_f32(env, sj, a, grid) : launch_align_gumbel_bf16(env, sj, a, grid);
+        else rc = f32 ? launch_align_topk_f32(env, &sj, a, grid) : launch_align_topk_bf16(env, &sj, a, grid);
     } else {
-        if (K == 1) launch(align_kernel<AASD_BF16, 1>, grid, kThreads, 0, ctx->stream, a);
-        else if (K == 2) launch(align_kernel<AASD_BF16, 2>, grid, kThreads, 0, ctx->stream, a);
-        else launch(align_kernel<AASD_BF16, 4>, grid, kThreads, 0, ctx->stream, a);
+        const unsigned int grid = (unsigned int)(n_rows * a.job.chunks);
+        rc = f32 ? launch_align_topk_f32(env, nullptr, a, grid) : launch_align_topk_bf16(env, nullptr, a, grid);
     }
+    if (rc != AASD_OK) return rc;
     return after_launch(ctx, 2);
 }
 
@@ -551,7 +427,7 @@ int verify_impl(aasd_ctx* ctx, const void* target_logits, const int32_t* draft_i
         a.seq.enabled = 1;
         a.seq.seq_tickets = reinterpret_cast<unsigned int*>(ws + L->off_seq_tickets);
         if (seq->table_ids) {
-            if (!L->full || !(a.job.vector_ok && a.job.nvec > 0)) return AASD_ERR_UNSUPPORTED;
+            if (!L->full || !stream_path(a.job, false)) return AASD_ERR_UNSUPPORTED;
             a.row_extra = reinterpret_cast<int32_t*>(ws + L->off_row_extra);
         }
     }
@@ -561,18 +437,19 @@ int verify_impl(aasd_ctx* ctx, const void* target_logits, const int32_t* draft_i
         launch(verify_empty_kernel, (unsigned int)((n_cands + 255) / 256), 256, 0, ctx->stream, a);
         return after_launch(ctx, 1);
     }
-    if (a.job.vector_ok && a.job.nvec > 0) {
+    const bool f32 = p->dtype == AASD_F32;
+    const LaunchEnv env = env_of(ctx);
+    int rc = AASD_OK;
+    if (stream_path(a.job, p->mode == AASD_VERIFY_STRICT_SAMPLED)) {
         StreamJob sj{};
         unsigned int sgrid = 0;
         plan_stream(ctx, sj, a.job, draft_ids, ws, *L, p->mode == AASD_VERIFY_STRICT_SAMPLED ? &a.smp : nullptr, &sgrid);
-        const int rc = p->dtype == AASD_F32 ? dispatch_verify_stream<AASD_F32>(ctx, sj, a, sgrid)
-                                            : dispatch_verify_stream<AASD_BF16>(ctx, sj, a, sgrid);
-        if (rc != AASD_OK) return rc;
-        return after_launch(ctx, 1);
+        rc = f32 ? launch_verify_f32(env, &sj, a, sgrid) : launch_verify_bf16(env, &sj, a, sgrid);
+    } else {
+        const unsigned int grid = (unsigned int)(n_rows * a.job.chunks);
+        rc = f32 ? launch_verify_f32(env, nullptr, a, grid) : launch_verify_bf16(env, nullptr, a, grid);
     }
-    const unsigned int grid = (unsigned int)(n_rows * a.job.chunks);
-    if (p->dtype == AASD_F32) launch(verify_kernel<AASD_F32>, grid, kThreads, 0, ctx->stream, a);
-    else launch(verify_kernel<AASD_BF16>, grid, kThreads, 0, ctx->stream, a);
+    if (rc != AASD_OK) return rc;
     return after_launch(ctx, 1);
 }
 
@@ -667,6 +544,14 @@ int aasd_step(aasd_ctx* ctx, const aasd_step_args* s, void* workspace, size_t wo
 
 }  // extern "C"
 
+extern "C" int aasd_debug_withhold_tile(aasd_ctx* ctx, int64_t item, int32_t tile, uint32_t wait_limit) {
+    if (ctx == nullptr || item < 0 || tile < 0 || wait_limit < 1024u) return AASD_ERR_INVALID_ARG;
+    ctx->withhold_item = item;
+    ctx->withhold_tile = tile;
+    ctx->test_wait_limit = wait_limit;
+    return AASD_OK;
+}
+
 extern "C" int aasd_probe_read(aasd_ctx* ctx, const void* buffer, size_t bytes, uint32_t* sink) {
     if (ctx == nullptr || buffer == nullptr || sink == nullptr) return AASD_ERR_INVALID_ARG;
     if (((uintptr_t)buffer % 16) != 0 || (bytes % 16) != 0) return AASD_ERR_INVALID_ARG;
@@ -678,21 +563,6 @@ extern "C" int aasd_probe_read(aasd_ctx* ctx, const void* buffer, size_t bytes, 
 }
 
 // ---- draft trees ----------------------------------------------------------------------------
-
-namespace {
-
-template <int DT, int ND>
-int launch_tree_stream(aasd_ctx* ctx, const StreamJob& sj, const TreeArgs& a, unsigned int grid) {
-    return launch_stream<DT, 1, ND, false, false, TreeEpilogue<DT>>(ctx, sj, a, grid, false);
-}
-
-template <int DT>
-int dispatch_tree_stream(aasd_ctx* ctx, const StreamJob& sj, const TreeArgs& a, unsigned int grid) {
-    return a.mode == AASD_VERIFY_STRICT_SAMPLED ? launch_tree_stream<DT, 1>(ctx, sj, a, grid)
-                                                : launch_tree_stream<DT, 0>(ctx, sj, a, grid);
-}
-
-}  // namespace
 
 extern "C" int aasd_tree_build(aasd_ctx* ctx, const int32_t* draft_ids, const uint8_t* draft_flags,
                                const int32_t* cand_len, const int32_t* n_cands, int32_t n_seqs, int32_t max_cands,
@@ -759,18 +629,19 @@ extern "C" int aasd_verify_tree(aasd_ctx* ctx, const void* target_logits, const 
     // rows without children keep the hint NONE (all bits set)
     AASD_CUDA(cudaMemsetAsync(a.hint, 0xFF, 4 * (size_t)n_rows, ctx->stream));
     launch(tree_hint_kernel, (unsigned int)((n_rows + 255) / 256), 256u, 0, ctx->stream, a);
-    if (a.job.vector_ok && a.job.nvec > 0) {
+    const bool f32 = p->dtype == AASD_F32;
+    const LaunchEnv env = env_of(ctx);
+    int rc = AASD_OK;
+    if (stream_path(a.job, p->mode == AASD_VERIFY_STRICT_SAMPLED)) {
         StreamJob sj{};
         unsigned int grid = 0;
         plan_stream(ctx, sj, a.job, a.hint, ws, *L, p->mode == AASD_VERIFY_STRICT_SAMPLED ? &a.smp : nullptr, &grid);
-        const int rc = p->dtype == AASD_F32 ? dispatch_tree_stream<AASD_F32>(ctx, sj, a, grid)
-                                            : dispatch_tree_stream<AASD_BF16>(ctx, sj, a, grid);
-        if (rc != AASD_OK) return rc;
-        return after_launch(ctx, 2);
+        rc = f32 ? launch_tree_f32(env, &sj, a, grid) : launch_tree_bf16(env, &sj, a, grid);
+    } else {
+        const unsigned int grid = (unsigned int)(n_rows * a.job.chunks);
+        rc = f32 ? launch_tree_f32(env, nullptr, a, grid) : launch_tree_bf16(env, nullptr, a, grid);
     }
-    const unsigned int grid = (unsigned int)(n_rows * a.job.chunks);
-    if (p->dtype == AASD_F32) launch(tree_kernel<AASD_F32>, grid, (unsigned int)kThreads, 0, ctx->stream, a);
-    else launch(tree_kernel<AASD_BF16>, grid, (unsigned int)kThreads, 0, ctx->stream, a);
+    if (rc != AASD_OK) return rc;
     return after_launch(ctx, 2);
 }
 
@@ -783,15 +654,8 @@ namespace {
 
 constexpr int64_t kStaticMaxRows = AASD_STATIC_MAX_ROWS;
 constexpr int64_t kStaticMaxCands = AASD_STATIC_MAX_CANDS;
-constexpr size_t kStaticWorkspaceBytes =
-    ((sizeof(RowPartial) * (size_t)kPartialSlots + 255) / 256 * 256) +   // pieces of split rows
-    ((4 * (size_t)kStaticMaxRows + 255) / 256 * 256) +                   // row tickets
-    2 * ((4 * (size_t)kStaticMaxCands + 255) / 256 * 256) +              // candidate and sequence tickets
-    256 +                                                                // work-item counters
-    (((size_t)kStaticMaxRows + 255) / 256 * 256) +                       // accept bits
-    ((8 * (size_t)kStaticMaxRows + 255) / 256 * 256) +                   // row states (own token, accept bit)
-    ((4 * (size_t)kStaticMaxRows + 255) / 256 * 256) +                   // next ids
-    ((sizeof(RaceSummary) * (size_t)kRaceSlots * kMaxK + 255) / 256 * 256);   // sampler records of cut rows
+// the same function that lays a caller's workspace out sizes the block, at compile time
+constexpr size_t kStaticWorkspaceBytes = make_layout(kStaticMaxRows, kStaticMaxCands, false).bytes;
 constexpr size_t kStaticBytes = kStaticWorkspaceBytes + 256;
 
 }  // namespace
@@ -805,6 +669,7 @@ struct StaticSlot {
     bool ready;
     int sm_count;
     char* scratch;   // device address of g_static_scratch on this device
+    Tuning tuning;
 };
 StaticSlot g_static_slots[kStaticMaxDevices];
 std::mutex g_static_mutex;
@@ -827,8 +692,8 @@ extern "C" int aasd_verify_static(int device, void* stream, const void* target_l
         if (p->rows_per_cand < 1 || (int64_t)n_cands * p->rows_per_cand != n_rows) return AASD_ERR_BAD_SHAPE;
     }
     if (n_rows > 0 && (draft_ids == nullptr || n_cands == 0)) return AASD_ERR_INVALID_ARG;
-    const WorkspaceLayout L = make_layout(kStaticMaxRows, kStaticMaxCands, false);
-    if (L.bytes != kStaticWorkspaceBytes) return AASD_ERR_WORKSPACE_TOO_SMALL;   // layouts out of step
+    constexpr WorkspaceLayout L = make_layout(kStaticMaxRows, kStaticMaxCands, false);
+    static_assert(L.bytes == kStaticWorkspaceBytes && L.bytes % 256 == 0, "the block holds exactly this layout");
 
     std::lock_guard<std::mutex> guard(g_static_mutex);
     AASD_CUDA(cudaSetDevice(device));
@@ -844,6 +709,7 @@ extern "C" int aasd_verify_static(int device, void* stream, const void* target_l
         if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || ptr == nullptr) return AASD_ERR_CUDA;
         slot.scratch = static_cast<char*>(ptr);
         slot.sm_count = sms;
+        slot.tuning = read_tuning();
         slot.ready = true;
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -859,6 +725,7 @@ extern "C" int aasd_verify_static(int device, void* stream, const void* target_l
     local.stream = s;
     local.sm_count = slot.sm_count;
     local.state = state;
+    local.tuning = slot.tuning;
     VerifyArgs a{};
     int err = plan_rows(&local, a.job, target_logits, p->dtype, p->vocab, p->row_stride, n_rows, p->inv_temperature,
                         ws, L);
@@ -880,17 +747,18 @@ extern "C" int aasd_verify_static(int device, void* stream, const void* target_l
     a.out = *out;
     if (n_rows == 0) {
         if (n_cands > 0) launch(verify_empty_kernel, (unsigned int)((n_cands + 255) / 256), 256, 0, s, a);
-    } else if (a.job.vector_ok && a.job.nvec > 0) {
+    } else if (stream_path(a.job, p->mode == AASD_VERIFY_STRICT_SAMPLED)) {
         StreamJob sj{};
         unsigned int sgrid = 0;
         plan_stream(&local, sj, a.job, draft_ids, ws, L, p->mode == AASD_VERIFY_STRICT_SAMPLED ? &a.smp : nullptr, &sgrid);
-        const int rc = p->dtype == AASD_F32 ? dispatch_verify_stream<AASD_F32>(&local, sj, a, sgrid)
-                                            : dispatch_verify_stream<AASD_BF16>(&local, sj, a, sgrid);
+        const int rc = p->dtype == AASD_F32 ? launch_verify_f32(env_of(&local), &sj, a, sgrid)
+                                            : launch_verify_bf16(env_of(&local), &sj, a, sgrid);
         if (rc != AASD_OK) return rc;
     } else {
         const unsigned int grid = (unsigned int)(n_rows * a.job.chunks);
-        if (p->dtype == AASD_F32) launch(verify_kernel<AASD_F32>, grid, kThreads, 0, s, a);
-        else launch(verify_kernel<AASD_BF16>, grid, kThreads, 0, s, a);
+        const int rc = p->dtype == AASD_F32 ? launch_verify_f32(env_of(&local), nullptr, a, grid)
+                                            : launch_verify_bf16(env_of(&local), nullptr, a, grid);
+        if (rc != AASD_OK) return rc;
     }
     if (cudaGetLastError() != cudaSuccess) return AASD_ERR_CUDA;
     if (status_bits != nullptr)

@@ -14,6 +14,8 @@ struct RowJob {
     int vocab;
     int vector_ok;          // rows are 16-byte aligned: take the vector path
     int nvec;               // whole vectors per row (vector path)
+    int stream_nvec;        // whole vectors every row has from its first 16-byte boundary on, whatever
+                            // its alignment (the streaming kernel's planning figure; 0: rows too short)
     int vec_elts;           // logits per 16-byte vector
     int chunks;             // CTAs per row
     int vec_per_chunk;      // vectors per chunk (multiple of 8)
@@ -645,6 +647,7 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(const VerifyArgs a) {
     if (threadIdx.x == 0) tally.flush(job.state);
 }
 
+#ifdef AASD_HOST_TU   // not a template: compiled in the host translation unit only
 // Candidates of a call without rows.
 __global__ void verify_empty_kernel(const VerifyArgs a) {
     pdl_launch_dependents();
@@ -652,6 +655,7 @@ __global__ void verify_empty_kernel(const VerifyArgs a) {
     int c = blockIdx.x * blockDim.x + threadIdx.x;
     if (c < a.n_cands) write_empty_candidate(a, c);
 }
+#endif
 
 // ---- alignment sampling ---------------------------------------------------------------------------
 
@@ -668,6 +672,7 @@ struct AlignArgs {
     aasd_align_out out;
 };
 
+#ifdef AASD_HOST_TU   // not a template: compiled in the host translation unit only
 // next_ids[t] = prompt_ids[t+1] unless t is the last row of its sequence.
 __global__ void align_next_kernel(const AlignArgs a) {
     pdl_launch_dependents();
@@ -685,6 +690,7 @@ __global__ void align_next_kernel(const AlignArgs a) {
     }
     a.next_ids[t] = nxt;
 }
+#endif
 
 // Does the row take keyed draws?  GUMBEL mode, a usable row, and a next token that is not the
 // greedy one (Sec. 2.3: only misaligned positions get extra tokens).

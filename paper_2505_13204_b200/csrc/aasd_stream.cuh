@@ -36,7 +36,7 @@ constexpr int stream_threads(int nf) { return kConsumers + 32 + 32 * nf; }
 constexpr int kShortRowFinishers = 3;
 constexpr int kRing = 16;
 constexpr int kSlots = 4;                         // item results in flight between consumers and finisher
-constexpr unsigned int kWaitLimit = 1u << 24;     // polls of try_wait before giving up
+constexpr unsigned int kWaitLimit = 1u << 24;     // polls of try_wait before giving up (StreamJob::wait_limit)
 
 // ---- mbarrier / bulk copy primitives ---------------------------------------------------
 __device__ __forceinline__ unsigned int smem_u32(const void* p) {
@@ -64,8 +64,8 @@ __device__ __forceinline__ bool mbar_try_wait(u64* bar, unsigned int parity) {
     return ok != 0;
 }
 // Bounded wait.  Returns false when the limit ran out or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(u64* bar, unsigned int parity, volatile int* abort_flag) {
-    for (unsigned int it = 0; it < kWaitLimit; ++it) {
+__device__ __forceinline__ bool mbar_wait(u64* bar, unsigned int parity, volatile int* abort_flag, unsigned int limit) {
+    for (unsigned int it = 0; it < limit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 255u) == 255u && *abort_flag) return false;
     }
@@ -106,8 +106,9 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(u64* bar, unsigned int par
         : "memory");
     return ok != 0;
 }
-__device__ __forceinline__ bool mbar_wait_cluster(u64* bar, unsigned int parity, volatile int* abort_flag) {
-    for (unsigned int it = 0; it < kWaitLimit; ++it) {
+__device__ __forceinline__ bool mbar_wait_cluster(u64* bar, unsigned int parity, volatile int* abort_flag,
+                                                  unsigned int limit) {
+    for (unsigned int it = 0; it < limit; ++it) {
         if (mbar_try_wait_cluster(bar, parity)) return true;
         if ((it & 255u) == 255u && *abort_flag) return false;
     }
@@ -139,6 +140,8 @@ struct ItemInfo {
     float hint_logit; // its raw logit when it lies inside
     int row;          // logits row of the item; kNoItem: the work list is exhausted
     int chunk;        // which piece of the row
+    int head;         // tokens of the row in front of its first 16-byte boundary (0 for aligned rows)
+    int nvec;         // whole 16-byte vectors of the row from that boundary on
 };
 constexpr int kNoItem = -1;
 constexpr int kMaxCluster = 8;   // portable cluster size
@@ -174,6 +177,10 @@ struct StreamJob {
     long long n_items;        // whole_rows + (n_rows - whole_rows) * tail_chunks
     int cluster_pieces;       // the launch is made of clusters of tail_chunks CTAs, one per row, every
                               // row is cut (whole_rows == 0) and the grid has one CTA per piece
+    unsigned int wait_limit;  // polls after which a wait inside the kernel gives up (kWaitLimit)
+    // testing aid (aasd_debug_withhold_tile): the copy of this tile of this item is never issued
+    long long withhold_item;  // -1: none
+    int withhold_tile;
     // sampling kernels only
     SampleJob smp;
     RaceSummary* race_partials;   // [slots x kMaxK] beside the partial records of cut rows
@@ -195,14 +202,26 @@ __device__ __forceinline__ void decode_item(const StreamJob& job, long long item
 __device__ __forceinline__ int chunks_of(const StreamJob& job, int row) {
     return row < job.whole_rows ? 1 : job.tail_chunks;
 }
-__device__ __forceinline__ void tile_range(const StreamJob& job, int row, int chunk, int& tb, int& te) {
+__device__ __forceinline__ int tiles_of(int nvec) { return (int)(((long long)nvec * 16 + kTileBytes - 1) / kTileBytes); }
+// nvec: the row's own vector count (rows that do not start on a 16-byte boundary differ by one)
+__device__ __forceinline__ void tile_range(const StreamJob& job, int row, int chunk, int nvec, int& tb, int& te) {
+    const int tiles = tiles_of(nvec);
     if (row < job.whole_rows) {
         tb = 0;
-        te = job.tiles_per_row;
+        te = tiles;
     } else {
-        tb = (int)(((long long)chunk * job.tiles_per_row) / job.tail_chunks);
-        te = (int)(((long long)(chunk + 1) * job.tiles_per_row) / job.tail_chunks);
+        tb = (int)(((long long)chunk * tiles) / job.tail_chunks);
+        te = (int)(((long long)(chunk + 1) * tiles) / job.tail_chunks);
     }
+}
+// Where a row's vectors begin: rows are streamed from their first 16-byte boundary, the few
+// tokens in front of it (none when the row is aligned) and behind the last whole vector are
+// left to the finisher.
+template <int DT>
+__device__ __forceinline__ void row_vectors(const char* rowp, int vocab, int& head, int& nvec) {
+    head = (int)(((16u - (unsigned int)((uintptr_t)rowp & 15u)) & 15u) / (unsigned int)Elt<DT>::kSize);
+    head = head < vocab ? head : vocab;
+    nvec = (vocab - head) / Elt<DT>::kVec;
 }
 
 __device__ __forceinline__ u64 make_vec_key(float vmax, int vec) {
@@ -391,10 +410,10 @@ template <> struct AheadCounter<AASD_BF16> {
     unsigned int acc;              // bf16x2 running counts of the current tile (exact: <= 16 each)
     int vd;                        // vector index of d
     int count;
-    __device__ __forceinline__ void begin_item(int d, float xd, bool valid) {
+    __device__ __forceinline__ void begin_item(int d, float xd, bool valid, int head) {
         count = 0;
         acc = 0;
-        vd = d / 8;
+        vd = d < head ? -1 : (d - head) / 8;   // every vector lies behind a token of the row's head
         unsigned int b = __float_as_uint(xd) >> 16;
         unsigned int below = (b & 0x7FFFu) == 0 ? 0x8001u : ((b & 0x8000u) ? b + 1 : b - 1);
         if (!valid || !(xd > -CUDART_INF_F)) b = below = 0x7F80u;   // +inf: nothing is ahead
@@ -424,10 +443,10 @@ template <> struct AheadCounter<AASD_F32> {
     float acc;
     int vd;
     int count;
-    __device__ __forceinline__ void begin_item(int d, float xd, bool valid) {
+    __device__ __forceinline__ void begin_item(int d, float xd, bool valid, int head) {
         count = 0;
         acc = 0.f;
-        vd = d / 4;
+        vd = d < head ? -1 : (d - head) / 4;
         const unsigned int b = __float_as_uint(xd);
         const unsigned int below = (b & 0x7FFFFFFFu) == 0 ? 0x80000001u : ((b & 0x80000000u) ? b + 1 : b - 1);
         thr_gt = xd;
@@ -452,14 +471,15 @@ template <> struct AheadCounter<AASD_F32> {
     }
 };
 
-// The sums of one vector in a sampling kernel: the sum of the vector's weights goes to `gs`
-// (the caller adds a whole group's sum to S at once, and needs it for the group's ratio).
-template <int DT, int K>
+// The sums of one vector in a sampling kernel: the vector's weights are added to `gs`, the
+// running sum of the sampling group the vector belongs to (the caller adds a whole group's sum
+// to S at once, and needs it for the group's ratio).
+template <int DT, int K, bool FIN>
 __device__ __forceinline__ void add_to_group(TileAccumulator<DT, K>& acc, const uint4& raw, float c1, float neg_refc,
                                              float2& gs) {
     constexpr int kVec = Elt<DT>::kVec;
     float x[kVec];
-    Elt<DT>::unpack(Clamp<DT>::apply(raw), x);
+    Elt<DT>::unpack(FIN ? raw : Clamp<DT>::apply(raw), x);
     const float2 cc = make_float2(c1, c1);
     const float2 rr = make_float2(neg_refc, neg_refc);
 #pragma unroll
@@ -565,10 +585,10 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
             unsigned int row_ctr = 0;
             float neg_refc = 0.f;
             bool alive = true, last = false;
-            int tb = 0, te = 1;
+            int tb = 0, te = 1, nvec = 0;
             for (int t = 0; t < te - tb; ++t, ++it) {
                 const int s = it % kStages;
-                if (!mbar_wait(&sh.full[s], (it / kStages) & 1u, abort_flag)) {
+                if (!mbar_wait(&sh.full[s], (it / kStages) & 1u, abort_flag, job.wait_limit)) {
                     if (lane == 0) give_up(abort_flag, rj.state);
                     alive = false;
                     break;
@@ -583,45 +603,48 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
                     }
                     neg_refc = info.neg_refc;
                     row_ctr = (unsigned int)info.row;
-                    if (TK) ahead.begin_item(info.hint, info.hint_logit, info.hint >= 0 && info.hint < rj.vocab);
-                    tile_range(job, info.row, info.chunk, tb, te);
+                    if (TK) ahead.begin_item(info.hint, info.hint_logit, info.hint >= 0 && info.hint < rj.vocab, info.head);
+                    nvec = info.nvec;
+                    tile_range(job, info.row, info.chunk, nvec, tb, te);
                 }
                 const unsigned char* base = tiles + (size_t)s * kTileBytes;
                 const int v0 = (tb + t) * kTileVecs;
-                const int nv = min(kTileVecs, rj.nvec - v0);
+                const int nv = min(kTileVecs, nvec - v0);
                 if (kLazyMax) tilemax.init();
                 if (ND > 0) {
                     // A thread takes the eight neighbouring vectors 8 * tid .. 8 * tid + 7 of the
-                    // tile: two sampling groups of bf16 ids, one group of fp32 ids.  The order in
-                    // which it reads them is rotated by the lane so that a quarter-warp covers
-                    // all shared-memory banks.
+                    // tile: two sampling groups of bf16 ids (vectors 0-3 and 4-7), one group of
+                    // fp32 ids.  So that a quarter-warp covers all shared-memory banks with every
+                    // load, a lane reads the two halves in an order given by bit 2 of its index
+                    // and rotates inside a half by its two low bits; which half a register holds
+                    // is then known at compile time up to one swap at the end.
                     constexpr int kPer = kTileVecs / kConsumers;
                     constexpr int kVecsPerGroup = kGroup / kVec;           // 4 (bf16) or 8 (fp32)
                     constexpr int kGroupsPerThread = kPer / kVecsPerGroup; // 2 or 1
                     static_assert(kPer == 8 && kGroupsPerThread >= 1, "eight vectors per thread and tile");
-                    const int rot = lane & (kPer - 1);
+                    const int hsel = (lane >> 2) & 1, rot = lane & 3;
                     uint4 q[kPer];
                     bool ok[kPer];
 #pragma unroll
                     for (int k = 0; k < kPer; ++k) {
-                        const int v = kPer * tid + ((k + rot) & (kPer - 1));
+                        const int v = kPer * tid + (((((k >> 2) ^ hsel) & 1) << 2) | ((k + rot) & 3));
                         ok[k] = v < nv;
                         if (ok[k]) q[k] = lds16(base + (size_t)v * 16);
                     }
-                    float2 gs[kGroupsPerThread];
-#pragma unroll
-                    for (int gi = 0; gi < kGroupsPerThread; ++gi) gs[gi] = make_float2(0.f, 0.f);
+                    float2 first = make_float2(0.f, 0.f), second = make_float2(0.f, 0.f);   // k < 4, k >= 4
 #pragma unroll
                     for (int k = 0; k < kPer; ++k)
                         if (ok[k]) {
-                            float2 one = make_float2(0.f, 0.f);
-                            add_to_group<DT, K>(acc, q[k], c1, neg_refc, one);
+                            add_to_group<DT, K, FIN>(acc, q[k], c1, neg_refc, k < 4 ? first : second);
                             tilemax.update(q[k]);
-                            const int gi = ((k + rot) & (kPer - 1)) / kVecsPerGroup;   // the group this vector belongs to
-#pragma unroll
-                            for (int j = 0; j < kGroupsPerThread; ++j)
-                                if (gi == j) gs[j] = __fadd2_rn(gs[j], one);
                         }
+                    float2 gs[kGroupsPerThread];
+                    if (kGroupsPerThread == 2) {
+                        gs[0] = hsel ? second : first;    // vectors 0-3 of the thread's share
+                        gs[kGroupsPerThread - 1] = hsel ? first : second;
+                    } else {
+                        gs[0] = __fadd2_rn(first, second);
+                    }
                     const int g0 = (v0 + kPer * tid) * kVec / kGroup;
 #pragma unroll
                     for (int gi = 0; gi < kGroupsPerThread; ++gi) {
@@ -701,7 +724,7 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
                 }
             }
             const int p = seq % kSlots;
-            if (!mbar_wait(&sh.freeb[p], ((seq / kSlots) & 1u) ^ 1u, abort_flag)) {
+            if (!mbar_wait(&sh.freeb[p], ((seq / kSlots) & 1u) ^ 1u, abort_flag, job.wait_limit)) {
                 if (lane == 0) give_up(abort_flag, rj.state);
                 break;
             }
@@ -712,7 +735,7 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
                 for (int j = 0; j < NF && ok; ++j) {
                     const unsigned int sq = seq + (unsigned int)j;
                     const int pj = sq % kSlots;
-                    if (j > 0) ok = mbar_wait(&sh.freeb[pj], ((sq / kSlots) & 1u) ^ 1u, abort_flag);
+                    if (j > 0) ok = mbar_wait(&sh.freeb[pj], ((sq / kSlots) & 1u) ^ 1u, abort_flag, job.wait_limit);
                     if (ok && lane == 0) mbar_arrive(&sh.done[pj]);
                 }
                 if (!ok && lane == 0) give_up(abort_flag, rj.state);
@@ -768,7 +791,7 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
                 // end of the work list: an empty stage use tells the consumers
                 if (lane == 0) {
                     const int s = it % kStages;
-                    if (mbar_wait(&sh.empty[s], ((it / kStages) & 1u) ^ 1u, abort_flag)) {
+                    if (mbar_wait(&sh.empty[s], ((it / kStages) & 1u) ^ 1u, abort_flag, job.wait_limit)) {
                         for (int j = 0; j < NF; ++j) sh.ring[(seq + j) % kRing].row = kNoItem;
                         mbar_arrive(&sh.full[s]);
                         // the last CTA to get here leaves the counters ready for the next launch
@@ -806,19 +829,25 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
                 info.hint_logit = hint_logit;
                 info.row = row;
                 info.chunk = chunk;
+                int head, nvec;
+                row_vectors<DT>(rowp, rj.vocab, head, nvec);
+                info.head = head;
+                info.nvec = nvec;
+                const char* vbase = rowp + (size_t)head * Elt<DT>::kSize;
                 int tb, te;
-                tile_range(job, row, chunk, tb, te);
+                tile_range(job, row, chunk, nvec, tb, te);
                 for (int t = tb; t < te; ++t, ++it) {
                     const int s = it % kStages;
-                    if (!mbar_wait(&sh.empty[s], ((it / kStages) & 1u) ^ 1u, abort_flag)) {
+                    if (!mbar_wait(&sh.empty[s], ((it / kStages) & 1u) ^ 1u, abort_flag, job.wait_limit)) {
                         alive = false;
                         break;
                     }
+                    if (item == job.withhold_item && t - tb == job.withhold_tile) continue;   // testing aid
                     const long long off = (long long)t * kTileBytes;
-                    const long long left = (long long)rj.nvec * 16 - off;
+                    const long long left = (long long)nvec * 16 - off;
                     const unsigned int bytes = (unsigned int)(left < kTileBytes ? left : kTileBytes);
                     mbar_arrive_expect_tx(&sh.full[s], bytes);
-                    bulk_copy_g2s(tiles + (size_t)s * kTileBytes, rowp + off, bytes, &sh.full[s]);
+                    bulk_copy_g2s(tiles + (size_t)s * kTileBytes, vbase + off, bytes, &sh.full[s]);
                     armed |= 1u << s;
                 }
             }
@@ -832,7 +861,7 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
                 const unsigned int j = it - back;
                 const int s = j % kStages;
                 if (armed & (1u << s)) {
-                    for (unsigned int w = 0; w < kWaitLimit; ++w)
+                    for (unsigned int w = 0; w < job.wait_limit; ++w)
                         if (mbar_try_wait(&sh.full[s], (j / kStages) & 1u)) break;
                 }
             }
@@ -847,7 +876,7 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
     tally.clear();
     for (unsigned int seq = (unsigned int)(warp - kConsumerWarps - 1);; seq += NF) {
         const int p = seq % kSlots;
-        if (!mbar_wait(&sh.done[p], (seq / kSlots) & 1u, abort_flag)) {
+        if (!mbar_wait(&sh.done[p], (seq / kSlots) & 1u, abort_flag, job.wait_limit)) {
             if (lane == 0) give_up(abort_flag, rj.state);
             break;
         }
@@ -857,6 +886,8 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
         const int chunk = info.chunk;
         const int chunks = chunks_of(job, info.row);
         const char* rowp = row_pointer<DT>(rj, row);
+        const int head = info.head, nvec = info.nvec;            // the row's vectors: tokens head + 0 ...
+        const char* vbase = rowp + (size_t)head * Elt<DT>::kSize;
         double S = 0.0, A = 0.0;
         u64 vk[K];
 #pragma unroll
@@ -908,7 +939,7 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
                 const unsigned int mine = (lane < kConsumerWarps && top == best) ? (unsigned int)vk[0] : 0u;
                 int n_holders = __reduce_add_sync(0xFFFFFFFFu, __popc(mine));
                 int tb, te;
-                tile_range(job, info.row, info.chunk, tb, te);
+                tile_range(job, info.row, info.chunk, nvec, tb, te);
                 int vfirst = 0x7FFFFFFF;
                 if (n_holders <= 16) {
 #pragma unroll
@@ -918,12 +949,12 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
                             const int l = __ffs(lanes) - 1;
                             lanes &= lanes - 1;
                             const int t = tb + (int)__shfl_sync(0xFFFFFFFFu, (unsigned int)my_tiles[w], l);
-                            const int v = first_vector_in_tile<DT, (ND > 0)>(rowp, rj.nvec, t, w * 32 + l, m);
+                            const int v = first_vector_in_tile<DT, (ND > 0)>(vbase, nvec, t, w * 32 + l, m);
                             if (v >= 0 && v < vfirst) vfirst = v;
                         }
                     }
                 } else {
-                    const int v = first_vector_of_range<DT>(rowp, rj.nvec, tb, te, m);
+                    const int v = first_vector_of_range<DT>(vbase, nvec, tb, te, m);
                     if (v >= 0) vfirst = v;
                 }
                 if (vfirst != 0x7FFFFFFF) mk[0] = make_vec_key(m, vfirst);
@@ -965,7 +996,7 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
                 for (int j = 0; j < kMaxK; ++j) mine.key[j] = j < K ? mk[j] : 0ull;
                 mine.ahead = n_ahead;
             }
-            if (!mbar_wait_cluster(&sh.cluster_bar, 0u, abort_flag)) {
+            if (!mbar_wait_cluster(&sh.cluster_bar, 0u, abort_flag, job.wait_limit)) {
                 if (lane == 0) give_up(abort_flag, rj.state);
                 break;
             }
@@ -1063,7 +1094,9 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
                 }
             }
         }
-        // Best tokens: they lie inside the K best vectors; plus the ragged tail of the row.
+        // Best tokens: they lie inside the K best vectors; plus the tokens outside the vectors
+        // (in front of the row's first 16-byte boundary and behind its last whole vector: fewer
+        // than two vectors' worth together).
         u64 ek[K];
 #pragma unroll
         for (int j = 0; j < K; ++j) ek[j] = 0;
@@ -1075,15 +1108,16 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
                 if (lane == j) mine = mk[j];
             if (lane < K && mine != 0) {
                 const int vec = key_id(mine);
-                const uint4 q = __ldg(reinterpret_cast<const uint4*>(rowp) + vec);
+                const uint4 q = __ldg(reinterpret_cast<const uint4*>(vbase) + vec);
                 float x[kVec];
                 Elt<DT>::unpack(q, x);
 #pragma unroll
                 for (int i = 0; i < kVec; ++i)
-                    if (x[i] > -CUDART_INF_F) key_insert<K>(ek, make_key(x[i], vec * kVec + i));
+                    if (x[i] > -CUDART_INF_F) key_insert<K>(ek, make_key(x[i], head + vec * kVec + i));
             }
-            const int tail0 = rj.nvec * kVec;
-            const int i = tail0 + lane - K;
+            static_assert(kMaxK + 2 * (16 / 2 - 1) <= 32, "one lane per token outside the vectors");
+            const int j = lane - K;
+            const int i = j < head ? j : nvec * kVec + j;   // head tokens first, then the tail
             if (lane >= K && i < rj.vocab) {
                 const float x = Elt<DT>::load(rowp, i);
                 float e, t;
@@ -1131,19 +1165,21 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
             long long extra = 0;
             if (d >= 0 && d < rj.vocab && info.hint_logit > -CUDART_INF_F) {
                 const float xd = info.hint_logit;
-                const int vd = d / kVec;
-                if (vd < rj.nvec) {
-                    const int i = vd * kVec + lane;
+                if (d >= head && d < head + nvec * kVec) {
+                    const int i = head + (d - head) / kVec * kVec + lane;
                     if (lane < kVec && i < d && Elt<DT>::load(rowp, i) == xd) extra += 1;
                 }
-                for (int i = rj.nvec * kVec + lane; i < rj.vocab; i += 32) {
+                // the tokens outside the vectors, one per lane
+                const int i = lane < head ? lane : nvec * kVec + lane;
+                if (i < rj.vocab) {
                     const float x = Elt<DT>::load(rowp, i);
                     extra += (x > xd || (x == xd && i < d)) ? 1 : 0;
                 }
             }
             fr.merged.ahead = n_ahead + warp_sum_i64(extra);
         }
-        // ids beyond the last complete group of the vector part were not raced
+        // ids beyond the last complete group of the vector part were not raced (sampling
+        // launches take aligned rows only: head == 0)
         const int tail_group = (ND > 0 && job.full_groups * kGroup < rj.vocab) ? job.full_groups : -1;
         E::template finish<ND>(args, rj, row, rowp, fr, info, races, tail_group, tally);
     }

@@ -30,6 +30,7 @@ struct TreeBuildArgs {
     int32_t* n_nodes;             // [n_seqs]
 };
 
+#ifdef AASD_HOST_TU   // not a template: compiled in the host translation unit only
 // One warp per sequence.  The candidates are walked in order; at each depth the warp looks
 // for the child that carries the same token (lowest node index, found with a ballot over
 // the nodes made so far, which live in shared memory) or appends a new node.
@@ -93,6 +94,7 @@ __global__ void __launch_bounds__(32) tree_build_kernel(const TreeBuildArgs a) {
     }
     if (lane == 0) a.n_nodes[b] = n;
 }
+#endif
 
 // ---- verification ----------------------------------------------------------------------------
 
@@ -122,6 +124,7 @@ struct TreeArgs {
     aasd_tree_out out;
 };
 
+#ifdef AASD_HOST_TU   // not a template: compiled in the host translation unit only
 // hint[row of parent] = token of the parent's first child (rows without children keep NONE,
 // set by the host).  Also checks the shape: a parent precedes its child.
 __global__ void tree_hint_kernel(const TreeArgs a) {
@@ -143,6 +146,7 @@ __global__ void tree_hint_kernel(const TreeArgs a) {
     const int tok = a.node_token[g];
     if (tok >= 0 && tok < a.job.vocab) a.hint[lo + p] = tok;
 }
+#endif
 
 // Results of trees without nodes (between the offsets of their neighbours).
 __device__ inline void write_empty_tree(const TreeArgs& a, int t) {
@@ -152,12 +156,14 @@ __device__ inline void write_empty_tree(const TreeArgs& a, int t) {
     if (a.out.emit_ids)
         for (int i = 0; i < a.emit_stride; ++i) a.out.emit_ids[(int64_t)t * a.emit_stride + i] = AASD_NONE;
 }
+#ifdef AASD_HOST_TU   // not a template: compiled in the host translation unit only
 __global__ void tree_empty_kernel(const TreeArgs a) {
     pdl_launch_dependents();
     pdl_wait();
     const int t = blockIdx.x * blockDim.x + threadIdx.x;
     if (t < a.n_trees) write_empty_tree(a, t);
 }
+#endif
 
 // Row epilogue, entered by a whole warp.  Phase one (lane 0): the row's statistics.  Phase
 // two (the warp that completes the tree): nodes, paths, result.

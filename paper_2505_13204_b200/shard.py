@@ -7,6 +7,11 @@ inputs from its own seed, and the only cross-rank operation is the reduction of 
 """
 from __future__ import annotations
 
+import os
+import socket
+import subprocess
+import sys
+
 import torch
 import torch.distributed as dist
 
@@ -36,3 +41,37 @@ def max_over_ranks(value: float, device=None) -> float:
 def whole_job_rate(units_per_rank_per_step: float, steps: int, world: int, ms_max: float) -> float:
     """Units per second of all ranks together, given the slowest rank's time for ``steps``."""
     return world * units_per_rank_per_step * steps / (ms_max * 1e-3)
+
+
+def launch_plan(gpus: int, env=None) -> str:
+    """What a program asked to use ``gpus`` GPUs has to do, given its environment:
+    "run" (it is the only rank, or one rank of a launcher's group of that size), or "spawn"
+    (it was started plainly and has to start the ranks itself).  A launcher's group of
+    another size than asked for is an error: the two would silently disagree."""
+    env = os.environ if env is None else env
+    if gpus < 1:
+        raise ValueError("--gpus must be at least 1")
+    world = env.get("WORLD_SIZE")
+    if world is None:
+        return "run" if gpus == 1 else "spawn"
+    if int(world) != gpus:
+        raise ValueError("--gpus %d but the launcher started %s ranks" % (gpus, world))
+    return "run"
+
+
+def free_port() -> int:
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def spawn_ranks(script: str, argv, gpus: int, port: int | None = None, extra_env=None) -> int:
+    """Starts ``gpus`` ranks of ``script argv`` on this node, one process per GPU, through
+    torch's launcher (rendezvous on 127.0.0.1) and returns its exit code.  The ranks find
+    RANK / LOCAL_RANK / WORLD_SIZE / MASTER_* in their environment; their output goes to
+    this process's stdout and stderr (NCCL's communicator lines with NCCL_DEBUG=INFO too)."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(int(gpus)),
+           "--master-addr", "127.0.0.1", "--master-port", str(port or free_port()), script] + list(argv)
+    env = dict(os.environ)
+    env.update(extra_env or {})
+    return subprocess.call(cmd, env=env)

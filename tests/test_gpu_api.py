@@ -114,3 +114,41 @@ def test_host_side_errors_of_tree_and_top_k_calls(ctx):
         ctx.tree_build(big, big.to(torch.uint8), torch.zeros((1, 64), dtype=torch.int32, device="cuda"),
                        torch.zeros(1, dtype=torch.int32, device="cuda"))
     assert e.value.code == 7
+
+
+def test_a_wait_that_runs_out_ends_the_launch_and_the_context_recovers():
+    """Every wait inside the streaming kernel is bounded.  The testing aid makes one CTA never
+    copy one tile and shortens the limit: that CTA's consumers run out of polls, the CTA
+    leaves, the launch ends by itself and the status word says so.  Nothing faults, nothing
+    traps; after the workspace is registered again the same call matches the oracle."""
+    import oracle
+    from parity import check_verify, to_oracle
+    ctx = binding.Context()
+    try:
+        rows, V = 640, 16384                     # more rows than CTA slots: whole rows, no clusters
+        rng = np.random.default_rng(3)
+        d = rng.integers(0, V, rows).astype(np.int32)
+        x = synth.logits(rows, V, torch.bfloat16, synth.LogitRecipe(sigma=2.5, p_hint=0.6, spike_lo=4, spike_hi=12),
+                         torch.as_tensor(d, dtype=torch.int64), 9)
+        offs = np.arange(0, rows + 1, 4, dtype=np.int32)
+        xd, dd, od = x.cuda(), torch.as_tensor(d).cuda(), torch.as_tensor(offs).cuda()
+        ref = oracle.verify(to_oracle(x), d, offs, threads=8)
+        check_verify(ctx.verify(xd, dd, od), ref, offs, torch.bfloat16)
+        assert ctx.poll_status() == 0
+        for item, tile in ((5, 0), (400, 0)):    # a CTA's first item, and one claimed later
+            ctx.debug_withhold_tile(item, tile, 1 << 14)
+            ctx.verify(xd, dd, od)
+            torch.cuda.synchronize()             # the launch ended by itself
+            assert ctx.poll_status() & binding.STATUS_TIMEOUT
+            ctx.reinit_workspace()
+            got = ctx.verify(xd, dd, od)
+            check_verify(got, ref, offs, torch.bfloat16)
+            assert ctx.poll_status() == 0
+        # the aid is used up by one launch; an item beyond the launch's items withholds nothing
+        ctx.debug_withhold_tile(10 ** 9, 0, 1 << 22)
+        check_verify(ctx.verify(xd, dd, od), ref, offs, torch.bfloat16)
+        assert ctx.poll_status() == 0
+        with pytest.raises(binding.AasdError):
+            ctx.debug_withhold_tile(0, 0, 10)    # a limit this short would cut healthy waits
+    finally:
+        ctx.close()

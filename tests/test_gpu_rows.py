@@ -286,6 +286,16 @@ def test_finite_hint_gives_the_same_results(ctx, V, dtype, stride, rows):
     vector_path = (stride is not None) or (V * (4 if dtype == torch.float32 else 2)) % 16 == 0
     if vector_path:
         assert c["redo_rows"] >= 2          # the masked rows were noticed and re-evaluated
+    # the sampling kernels take the hint too: the same draws with and without it
+    refs = oracle.verify(to_oracle(x), d, offs, mode=oracle.VERIFY_STRICT_SAMPLED, seed=77, step=2)
+    gots = ctx.verify(_to_dev(x), torch.as_tensor(d).cuda(), torch.as_tensor(offs).cuda(),
+                      mode=binding.VERIFY_STRICT_SAMPLED, seed=77, step=2, finite_hint=True)
+    check_verify(gots, refs, offs, dtype)
+    refg = oracle.align_sample(to_oracle(x), prompt, [0, rows], k_extra=2, mode=oracle.ALIGN_GUMBEL, seed=78)
+    gotg = ctx.align_sample(_to_dev(x), torch.as_tensor(prompt).cuda(), [0, rows], k_extra=2,
+                            mode=binding.ALIGN_GUMBEL, seed=78, finite_hint=True)
+    check_align(gotg, refg, dtype)
+    assert ctx.poll_status() == 0
 
 
 def test_temperature_and_thresholds(ctx):
@@ -358,7 +368,7 @@ def test_host_side_errors(ctx):
 @pytest.mark.parametrize("V,dtype,rows", [(32000, torch.float32, 8), (128256, torch.bfloat16, 12),
                                           (152064, torch.bfloat16, 3), (70000, torch.bfloat16, 50),
                                           (20000, torch.float32, 147)])
-def test_cluster_and_global_combine_agree(ctx, V, dtype, rows, monkeypatch):
+def test_cluster_and_global_combine_agree(V, dtype, rows, monkeypatch):
     """Scarce rows are cut into pieces; the pieces meet in a cluster's shared memory, or, with
     the switch set, in global memory.  Both give the oracle's results and each other's bytes,
     in verification (with the top-k count) and in alignment sampling."""
@@ -375,6 +385,7 @@ def test_cluster_and_global_combine_agree(ctx, V, dtype, rows, monkeypatch):
             monkeypatch.setenv("AASD_NO_CLUSTER", "1")
         else:
             monkeypatch.delenv("AASD_NO_CLUSTER", raising=False)
+        ctx = binding.Context()          # the switch is read when a context is made
         v = ctx.verify(xd, dd, od, alpha=alpha, beta=beta)
         t = ctx.verify(xd, dd, od, mode=binding.VERIFY_TOP_K, top_k=3)
         a = ctx.align_sample(xd, dd, seq, k_extra=2)
@@ -385,9 +396,10 @@ def test_cluster_and_global_combine_agree(ctx, V, dtype, rows, monkeypatch):
         rt = oracle.verify(to_oracle(x), d, offs, mode=binding.VERIFY_TOP_K, top_k=3)
         assert np.array_equal(cpu(t["n_greater"]), rt["n_greater"])
         check_align(a, oracle.align_sample(to_oracle(x), d, seq, k_extra=2), dtype)
+        assert ctx.poll_status() == 0
+        ctx.close()
     for k in results[0]:
         assert torch.equal(results[0][k], results[1][k]), k
-    assert ctx.poll_status() == 0
 
 
 @pytest.mark.parametrize("V,dtype", [(1000, torch.float32), (32000, torch.float32), (4096, torch.bfloat16)])

@@ -147,7 +147,7 @@ def test_closed_loop_step_matches_oracle(ctx):
     """Algorithm 1's loop on a reduced configuration: both sides start from the same state,
     logits are drawn for the candidates of each step, and every step's outputs and the
     final histories must agree."""
-    w = synth.scaled(synth.workload(2), batch=3, vocab=4096, prompt_len=300, steps=6)
+    w = synth.scaled(synth.workload(2), batch=3, vocab=4096, prompt_len=300, steps=10)
     alpha, beta = F32(0.1), F32(0.1)
     prompts = [synth.prompt_ids(w, b) for b in range(w.batch)]
     hints = torch.cat([synth.next_token_hints(p) for p in prompts])
@@ -158,7 +158,7 @@ def test_closed_loop_step_matches_oracle(ctx):
     align_gpu = ctx.align_sample(pre.cuda(), ids_all.cuda(), seq_offs, k_extra=2)
     assert np.array_equal(cpu(align_gpu["align_ids"]), align_ref["align_ids"])
 
-    cap = 64
+    cap = 128
     st = binding.DecodeState(ctx, prompts, cap, w.ngram, w.draft_len, w.max_cands, w.vocab,
                              w.torch_dtype, align=align_gpu, alpha=alpha, beta=beta)
     hoffs = cpu(st.hist_offsets)
@@ -174,9 +174,10 @@ def test_closed_loop_step_matches_oracle(ctx):
         dr = _oracle_step(hist, hoffs, hlen, plen, align_ref, arow, w, None, alpha, beta)
         dg = st.run_draft()
         check_draft(dg, dr)
-        x = synth.logits(R, w.vocab, w.torch_dtype, w.recipe,
-                         torch.as_tensor(dr["draft_ids"].reshape(-1), dtype=torch.int64),
-                         w.seed * 7919 + s)
+        # a stand-in target that copies from its context, so that every step drafts real tokens
+        x = synth.closed_loop_logits(w, prompts, torch.as_tensor(dr["draft_ids"]), w.seed * 7919 + s)
+        if s > 0:
+            assert (dr["match_len"] > 0).all() and (dr["draft_ids"][:, 0, :] >= 0).mean() > 0.8
         ref = oracle.verify(to_oracle(x), dr["draft_ids"].reshape(-1), coffs,
                             draft_flags=dr["draft_flags"].reshape(-1), alpha=alpha, beta=beta)
         sel = oracle.select(ref["accept_len"], ref["next_token"], dr["draft_ids"].reshape(-1), coffs,
@@ -192,5 +193,5 @@ def test_closed_loop_step_matches_oracle(ctx):
         assert np.array_equal(cpu(st.hist_len), hlen)
         assert np.array_equal(cpu(st.hist_ids), hist)
         emitted += int(sel["n_emit"].sum())
-    assert emitted >= w.steps * w.batch          # every step emits at least the target's token
+    assert 1.5 * w.steps * w.batch <= emitted    # accepted draft tokens on top of the target's own token
     assert ctx.poll_status() == 0

@@ -62,3 +62,45 @@ def test_single_process_needs_no_group():
     assert shard.max_over_ranks(3.5) == 3.5
     assert list(shard.rank_sequences(4, 1, 0)) == [0, 1, 2, 3]
     assert shard.rank_seed(4, 0) == 4
+
+
+def test_launch_plan():
+    assert shard.launch_plan(1, {}) == "run"
+    assert shard.launch_plan(4, {}) == "spawn"
+    assert shard.launch_plan(4, {"WORLD_SIZE": "4"}) == "run"
+    assert shard.launch_plan(1, {"WORLD_SIZE": "1"}) == "run"
+    for bad in ((2, {"WORLD_SIZE": "4"}), (1, {"WORLD_SIZE": "2"}), (0, {})):
+        try:
+            shard.launch_plan(*bad)
+        except ValueError:
+            continue
+        raise AssertionError(bad)
+
+
+_RANK_SCRIPT = """
+import os, sys, json
+sys.path.insert(0, %r)
+import torch.distributed as dist
+from paper_2505_13204_b200 import shard
+assert shard.launch_plan(int(sys.argv[1])) == "run"
+dist.init_process_group("gloo")
+rank, world = dist.get_rank(), dist.get_world_size()
+ms = shard.max_over_ranks(7.0 + rank)
+if rank == 0:
+    print(json.dumps({"n_gpus": world, "ms": ms, "seed": shard.rank_seed(4, rank)}))
+dist.destroy_process_group()
+"""
+
+
+def test_spawned_ranks_form_a_group_of_the_size_asked_for(tmp_path, capfd):
+    """The launcher path of `bench.py --gpus N` (started plainly, N > 1): the program starts N
+    ranks of itself; every rank sees the group, rank 0 prints the line."""
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    script = tmp_path / "rank_script.py"
+    script.write_text(_RANK_SCRIPT % root)
+    rc = shard.spawn_ranks(str(script), ["2"], 2, extra_env={"OMP_NUM_THREADS": "1"})
+    out = capfd.readouterr().out
+    assert rc == 0
+    import json
+    line = [json.loads(l) for l in out.splitlines() if l.startswith("{")][-1]
+    assert line == {"n_gpus": 2, "ms": 8.0, "seed": 4}

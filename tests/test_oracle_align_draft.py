@@ -104,10 +104,30 @@ def test_gumbel_mode_rules():
 
 # ----------------------------------------------------------------------------- drafting
 
-def _naive_draft(h, plen, rec, n, draft_len, max_cands, extras=None, match_align=False):
-    """Independent restatement: a double loop over positions and key lengths."""
+def _dictionary_lookup(h, rec, n):
+    """The draft pool of Algorithm 1 as a dictionary: every k-gram (k <= n) of the sequence
+    maps to the places right after its occurrences; keys are tried longest first.  Returns
+    (k*, places with a continuation, most recent first)."""
+    pool = {}
+    for k in range(1, n + 1):
+        for i in range(0, len(h) - k + 1):
+            pool.setdefault(tuple(h[i:i + k]), []).append(i + k)
+    for k in range(min(n, len(rec)), 0, -1):
+        places = [p for p in pool.get(tuple(rec[len(rec) - k:]), []) if p < len(h)]
+        if places:
+            return k, sorted(places, reverse=True)
+    return 0, []
+
+
+def _naive_draft(h, plen, rec, n, draft_len, max_cands, extras=None, match_align=False, pool=None,
+                 pool_extras=None):
+    """Independent restatement: a double loop over positions and key lengths; the places of
+    an external pool (a list with -1 between documents) come after those of the sequence."""
     extras = extras or {}
+    pool_extras = pool_extras or {}
     L = len(h)
+    if pool is not None:
+        return _naive_draft_with_pool(h, plen, rec, n, draft_len, max_cands, extras, pool, pool_extras)
 
     def tok_ok(q, want, last):
         if h[q] == want:
@@ -138,6 +158,40 @@ def _naive_draft(h, plen, rec, n, draft_len, max_cands, extras=None, match_align
                     if len(cands) < max_cands:
                         cands.append((p, toks[:i] + [(e, 3)]))
     return best_k, cands
+
+
+def _naive_draft_with_pool(h, plen, rec, n, draft_len, max_cands, extras, pool, pool_extras):
+    def mlen(seq, p):
+        m = 0
+        for k in range(1, min(n, p, len(rec)) + 1):
+            if seq[p - k] == -1 or seq[p - k] != rec[len(rec) - k]:
+                break
+            m = k
+        return m
+
+    places = [(0, p, mlen(h, p)) for p in range(len(h) - 1, 0, -1)]
+    places += [(1, p, mlen(pool, p)) for p in range(len(pool) - 1, 0, -1) if pool[p] != -1]
+    best = max([m for _, _, m in places], default=0)
+    mains = [(src, p) for src, p, m in places if m == best and best > 0][:max_cands]
+    cands = []
+    for src, p in mains:
+        if src == 0:
+            toks = [(h[q], 1 if q < plen else 0) for q in range(p, min(p + draft_len, len(h)))]
+        else:
+            toks = []
+            for q in range(p, min(p + draft_len, len(pool))):
+                if pool[q] == -1:
+                    break
+                toks.append((pool[q], 0))
+        cands.append((p if src == 0 else -2 - p, toks))
+    for (src, p), (pos, toks) in zip(mains, list(cands)):
+        for i in range(len(toks)):
+            q = p + i
+            es = (extras.get(q, []) if 1 <= q < plen else []) if src == 0 else pool_extras.get(q, [])
+            for e in es:
+                if len(cands) < max_cands:
+                    cands.append((pos, toks[:i] + [(e, 3)]))
+    return best, cands
 
 
 def _check_draft(h, plen, rec, n, draft_len, max_cands, extras=None, match_align=False, K=2):
@@ -216,3 +270,97 @@ def test_draft_flags_and_alternatives():
     assert list(out["draft_ids"][0, 3]) == [40, -1, -1]
     assert list(out["draft_ids"][0, 4]) == [41, -1, -1]
     assert list(out["draft_ids"][0, 5]) == [7, 50, -1] and list(out["draft_flags"][0, 5][:2]) == [1, 3]
+
+
+def test_draft_lookup_is_algorithm_1s_dictionary():
+    """The places the oracle finds are those of Algorithm 1's pool of k-grams, tried with the
+    longest key first (Sec. 3.1)."""
+    rng = np.random.default_rng(23)
+    for trial in range(80):
+        L = int(rng.integers(3, 120))
+        h = rng.integers(0, 3 + trial % 4, L)
+        n = int(rng.integers(1, 8))
+        rl = int(rng.integers(1, n + 1))
+        rec = h[L - rl:] if trial % 3 else rng.integers(0, 4, rl)
+        k, places = _dictionary_lookup(list(h), list(rec), n)
+        recent = np.full(n, -1, np.int32)
+        recent[:rl] = rec
+        out = oracle.draft(h, [0, L], [L], [L], recent, [rl], n, 3, 64)
+        assert out["match_len"][0] == k
+        assert out["cand_pos"][0, :out["n_cands"][0]].tolist() == places[:64]
+
+
+def _check_pool(h, plen, rec, n, draft_len, max_cands, pool, extras=None, pool_extras=None, K=2):
+    L, P = len(h), len(pool)
+    table = dict(align_ids=None, align_n=None, align_row_offsets=None, pool_align_ids=None, pool_align_n=None)
+    if extras is not None:
+        table["align_ids"] = np.full((plen, K), -1, np.int32)
+        table["align_n"] = np.zeros(plen, np.int32)
+        for q, es in extras.items():
+            table["align_ids"][q - 1, :len(es)] = es
+            table["align_n"][q - 1] = len(es)
+        table["align_row_offsets"] = [0, plen]
+    if pool_extras is not None:
+        table["pool_align_ids"] = np.full((P, K), -1, np.int32)
+        table["pool_align_n"] = np.zeros(P, np.int32)
+        for q, es in pool_extras.items():
+            table["pool_align_ids"][q - 1, :len(es)] = es
+            table["pool_align_n"][q - 1] = len(es)
+    recent = np.full(n, -1, np.int32)
+    recent[:len(rec)] = rec
+    out = oracle.draft(h, [0, L + 2], [L], [plen], recent, [len(rec)], n, draft_len, max_cands, k_extra=K,
+                       pool_ids=np.asarray(pool, np.int32), **table)
+    k, cands = _naive_draft(list(h), plen, list(rec), n, draft_len, max_cands, extras, pool=list(pool),
+                            pool_extras=pool_extras)
+    assert out["match_len"][0] == k and out["n_cands"][0] == len(cands)
+    for c, (p, toks) in enumerate(cands):
+        assert out["cand_pos"][0, c] == p and out["cand_len"][0, c] == len(toks)
+        assert list(out["draft_ids"][0, c, :len(toks)]) == [t for t, _ in toks]
+        assert list(out["draft_flags"][0, c, :len(toks)]) == [f for _, f in toks]
+        assert np.all(out["draft_ids"][0, c, len(toks):] == -1)
+    return out
+
+
+def test_draft_external_pool_hand_case():
+    # the sequence ends in "7 8"; the pool holds "7 8 9 4 | 3 7 8 5" (| = a document boundary)
+    h = [1, 2, 7, 8]
+    pool = [7, 8, 9, 4, -1, 3, 7, 8, 5]
+    out = _check_pool(h, 4, [7, 8], 2, 3, 4, pool)
+    assert out["match_len"][0] == 2
+    assert out["cand_pos"][0].tolist() == [-2 - 8, -2 - 2, -1, -1]       # pool places, the later one first
+    assert out["draft_ids"][0, 0].tolist() == [5, -1, -1]                # the pool ends there
+    assert out["draft_ids"][0, 1].tolist() == [9, 4, -1]                 # stops at the document boundary
+    assert out["draft_flags"][0, 1].tolist() == [0, 0, 0]                # pool tokens are verified strictly
+    # a longer match inside the sequence itself beats the pool; an equal one comes first
+    h = [7, 8, 6, 1, 7, 8]
+    out = _check_pool(h, 6, [7, 8], 2, 2, 4, pool)
+    assert out["cand_pos"][0].tolist() == [2, -10, -4, -1] and out["draft_flags"][0, 0].tolist() == [1, 1]
+    out = _check_pool(h, 6, [1, 7, 8], 3, 2, 4, pool)
+    assert out["match_len"][0] == 2            # "1 7 8" has no continuation anywhere: fall back to "7 8"
+    # a key that crosses the boundary does not match: "4 3" never occurs inside one document
+    out = _check_pool([0, 4, 3], 3, [4, 3], 2, 2, 4, pool)
+    assert out["match_len"][0] == 1 and out["cand_pos"][0, 0] == -2 - 6 and out["draft_ids"][0, 0].tolist() == [7, 8]
+    # extras of pool positions make alternatives, flagged as alignment-sampled tokens
+    out = _check_pool([1, 2, 7, 8], 4, [7, 8], 2, 3, 4, pool, pool_extras={2: [40], 3: [50, 51]})
+    assert out["draft_ids"][0, 2].tolist() == [40, -1, -1] and out["draft_flags"][0, 2, 0] == 3
+    assert out["draft_ids"][0, 3].tolist() == [9, 50, -1] and out["draft_flags"][0, 3].tolist() == [0, 3, 0]
+
+
+def test_draft_external_pool_random_against_naive():
+    rng = np.random.default_rng(31)
+    for trial in range(80):
+        L = int(rng.integers(2, 40))
+        plen = int(rng.integers(1, L + 1))
+        h = rng.integers(0, 4, L)
+        P = int(rng.integers(1, 60))
+        pool = rng.integers(0, 4, P)
+        pool[rng.random(P) < 0.12] = -1
+        n = int(rng.integers(1, 6))
+        rl = int(rng.integers(1, n + 1))
+        rec = h[L - rl:] if trial % 2 else rng.integers(0, 4, rl)
+        extras = pool_extras = None
+        if trial % 3 == 0:
+            extras = {q: list(rng.choice(6, size=int(rng.integers(0, 3)), replace=False) + 10) for q in range(1, plen)}
+            pool_extras = {q: list(rng.choice(6, size=int(rng.integers(0, 3)), replace=False) + 20)
+                           for q in range(1, P) if pool[q] != -1}
+        _check_pool(h, plen, rec, n, int(rng.integers(1, 7)), int(rng.integers(1, 8)), pool, extras, pool_extras)

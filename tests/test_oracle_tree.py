@@ -83,17 +83,18 @@ def test_tree_verification_equals_the_longest_passing_flat_candidate():
             kids = [c for c in range(1, n) if par[c] == v]
             if kids and rng.random() < 0.7:
                 x[v, tok[kids[int(rng.integers(0, len(kids)))]]] += 8.0
-        for mode in (oracle.VERIFY_CONDITIONAL, oracle.VERIFY_STRICT_GREEDY, oracle.VERIFY_STRICT_SAMPLED):
+        for mode in (oracle.VERIFY_CONDITIONAL, oracle.VERIFY_STRICT_GREEDY, oracle.VERIFY_STRICT_SAMPLED,
+                     oracle.VERIFY_TOP_K):
             got = oracle.verify_tree(x, tok, par, [0, n], 6, node_flags=fl, alpha=0.1, beta=0.05, mode=mode,
-                                     seed=3, step=trial)
+                                     seed=3, step=trial, top_k=3)
             best_len, best_emits = -1, []
             for path in _paths(par, n):
                 rows = [0] + path                               # row that judges token i, then the leaf's row
                 xs = x[rows]
                 ids = np.array([tok[v] for v in path] + [-1], np.int32)
                 fls = np.array([fl[v] for v in path] + [0], np.uint8)
-                ref = oracle.verify(xs, ids, [0, len(ids)], draft_flags=fls, alpha=0.1, beta=0.05,
-                                    mode=oracle.VERIFY_CONDITIONAL if mode == oracle.VERIFY_CONDITIONAL
+                ref = oracle.verify(xs, ids, [0, len(ids)], draft_flags=fls, alpha=0.1, beta=0.05, top_k=3,
+                                    mode=mode if mode in (oracle.VERIFY_CONDITIONAL, oracle.VERIFY_TOP_K)
                                     else oracle.VERIFY_STRICT_GREEDY)
                 if mode == oracle.VERIFY_STRICT_SAMPLED:
                     continue                                    # keyed by the row index: checked below
@@ -119,6 +120,31 @@ def test_tree_verification_equals_the_longest_passing_flat_candidate():
             # several candidates may pass equally far (siblings under conditional verification)
             assert got["emit_ids"][0][:got["n_emit"][0]].tolist() in best_emits
             assert got["n_emit"][0] == min(6, best_len + 1)
+
+
+def test_tree_top_k_counts_against_a_full_sort():
+    """Top-k verification on a tree (Sec. 3.3): a node's token is ranked in its parent's row."""
+    rng = np.random.default_rng(11)
+    V, n = 19, 9
+    x = np.round(rng.standard_normal((n, V)) * 2, 1).astype(np.float32)      # rounded: many ties
+    x[2, 4] = -np.inf
+    par = np.array([-1, 0, 0, 1, 1, 2, 2, 3, 5], np.int32)
+    tok = np.array([-1, 3, 7, 1, 0, 4, 9, 18, 2], np.int32)                  # node 5's token is masked in row 2
+    order = np.argsort(-x, axis=1, kind="stable")
+    rank = [-1] + [int(np.where(order[par[v]] == tok[v])[0][0]) for v in range(1, n)]
+    rank[5] = -1
+    for k in (1, 4, 19):
+        out = oracle.verify_tree(x, tok, par, [0, n], 5, mode=oracle.VERIFY_TOP_K, top_k=k)
+        assert out["n_greater"].tolist() == rank
+        assert out["accept"].tolist() == [int(0 <= r < k) for r in rank]
+    # k = 1 is strict greedy verification along the tree
+    a = oracle.verify_tree(x, tok, par, [0, n], 5, mode=oracle.VERIFY_TOP_K, top_k=1)
+    b = oracle.verify_tree(x, tok, par, [0, n], 5, mode=oracle.VERIFY_STRICT_GREEDY)
+    for key in ("accept", "best_node", "n_accept", "emit_ids"):
+        assert np.array_equal(a[key], b[key]), key
+    # nodes that are not eligible are verified strictly
+    c = oracle.verify_tree(x, tok, par, [0, n], 5, node_flags=np.zeros(n, np.uint8), mode=oracle.VERIFY_TOP_K, top_k=19)
+    assert np.array_equal(c["accept"], b["accept"])
 
 
 def test_tree_edge_cases():

@@ -13,7 +13,9 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2505_13204_b200 import binding, synth
+from parity import check_verify, cpu, to_oracle
 
 pytestmark = pytest.mark.gpu
 
@@ -65,6 +67,65 @@ def test_static_entry_point_matches_aasd_verify_twice_in_a_row(rows, V, dtype, r
             assert int(status.item()) == ctx.poll_status() == 0
     finally:
         ctx.close()
+
+
+MODES = [(binding.VERIFY_STRICT_SAMPLED, 6, 32000, torch.float32), (binding.VERIFY_STRICT_SAMPLED, 500, 4096, torch.bfloat16),
+         (binding.VERIFY_TOP_K, 9, 152064, torch.bfloat16), (binding.VERIFY_TOP_K, 300, 1003, torch.float32),
+         (binding.VERIFY_CONDITIONAL, 12, 128256, torch.bfloat16)]
+
+
+@pytest.mark.parametrize("mode,rows,V,dtype", MODES)
+def test_static_entry_point_matches_the_oracle_in_every_mode(mode, rows, V, dtype):
+    """Against the CPU oracle directly, twice in a row, in the modes that use the parts of the
+    block the conditional mode never touches: the sampler records of rows cut into pieces
+    (STRICT_SAMPLED with few rows) and the count of tokens ahead of the draft token (TOP_K)."""
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for call in range(2):
+        x, d, fl, offs = _case(rows, V, dtype, 50 * call + rows, regular=False)
+        kw = dict(alpha=float(np.float32(0.1)), beta=float(np.float32(0.05)), mode=mode, seed=1234 + call,
+                  step=3 + call, top_k=4)
+        ref = oracle.verify(to_oracle(x), cpu(d), cpu(offs), draft_flags=cpu(fl), **kw)
+        got = binding.verify_static(x, d, offs, draft_flags=fl, status_bits=status, **kw)
+        torch.cuda.synchronize()
+        if mode != binding.VERIFY_STRICT_SAMPLED:
+            got = {k: v for k, v in got.items() if k != "sampled"}
+        check_verify(got, ref, cpu(offs), dtype)
+        if mode == binding.VERIFY_TOP_K:
+            assert np.array_equal(cpu(got["n_greater"]), ref["n_greater"])
+        assert int(status.item()) == 0
+
+
+def test_static_entry_point_at_its_row_and_candidate_limits():
+    R = binding.STATIC_MAX_ROWS
+    V = 256
+    rng = np.random.default_rng(8192)
+    x = torch.as_tensor(rng.standard_normal((R, V)).astype(np.float32) * 3).cuda()
+    d = torch.as_tensor(rng.integers(0, V, R).astype(np.int32)).cuda()
+    offs = torch.arange(0, R + 1, dtype=torch.int32, device="cuda")      # 8192 candidates of one row
+    ref = oracle.verify(to_oracle(x), cpu(d), cpu(offs), threads=8)
+    for _ in range(2):
+        got = binding.verify_static(x, d, offs)
+        torch.cuda.synchronize()
+        got = {k: v for k, v in got.items() if k != "sampled"}
+        check_verify(got, ref, cpu(offs), torch.float32)
+
+
+def test_static_entry_point_allocates_no_device_memory():
+    """With every output handed in ready-made, a call leaves the device's free memory as it
+    found it (the driver's own figure, which also sees allocations that bypass torch)."""
+    rows, V = 64, 32000
+    x, d, fl, offs = _case(rows, V, torch.bfloat16, 5, regular=True)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    kw = dict(draft_flags=fl, rows_per_cand=4, status_bits=status)
+    outs = binding.verify_static(x, d, None, **kw)          # the first call on a device sets the block up
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    held0 = torch.cuda.memory_allocated()
+    for mode in (binding.VERIFY_CONDITIONAL, binding.VERIFY_STRICT_SAMPLED, binding.VERIFY_TOP_K):
+        binding.verify_static(x, d, None, outputs=outs, mode=mode, **kw)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0 and torch.cuda.memory_allocated() == held0
 
 
 def test_static_entry_point_reports_status_and_rejects_oversize():
