@@ -34,7 +34,6 @@ import os
 import subprocess
 import sys
 import tempfile
-import threading
 import time
 
 import numpy as np
@@ -79,12 +78,31 @@ def measured_peaks():
     return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
 
 
+_SAMPLER_CODE = r"""
+import sys, time, os
+import pynvml
+index, period = int(sys.argv[1]), float(sys.argv[2])
+pynvml.nvmlInit()
+h = pynvml.nvmlDeviceGetHandleByIndex(index)
+print("max", pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM), flush=True)
+while True:
+    try:
+        print(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM),
+              pynvml.nvmlDeviceGetCurrentClocksEventReasons(h),
+              pynvml.nvmlDeviceGetPowerUsage(h), flush=True)
+    except Exception:
+        pass
+    time.sleep(period)
+"""
+
+
 class ClockSampler:
     """SM clock and throttle reasons of one GPU, read while a timed region runs.
 
-    Reads only (NVML's clock and clocks-event-reasons queries from a thread, every
-    millisecond or so: the short timed region lasts a few milliseconds); falls back to an
-    nvidia-smi loop when the NVML binding is missing.  Changes no setting of the GPU."""
+    Reads only: a child process polls NVML's clock, clocks-event-reasons and power queries
+    every millisecond or so (the short timed region lasts a few milliseconds; a thread of this
+    process would starve behind the launch loop) and is stopped after the region; falls back
+    to an nvidia-smi loop when the NVML binding is missing.  Changes no setting of the GPU."""
     REASONS = {"hw_slowdown": 0x8, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20,
                "sw_power_cap": 0x4}
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
@@ -92,51 +110,43 @@ class ClockSampler:
          "clocks_event_reasons.sw_power_cap")
 
     def __init__(self, index: int, period_s: float = 0.001):
-        self.sm, self.power, self.bits = [], [], 0
-        self.max_mhz = None
-        self.p = self.f = self.thread = None
-        self.stop_flag = False
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p, self.how = None, None
+        vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+        phys = index
+        if vis:
+            t = vis.split(",")
+            if index < len(t) and t[index].strip().isdigit():
+                phys = int(t[index])
         try:
-            import pynvml
-            pynvml.nvmlInit()
-            vis = os.environ.get("CUDA_VISIBLE_DEVICES")
-            phys = int(vis.split(",")[index]) if vis and vis.split(",")[index].isdigit() else index
-            h = pynvml.nvmlDeviceGetHandleByIndex(phys)
-            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
-
-            def loop():
-                while not self.stop_flag:
-                    try:
-                        self.sm.append(float(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)))
-                        self.bits |= int(pynvml.nvmlDeviceGetCurrentClocksEventReasons(h))
-                        self.power.append(pynvml.nvmlDeviceGetPowerUsage(h) / 1000.0)
-                    except Exception:
-                        pass
-                    time.sleep(period_s)
-            self.thread = threading.Thread(target=loop, daemon=True)
-            self.thread.start()
+            import pynvml  # noqa: F401
+            self.p = subprocess.Popen([sys.executable, "-c", _SAMPLER_CODE, str(phys), str(period_s)],
+                                      stdout=self.f, stderr=subprocess.DEVNULL)
+            self.how = "nvml"
+            deadline = time.time() + 10.0            # wait until the child has taken its first samples
+            while time.time() < deadline and self.p.poll() is None:
+                with open(self.f.name) as probe:
+                    if probe.read().count("\n") >= 3:
+                        break
+                time.sleep(0.01)
         except Exception:
-            self.thread = None
-            self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            self.p = None
+        if self.p is None or self.p.poll() is not None:
             try:
                 self.p = subprocess.Popen(
-                    ["nvidia-smi", "-i", str(index), "--query-gpu=" + self.Q,
+                    ["nvidia-smi", "-i", str(phys), "--query-gpu=" + self.Q,
                      "--format=csv,noheader,nounits", "-lms", "20"], stdout=self.f,
                     stderr=subprocess.DEVNULL)
+                self.how = "nvidia-smi"
             except OSError:
-                pass
+                self.p = None
 
-    def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "how": None}
-        if self.thread is not None:
-            self.stop_flag = True
-            self.thread.join(timeout=2)
-            if self.sm:
-                out.update(sm_mhz=float(np.median(self.sm)), sm_min_mhz=float(min(self.sm)),
-                           sm_max_mhz=self.max_mhz, samples=len(self.sm),
-                           power_w_max=max(self.power) if self.power else None,
-                           reasons=sorted(n for n, b in self.REASONS.items() if self.bits & b), how="nvml")
-            return out
+    def mark(self):
+        """Byte offset of the samples taken so far (samples before a mark can be left out)."""
+        return os.path.getsize(self.f.name)
+
+    def stop(self, since: int = 0):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "how": self.how}
         if self.p is None:
             return out
         self.p.terminate()
@@ -146,25 +156,43 @@ class ClockSampler:
             self.p.kill()
         self.f.flush()
         self.f.seek(0)
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for line in self.f.read().splitlines():
-            t = [c.strip() for c in line.split(",")]
-            if len(t) < 7:
-                continue
-            try:
-                sm.append(float(t[0]))
-                mx.append(float(t[1]))
-            except ValueError:
-                continue
-            for n, v in zip(names, t[3:7]):
-                if v.lower().startswith("active"):
-                    reasons.add(n)
+        text = self.f.read()
         self.f.close()
         os.unlink(self.f.name)
+        sm, power, bits, mx, reasons = [], [], 0, None, set()
+        if self.how == "nvml":
+            head = text[:since].splitlines()
+            for line in text.splitlines()[:1]:
+                if line.startswith("max"):
+                    mx = float(line.split()[1])
+            lines = text[since:].splitlines() if since else text.splitlines()[1:]
+            for line in lines:
+                t = line.split()
+                if len(t) != 3 or not t[0].isdigit():
+                    continue
+                sm.append(float(t[0]))
+                bits |= int(t[1])
+                power.append(int(t[2]) / 1000.0)
+            reasons = {n for n, b in self.REASONS.items() if bits & b}
+            del head
+        else:
+            names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+            for line in text[since:].splitlines():
+                t = [c.strip() for c in line.split(",")]
+                if len(t) < 7:
+                    continue
+                try:
+                    sm.append(float(t[0]))
+                    mx = max(mx or 0.0, float(t[1]))
+                    power.append(float(t[2]))
+                except ValueError:
+                    continue
+                for n, v in zip(names, t[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
         if sm:
-            out.update(sm_mhz=float(np.median(sm)), sm_min_mhz=float(min(sm)), sm_max_mhz=float(max(mx)),
-                       samples=len(sm), reasons=sorted(reasons), how="nvidia-smi")
+            out.update(sm_mhz=float(np.median(sm)), sm_min_mhz=float(min(sm)), sm_max_mhz=mx, samples=len(sm),
+                       power_w_max=max(power) if power else None, reasons=sorted(reasons))
         return out
 
 
@@ -406,6 +434,7 @@ def run_ours(args, rank, world, local_rank):
     # the warm-up steps run straight into the timed ones: step s of the timed region is step
     # W + s of one uninterrupted sequence, and the clock sampler covers all of it
     clocks = ClockSampler(local_rank)
+    clock_mark = clocks.mark()                     # samples from here on: warm-up and timed steps
     for s in range(W):
         bench.step(s)
     barrier()
@@ -415,7 +444,7 @@ def run_ours(args, rank, world, local_rank):
         bench.step(W + s, evs[s])
     t_end.record()
     barrier()
-    clk = clocks.stop()
+    clk = clocks.stop(since=clock_mark)
     ms = t_begin.elapsed_time(t_end)
     launches = bench.ctx.launch_count() - launches0
     align_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in evs]))
@@ -436,12 +465,13 @@ def run_ours(args, rank, world, local_rank):
         s_begin, s_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         barrier()
         sclocks = ClockSampler(local_rank, period_s=0.005)
+        smark = sclocks.mark()
         s_begin.record()
         for s in range(n_sus):
             bench.step(W + K + s, sev[s // every] if s % every == 0 else None)
         s_end.record()
         barrier()
-        sclk = sclocks.stop()
+        sclk = sclocks.stop(since=smark)
         s_ms = shard.max_over_ranks(s_begin.elapsed_time(s_end), dev)
         used = [e for i, e in enumerate(sev) if i * every < n_sus]
         s_align = float(np.mean([e[0].elapsed_time(e[1]) for e in used]))
@@ -599,9 +629,32 @@ def decode_step_latency(index: int, dev, n_buf: int = 4, reps: int = 50):
 
         us = timed(True)
         us_verify = timed(False)
+
+        # the floor: the same graph with the library's smallest kernel (selection over one
+        # sequence, one thread at work) in the place of the verification launch
+        def floor():
+            graph = torch.cuda.CUDAGraph()
+            vo = st.verify_out
+            with torch.cuda.graph(graph, stream=side):
+                st.hist_ids.copy_(hist0)
+                st.hist_len.copy_(len0)
+                for j in range(n_buf):
+                    ctx.select(vo["accept_len"], vo["next_token"], st.draft_out["draft_ids"], w.draft_len + 1,
+                               rows_per_cand=w.draft_len, cands_per_seq=w.max_cands, n_seqs=1)
+            for _ in range(3):
+                graph.replay()
+            t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            t0.record()
+            for _ in range(reps):
+                graph.replay()
+            t1.record()
+            side.synchronize()
+            return t0.elapsed_time(t1) * 1e3 / (reps * n_buf)
+
+        us_floor = floor()
     torch.cuda.synchronize()
     ctx.close()
-    return {"us_per_step": us, "verify_launch_us": us_verify, "verify_rows": st.rows,
+    return {"us_per_step": us, "verify_launch_us": us_verify, "launch_floor_us": us_floor, "verify_rows": st.rows,
             "real_draft_rows": real / n_buf, "sequences": w.batch,
             "note": "draft + verify/select/append, graph replay; includes 1/%d of a state restore" % n_buf}
 

@@ -21,10 +21,12 @@
  *    vocabulary, NaN or +inf logit, history overflow) set bits in a device status word
  *    that aasd_poll_status returns and clears; the kernels never trap.
  *  - Logits are row-major [rows x vocab] with a row stride given in elements; dtype is
- *    AASD_F32 or AASD_BF16.  When the buffer and the row stride in bytes are multiples of
- *    16, so that every row starts on a 16-byte boundary, the rows are streamed at close to
- *    memory speed; other layouts (a bf16 vocabulary of 50257 with stride = vocab, say) are
- *    handled by a path about half as fast with identical results, so pad the stride.
+ *    AASD_F32 or AASD_BF16.  Rows are streamed at close to memory speed whatever their
+ *    alignment (a bf16 vocabulary of 50257 with stride = vocab is as fast as a padded one:
+ *    every row is copied from its first 16-byte boundary on).  Two exceptions take a much
+ *    slower path with identical results: rows shorter than 256 bytes, and calls that draw
+ *    keyed samples (AASD_ALIGN_GUMBEL, AASD_VERIFY_STRICT_SAMPLED) from rows that do not all
+ *    start on 16-byte boundaries - pad the row stride for those.
  *  - Token ids are int32, AASD_NONE (-1) means "no token".  Offsets arrays are CSR.
  *  - Scratch memory comes from the caller: a workspace of aasd_workspace_bytes() bytes
  *    that was registered once with aasd_workspace_init().  A workspace must not be shared
@@ -90,6 +92,9 @@ typedef enum aasd_verify_mode {
 #define AASD_STATUS_TIMEOUT 16u       /* a bounded wait inside a kernel ran out: the results of
                                          that call are invalid and the workspace must be
                                          registered again before its next use */
+#define AASD_STATUS_INTERNAL 32u      /* checked builds only (compiled with AASD_BOUNDS_CHECK): an
+                                         index computed inside a kernel fell outside its array;
+                                         the access was skipped */
 
 /* Bits of a draft token's flag byte (Sec. 3.3, last paragraph). */
 #define AASD_FLAG_CONDITIONAL 1u /* from the input context or alignment sampling */
@@ -198,16 +203,26 @@ typedef struct aasd_draft_in {
     const int32_t* align_row_offsets; /* [n_seqs] table row of each sequence's first position */
     const int32_t* recent_ids;    /* [n_seqs x n] key tokens, the last recent_len[b] ... */
     const int32_t* recent_len;    /* ... of which end the current sequence (0..n) */
+    /* external pool (Limitations: retrieval from a source other than the sequence itself):
+       one token buffer shared by all sequences, NONE between its documents; NULL = none */
+    const int32_t* pool_ids;      /* [pool_len] */
+    const int32_t* pool_align_ids;/* [pool_len x k_extra] alignment table of the pool (extras of pool
+                                     position q in row q - 1), or NULL */
+    const int32_t* pool_align_n;  /* [pool_len] extras per row */
+    int32_t pool_len;
 } aasd_draft_in;
 
 typedef struct aasd_draft_out {
     int32_t* draft_ids;    /* [n_seqs x max_cands x draft_len], NONE padded */
     uint8_t* draft_flags;  /* same shape, AASD_FLAG_* */
     int32_t* cand_len;     /* [n_seqs x max_cands] */
-    int32_t* cand_pos;     /* [n_seqs x max_cands] match position of the candidate's main */
+    int32_t* cand_pos;     /* [n_seqs x max_cands] match position of the candidate's main; a place p of
+                              the external pool is reported as AASD_POOL_PLACE(p) = -2 - p */
     int32_t* n_cands;      /* [n_seqs] */
     int32_t* match_len;    /* [n_seqs] length of the matched key, 0 = no match */
 } aasd_draft_out;
+
+#define AASD_POOL_PLACE(p) (-2 - (p))
 
 /* For every sequence: the longest k <= min(n, recent_len) such that the last k key tokens
  * occur in the history at a place that has a continuation; the places (index right after
@@ -215,7 +230,13 @@ typedef struct aasd_draft_out {
  * draft_len history tokens; then, while slots remain, alternatives in (main, depth i,
  * extra slot) order made of the main's first i tokens plus one alignment extra of position
  * p+i (extras of prompt position q are table row align_row_offsets[b] + q - 1).  All
- * outputs are required. */
+ * outputs are required.
+ * With an external pool the places of the pool compete with the history's for the longest
+ * key and follow them in the list (descending within the pool); a key never matches across
+ * a NONE token of the pool and a candidate ends in front of one.  Pool tokens are not input
+ * context: their flag is 0 (strict verification); extras of the pool's own table are
+ * alignment-sampled tokens like any other (flags 3).  The pool is scanned by every sequence's
+ * CTA, so its cost grows with n_seqs x pool_len: meant for pools of up to some 10^5 tokens. */
 int aasd_draft(aasd_ctx* ctx, const aasd_draft_in* in, const aasd_draft_params* params,
                const aasd_draft_out* out);
 
@@ -331,9 +352,9 @@ int aasd_step(aasd_ctx* ctx, const aasd_step_args* args, void* workspace,
  * launch that appends the token; positions beyond the history's capacity are dropped like
  * their tokens.  The table must therefore have a row for every position of every history
  * buffer (rows laid out like hist_offsets), and a caller who wants drafts to use the new
- * rows passes prompt_len = hist_len to aasd_draft.  CONDITIONAL and STRICT_GREEDY modes,
- * draft.k_extra 1 or 2, rows the streaming kernel takes (16-byte aligned, vocab * element
- * size >= 16); AASD_ERR_UNSUPPORTED otherwise. */
+ * rows passes prompt_len = hist_len to aasd_draft.  Every verification mode (the rule does not
+ * ask how a token came to be accepted), draft.k_extra 1 to AASD_MAX_EXTRA, every logits
+ * layout; the workspace must have been sized by aasd_workspace_bytes. */
 
 /* ---- draft trees (Eq. 2, Sec. 3.2) and their verification (Sec. 3.3) ---------------- */
 
@@ -364,16 +385,20 @@ typedef struct aasd_tree_out {
     int32_t* n_emit;      /* [n_trees] tokens in emit_ids */
     int32_t* emit_ids;    /* [n_trees x emit_stride] the tokens on the path to best_node followed by
                              the target's own token of best_node's row; NONE padded, clipped */
+    int32_t* n_greater;   /* [n_rows] AASD_VERIFY_TOP_K only: tokens of the parent's row that are ahead of
+                             the node's token (logit descending, id ascending); NONE for roots, NONE or
+                             masked tokens, bad rows, and in the other modes */
 } aasd_tree_out;
 
 /* Verifies draft trees.  Trees are CSR ranges of nodes (tree_offsets[n_trees+1], the last
  * offset equals n_rows); row v of target_logits is the distribution that follows node v
  * given the path from the root, so the token of node v is judged with its parent's row by
- * the rules of aasd_verify (modes CONDITIONAL, STRICT_GREEDY, STRICT_SAMPLED; node_flags may
- * be NULL: every node conditional-eligible).  A node passes when it and all its ancestors
+ * the rules of aasd_verify (all four modes; in TOP_K mode an eligible node passes iff fewer than
+ * top_k tokens of its parent's row are ahead of its token; node_flags may be NULL: every node
+ * conditional-eligible).  A node passes when it and all its ancestors
  * are accepted; per tree the deepest passing node wins (ties: lowest index), which is the
  * longest candidate that passes.  Because every node has a row of its own, the token after
- * the accepted path is always available.  params->rows_per_cand and top_k are ignored.
+ * the accepted path is always available.  params->rows_per_cand is ignored.
  * A node whose parent index is not smaller than its own raises AASD_STATUS_BAD_OFFSETS and
  * never passes.  best_node, n_accept, n_emit and emit_ids are required. */
 int aasd_verify_tree(aasd_ctx* ctx, const void* target_logits, const int32_t* node_token,

@@ -18,6 +18,7 @@ F32, BF16 = 0, 1
 ALIGN_TOPK, ALIGN_GUMBEL = 0, 1
 VERIFY_CONDITIONAL, VERIFY_STRICT_GREEDY, VERIFY_STRICT_SAMPLED, VERIFY_TOP_K = 0, 1, 2, 3
 STATUS_BAD_ROW, STATUS_ID_RANGE, STATUS_HIST_OVERFLOW, STATUS_BAD_OFFSETS, STATUS_TIMEOUT = 1, 2, 4, 8, 16
+STATUS_INTERNAL = 32
 FLAG_CONDITIONAL, FLAG_EXTRA = 1, 2
 DRAFT_MATCH_ALIGN = 1
 HINT_FINITE = 1
@@ -56,7 +57,8 @@ class DraftParams(C.Structure):
 class DraftIn(C.Structure):
     _fields_ = [(n, _vp) for n in ("hist_ids", "hist_offsets", "hist_len", "prompt_len",
                                    "align_ids", "align_n", "align_row_offsets", "recent_ids",
-                                   "recent_len")]
+                                   "recent_len", "pool_ids", "pool_align_ids", "pool_align_n")] + [
+                                       ("pool_len", C.c_int32)]
 
 
 class DraftOut(C.Structure):
@@ -78,7 +80,7 @@ class VerifyOut(C.Structure):
 
 class TreeOut(C.Structure):
     _fields_ = [(n, _vp) for n in ("p_token", "accept", "entropy", "pmax", "argmax", "threshold",
-                                   "sampled", "best_node", "n_accept", "n_emit", "emit_ids")]
+                                   "sampled", "best_node", "n_accept", "n_emit", "emit_ids", "n_greater")]
 
 
 class StepArgs(C.Structure):
@@ -223,8 +225,9 @@ def verify_static(target_logits, draft_ids, cand_offsets=None, draft_flags=None,
 class Context:
     """One library context bound to a device and the current torch stream."""
 
-    def __init__(self, device: int | None = None, stream: torch.cuda.Stream | None = None):
-        self.lib = load_library()
+    def __init__(self, device: int | None = None, stream: torch.cuda.Stream | None = None, lib=None):
+        """``lib``: another build of the library (``load_library(path)``), e.g. the checked one."""
+        self.lib = lib or load_library()
         if not torch.cuda.is_available():
             raise RuntimeError("no CUDA device: the AASD path runs only on sm_100 GPUs")
         self.device_index = torch.cuda.current_device() if device is None else int(device)
@@ -338,11 +341,16 @@ class Context:
 
     def draft(self, hist_ids, hist_offsets, hist_len, prompt_len, n, draft_len, max_cands,
               recent_ids=None, recent_len=None, align_ids=None, align_n=None,
-              align_row_offsets=None, match_align=False, outputs=None):
-        """aasd_draft.  ``recent_ids=None`` uses each history's own tail as the key."""
+              align_row_offsets=None, match_align=False, outputs=None, pool_ids=None,
+              pool_align_ids=None, pool_align_n=None):
+        """aasd_draft.  ``recent_ids=None`` uses each history's own tail as the key.
+        ``pool_ids``: an external pool (int32 on the device, NONE between documents), with
+        ``pool_align_ids`` [len x k_extra] / ``pool_align_n`` [len] when it has a table."""
         dev = hist_ids.device
         B = hist_len.numel()
         K = 0 if align_ids is None else int(align_ids.shape[1])
+        if align_ids is None and pool_align_ids is not None:
+            K = int(pool_align_ids.shape[1])
         o = outputs or dict(
             draft_ids=torch.empty((B, max_cands, draft_len), dtype=torch.int32, device=dev),
             draft_flags=torch.empty((B, max_cands, draft_len), dtype=torch.uint8, device=dev),
@@ -351,7 +359,8 @@ class Context:
             n_cands=torch.empty(B, dtype=torch.int32, device=dev),
             match_len=torch.empty(B, dtype=torch.int32, device=dev))
         din = DraftIn(_p(hist_ids), _p(hist_offsets), _p(hist_len), _p(prompt_len), _p(align_ids),
-                      _p(align_n), _p(align_row_offsets), _p(recent_ids), _p(recent_len))
+                      _p(align_n), _p(align_row_offsets), _p(recent_ids), _p(recent_len), _p(pool_ids),
+                      _p(pool_align_ids), _p(pool_align_n), 0 if pool_ids is None else int(pool_ids.numel()))
         prm = DraftParams(B, int(n), int(draft_len), int(max_cands), K,
                           DRAFT_MATCH_ALIGN if match_align else 0)
         out = DraftOut(*[_p(o[n_]) for n_, _ in DraftOut._fields_])
@@ -409,7 +418,7 @@ class Context:
 
     def verify_tree(self, target_logits, node_token, node_parent, tree_offsets, emit_stride,
                     node_flags=None, alpha=0.1, beta=0.1, mode=VERIFY_CONDITIONAL, seed=0, step=0,
-                    inv_temperature=1.0, outputs=None):
+                    inv_temperature=1.0, outputs=None, top_k=5):
         """aasd_verify_tree: trees are CSR ranges of nodes, row v follows node v."""
         x = target_logits
         assert x.is_cuda and x.dim() == 2 and x.stride(1) == 1
@@ -428,9 +437,10 @@ class Context:
             best_node=torch.empty(T, dtype=torch.int32, device=dev),
             n_accept=torch.empty(T, dtype=torch.int32, device=dev),
             n_emit=torch.empty(T, dtype=torch.int32, device=dev),
-            emit_ids=torch.empty((T, emit_stride), dtype=torch.int32, device=dev))
+            emit_ids=torch.empty((T, emit_stride), dtype=torch.int32, device=dev),
+            n_greater=torch.empty(R, dtype=torch.int32, device=dev))
         prm = VerifyParams(V, _dtype_code(x), x.stride(0), float(alpha), float(beta),
-                           float(inv_temperature), int(mode), 0, int(step), int(seed), 0)
+                           float(inv_temperature), int(mode), 0, int(step), int(seed), int(top_k))
         out = TreeOut(*[_p(o.get(n)) for n, _ in TreeOut._fields_])
         ws = self.workspace(R, T)
         fl = None if node_flags is None else node_flags.reshape(-1)
@@ -543,7 +553,7 @@ class DecodeState:
                              _p(self.prompt_len),
                              _p(align["align_ids"]) if align else None,
                              _p(align["n_extra"]) if align else None,
-                             _p(self.align_row_offsets), None, None)
+                             _p(self.align_row_offsets), None, None, None, None, None, 0)
         K = int(align["align_ids"].shape[1]) if align else 0
         a.draft = DraftParams(B, n, draft_len, max_cands, K, DRAFT_MATCH_ALIGN if match_align else 0)
         a.draft_out = DraftOut(*[_p(self.draft_out[k]) for k, _ in DraftOut._fields_])

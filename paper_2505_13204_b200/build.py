@@ -25,8 +25,10 @@ UNITS = [("aasd.cu", "host", [])] + [
 DEPENDS = ["aasd.cu", "aasd_verify.cu", "aasd_align.cu", "aasd_align_gumbel.cu", "aasd_tree.cu", "aasd_host.h",
            "aasd_device.cuh", "aasd_rows.cuh", "aasd_sampler.cuh", "aasd_stream.cuh", "aasd_tokens.cuh",
            "aasd_tree.cuh", os.path.join("..", "..", "include", "aasd.h")]
+# -fno-gnu-unique / -Bsymbolic: two builds of the library (the normal and the checked one) can
+# live in one process without sharing function-local statics or binding to each other's symbols
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "-Xcompiler", "-fPIC"]
+              "-Xcompiler", "-fPIC", "-Xcompiler", "-fno-gnu-unique"]
 
 
 def _nvcc() -> str:
@@ -68,7 +70,8 @@ def build(force: bool = False, verbose: bool = False, check: bool = False) -> st
             raise subprocess.CalledProcessError(rc, cmd)
         objs.append(obj)
     tmp = lib + ".tmp.%d" % os.getpid()
-    subprocess.check_call([_nvcc(), "-shared", "-gencode", "arch=compute_100a,code=sm_100a"] + objs + ["-o", tmp])
+    subprocess.check_call([_nvcc(), "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-Xlinker", "-Bsymbolic"]
+                          + objs + ["-o", tmp])
     os.replace(tmp, lib)
     for obj in objs:
         os.unlink(obj)

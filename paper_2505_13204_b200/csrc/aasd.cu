@@ -374,6 +374,8 @@ int aasd_draft(aasd_ctx* ctx, const aasd_draft_in* in, const aasd_draft_params* 
     if (!in->hist_ids || !in->hist_offsets || !in->hist_len || !in->prompt_len) return AASD_ERR_INVALID_ARG;
     if (in->recent_ids && !in->recent_len) return AASD_ERR_INVALID_ARG;
     if (in->align_ids && p->k_extra > 0 && (!in->align_n || !in->align_row_offsets)) return AASD_ERR_INVALID_ARG;
+    if (in->pool_len < 0 || (in->pool_len > 0 && !in->pool_ids)) return AASD_ERR_INVALID_ARG;
+    if (in->pool_align_ids && p->k_extra > 0 && !in->pool_align_n) return AASD_ERR_INVALID_ARG;
     if (!out->draft_ids || !out->draft_flags || !out->cand_len || !out->cand_pos || !out->n_cands || !out->match_len)
         return AASD_ERR_INVALID_ARG;
     DraftArgs a{*in, *p, *out, ctx->state};
@@ -427,7 +429,7 @@ int verify_impl(aasd_ctx* ctx, const void* target_logits, const int32_t* draft_i
         a.seq.enabled = 1;
         a.seq.seq_tickets = reinterpret_cast<unsigned int*>(ws + L->off_seq_tickets);
         if (seq->table_ids) {
-            if (!L->full || !stream_path(a.job, false)) return AASD_ERR_UNSUPPORTED;
+            if (!L->full) return AASD_ERR_UNSUPPORTED;
             a.row_extra = reinterpret_cast<int32_t*>(ws + L->off_row_extra);
         }
     }
@@ -505,9 +507,7 @@ int aasd_step(aasd_ctx* ctx, const aasd_step_args* s, void* workspace, size_t wo
     if (!s->verify_out.accept_len || !s->verify_out.next_token) return AASD_ERR_INVALID_ARG;
     if (s->flags & AASD_STEP_EXTEND_TABLE) {
         if (!s->table_ids || !s->table_n || !s->draft_in.align_row_offsets) return AASD_ERR_INVALID_ARG;
-        if (dp.k_extra < 1 || dp.k_extra > 2) return AASD_ERR_UNSUPPORTED;
-        if (s->verify.mode != AASD_VERIFY_CONDITIONAL && s->verify.mode != AASD_VERIFY_STRICT_GREEDY)
-            return AASD_ERR_UNSUPPORTED;
+        if (dp.k_extra < 1 || dp.k_extra > AASD_MAX_EXTRA) return AASD_ERR_INVALID_ARG;
     }
     int err = AASD_OK;
     if (!(s->flags & AASD_STEP_REUSE_DRAFT)) {
@@ -592,7 +592,8 @@ extern "C" int aasd_verify_tree(aasd_ctx* ctx, const void* target_logits, const 
     TraceRange trace("aasd_verify_tree");
     if (ctx == nullptr || p == nullptr || out == nullptr) return AASD_ERR_INVALID_ARG;
     if (n_trees < 0 || n_rows < 0 || emit_stride < 1) return AASD_ERR_BAD_SHAPE;
-    if (p->mode < AASD_VERIFY_CONDITIONAL || p->mode > AASD_VERIFY_STRICT_SAMPLED) return AASD_ERR_UNSUPPORTED;
+    if (p->mode < AASD_VERIFY_CONDITIONAL || p->mode > AASD_VERIFY_TOP_K) return AASD_ERR_INVALID_ARG;
+    if (p->mode == AASD_VERIFY_TOP_K && p->top_k < 1) return AASD_ERR_INVALID_ARG;
     if (!(p->alpha >= 0.f) || !(p->beta >= 0.f)) return AASD_ERR_INVALID_ARG;
     if (n_trees > 0 && tree_offsets == nullptr) return AASD_ERR_INVALID_ARG;
     if (n_rows > 0 && (node_token == nullptr || node_parent == nullptr || n_trees == 0)) return AASD_ERR_INVALID_ARG;
@@ -613,6 +614,7 @@ extern "C" int aasd_verify_tree(aasd_ctx* ctx, const void* target_logits, const 
     a.alpha = p->alpha;
     a.beta = p->beta;
     a.mode = p->mode;
+    a.top_k = p->top_k;
     a.emit_stride = emit_stride;
     a.smp = make_sample_job(p->seed, p->step, false, p->inv_temperature);
     a.hint = reinterpret_cast<int32_t*>(ws + L->off_next);

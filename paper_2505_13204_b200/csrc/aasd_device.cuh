@@ -32,6 +32,20 @@ struct DeviceState {
 };
 enum Counter { kCntRows = 0, kCntBad, kCntRedo, kCntNear, kCntAccepted, kCntRecheck, kCntExact };
 
+// Checked build (-DAASD_BOUNDS_CHECK): the kernels range-check the indices they compute
+// before they use them (shared-memory stages and slots, vectors and tokens of a row, rows,
+// candidates, scratch records); a violation raises AASD_STATUS_INTERNAL and the access is
+// skipped.  In the normal build the macro is the constant true and costs nothing.
+#ifdef AASD_BOUNDS_CHECK
+__device__ __forceinline__ bool checked_range(bool ok, DeviceState* state) {
+    if (!ok) atomicOr(&state->status, AASD_STATUS_INTERNAL);
+    return ok;
+}
+#define AASD_IN_RANGE(cond, state) (::aasd::checked_range((cond), (state)))
+#else
+#define AASD_IN_RANGE(cond, state) (true)
+#endif
+
 // Per (row, chunk) result of the streaming pass.
 struct RowPartial {
     double S;          // sum 2^(x*c1 - refc)
@@ -89,6 +103,15 @@ __device__ __forceinline__ float ex2_approx(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
+}
+
+// Takes a ticket: adds 1 to a counter in global memory and returns its old value.  The
+// addition releases what this thread wrote before it and acquires what earlier ticket holders
+// released, in one instruction (instead of a fence, an atomic and another fence).
+__device__ __forceinline__ unsigned int take_ticket(unsigned int* counter) {
+    unsigned int old;
+    asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(counter) : "memory");
+    return old;
 }
 
 // ---- programmatic dependent launch -----------------------------------------------------

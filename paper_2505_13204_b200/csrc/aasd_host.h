@@ -54,7 +54,7 @@ constexpr WorkspaceLayout make_layout(int64_t max_rows, int64_t max_cands, bool 
     L.off_tree_stats = o;
     if (with_tree) o = align_up(o + sizeof(TreeRowStat) * (size_t)max_rows, 256);
     L.off_row_extra = o;
-    if (with_tree) o = align_up(o + 12 * (size_t)max_rows, 256);
+    if (with_tree) o = align_up(o + sizeof(int32_t) * kRowExtraInts * (size_t)max_rows, 256);
     L.full = with_tree;
     L.bytes = o;
     return L;

@@ -352,6 +352,8 @@ struct SeqTail {
     int table_k;                        // row width of table_ids
 };
 
+constexpr int kRowExtraInts = 1 + kMaxK;   // per row: how many tokens rank above its draft token, and which
+
 struct VerifyArgs {
     RowJob job;
     const int32_t* draft_ids;
@@ -363,7 +365,7 @@ struct VerifyArgs {
     int mode;
     unsigned int* cand_tickets;
     u64* row_state;                // scratch [n_rows]: the row's own token << 32 | its accept bit
-    int32_t* row_extra;            // scratch [n_rows x 3] or NULL: (count, two ids) ranked above the row's draft token
+    int32_t* row_extra;            // scratch [n_rows x kRowExtraInts] or NULL: (count, ids) ranked above the row's draft token
     SampleJob smp;                 // STRICT_SAMPLED: the row's own token is a keyed draw
     int top_k;                     // TOP_K mode
     unsigned int hints;            // AASD_HINT_*
@@ -418,6 +420,7 @@ __device__ unsigned int verify_row(const VerifyArgs& a, const RowJob& job, int64
                                    Tally& tally) {
     const bool d_ok = d >= 0 && d < job.vocab;
     const RowFinal f = finish_row(merged, job.c1, neg_refc, centered);
+    if (!AASD_IN_RANGE(row >= 0 && row < job.n_rows && (f.bad || (f.top1 >= 0 && f.top1 < job.vocab)), job.state)) return 0xFFFFFFFFu;
     const unsigned int flag = a.draft_flags ? a.draft_flags[row] : AASD_FLAG_CONDITIONAL;
     const double lin = (double)a.alpha * f.H + (double)a.beta;
     const double thr = f.bad ? 0.0 : fmin(lin, f.pmax);
@@ -441,23 +444,31 @@ __device__ unsigned int verify_row(const VerifyArgs& a, const RowJob& job, int64
     a.row_state[row] = ((u64)(unsigned int)own << 32) | (acc ? 1ull : 0ull);
     if (a.row_extra) {
         // Fig. 2's rule with the draft token in the place of the prompt's next token
-        int n = 0, ids[2] = {AASD_NONE, AASD_NONE};
+        int n = 0, ids[kMaxK];
+#pragma unroll
+        for (int j = 0; j < kMaxK; ++j) ids[j] = AASD_NONE;
         if (d_ok && !f.bad) {
-            const int width = a.seq.table_k < 2 ? a.seq.table_k : 2;
-            for (int j = 0; j < width; ++j) {
+            const int width = a.seq.table_k < kMaxK ? a.seq.table_k : kMaxK;
+#pragma unroll
+            for (int j = 0; j < kMaxK; ++j) {
                 const u64 k = merged.key[j];
-                if (k == 0) break;
+                if (j >= width || k == 0) break;
                 const float xv = key_value(k);
                 const int id = key_id(k);
-                if (xv > xd || (xv == xd && id < d)) ids[n++] = id;
+                if (xv > xd || (xv == xd && id < d)) {
+#pragma unroll
+                    for (int q = 0; q < kMaxK; ++q)
+                        if (q == n) ids[q] = id;
+                    ++n;
+                }
             }
         }
-        a.row_extra[row * 3 + 0] = n;
-        a.row_extra[row * 3 + 1] = ids[0];
-        a.row_extra[row * 3 + 2] = ids[1];
+        int32_t* x = a.row_extra + row * kRowExtraInts;
+        x[0] = n;
+#pragma unroll
+        for (int j = 0; j < kMaxK; ++j) x[1 + j] = ids[j];
     }
-    __threadfence();
-    const unsigned int t = atomicAdd(ticket, 1u);
+    const unsigned int t = take_ticket(ticket);
     if (a.out.n_greater)
         a.out.n_greater[row] = (a.mode == AASD_VERIFY_TOP_K && d_ok && !f.bad && xd > -CUDART_INF_F)
                                    ? (int)merged.ahead : AASD_NONE;
@@ -506,6 +517,7 @@ __device__ void verify_finish_warp(const VerifyArgs& a, const RowJob& job, int64
     int64_t lo = 0, hi = 0;
     if (lane == 0) {
         c = candidate_of_row(a, job.n_rows, row, lo, hi);
+        if (!AASD_IN_RANGE(c >= 0 && c < a.n_cands && lo >= 0 && lo <= row && row < hi && hi <= job.n_rows, job.state)) c = 0, hi = lo = 0;
         const unsigned int t = verify_row<DT>(a, job, row, merged, neg_refc, centered, d, xd, sampled,
                                               &a.cand_tickets[c], tally);
         last = (t == (unsigned int)(hi - lo) - 1u);
@@ -539,15 +551,16 @@ __device__ void verify_finish_warp(const VerifyArgs& a, const RowJob& job, int64
     // The warp that completes a sequence's last candidate selects and appends.
     const int cps = a.seq.cands_per_seq;
     const int b = c / cps;
-    if (lane == 0) {
+    if (cps > 1) {     // a sequence with a single candidate is complete with it: no second ticket
+        if (lane == 0) {
+            const unsigned int t = take_ticket(&a.seq.seq_tickets[b]);
+            last = (t == (unsigned int)cps - 1u);
+            if (last) a.seq.seq_tickets[b] = 0;
+        }
+        last = __shfl_sync(0xFFFFFFFFu, last, 0);
+        if (!last) return;
         __threadfence();
-        const unsigned int t = atomicAdd(&a.seq.seq_tickets[b], 1u);
-        last = (t == (unsigned int)cps - 1u);
-        if (last) a.seq.seq_tickets[b] = 0;
     }
-    last = __shfl_sync(0xFFFFFFFFu, last, 0);
-    if (!last) return;
-    __threadfence();
     // longest accepted prefix, ties to the lowest candidate: key = (length + 1, ~candidate)
     u64 key = 0;
     for (int j = lane; j < cps; j += 32) {
@@ -584,15 +597,19 @@ __device__ void verify_finish_warp(const VerifyArgs& a, const RowJob& job, int64
         const int K = a.seq.table_k;
         for (int i = lane; i < ne; i += 32) {
             if (len + i >= cap || len + i < 1) continue;
-            int n = 0, ids[2] = {AASD_NONE, AASD_NONE};
+            int n = 0, ids[kMaxK];
+#pragma unroll
+            for (int j = 0; j < kMaxK; ++j) ids[j] = AASD_NONE;
             if (i < best_a) {
-                const int32_t* x = a.row_extra + ((int64_t)best * a.rows_per_cand + i) * 3;
+                const int32_t* x = a.row_extra + ((int64_t)best * a.rows_per_cand + i) * kRowExtraInts;
                 n = __ldcg(x);
-                ids[0] = __ldcg(x + 1);
-                ids[1] = __ldcg(x + 2);
+#pragma unroll
+                for (int j = 0; j < kMaxK; ++j) ids[j] = __ldcg(x + 1 + j);
             }
             a.seq.table_n[row0 + i] = n;
-            for (int j = 0; j < K; ++j) a.seq.table_ids[(row0 + i) * K + j] = j < 2 ? ids[j] : AASD_NONE;
+#pragma unroll
+            for (int j = 0; j < kMaxK; ++j)
+                if (j < K) a.seq.table_ids[(row0 + i) * K + j] = ids[j];
         }
     }
     __syncwarp();
@@ -606,7 +623,9 @@ __device__ void verify_finish_warp(const VerifyArgs& a, const RowJob& job, int64
 
 // One CTA (or `chunks` CTAs) per row with plain vector / scalar loads: the path for logits
 // whose rows are not 16-byte aligned.
-template <int DT>
+// K: how many of the row's best tokens are kept (1, or the table's width when the step also
+// enters the emitted tokens into the alignment table).
+template <int DT, int K = 1>
 __global__ void __launch_bounds__(kThreads) verify_kernel(const VerifyArgs a) {
     __shared__ BlockScratch sc;
     pdl_launch_dependents();
@@ -619,7 +638,7 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(const VerifyArgs a) {
     const bool d_ok = d >= 0 && d < job.vocab;
     float neg_refc;
     bool centered;
-    if (!row_reduce<DT, 1>(job, row, chunk, d_ok ? d : -1, rowp, neg_refc, centered, sc)) return;
+    if (!row_reduce<DT, K>(job, row, chunk, d_ok ? d : -1, rowp, neg_refc, centered, sc)) return;
     if (threadIdx.x >= 32) return;
     const float xd = d_ok ? Elt<DT>::load(rowp, d) : 0.f;
     Tally tally;

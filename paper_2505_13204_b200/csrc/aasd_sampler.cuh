@@ -119,13 +119,20 @@ struct GroupRace {
             best_g[j] = -1;
         }
     }
-    // group g with softmax share gsum (relative to the row's reference)
-    __device__ __forceinline__ void offer(float gsum, int g, unsigned int row, const SampleJob& sj) {
+    // 1 / E for the ND draws of group g: depends on the group's index only, not on its logits, so
+    // a caller can have it computed while the logits are still on their way through the pipes
+    static __device__ __forceinline__ void inverse_variates(int g, unsigned int row, const SampleJob& sj, float (&inv_e)[ND]) {
         unsigned int w[4];
         philox4x32_10((unsigned int)g, row, sj.step, sj.dom_group, sj.key0, sj.key1, w);
 #pragma unroll
+        for (int j = 0; j < ND; ++j) inv_e[j] = rcp_approx(exponential_fast(w[j]));
+    }
+    // group g with softmax share gsum (relative to the row's reference); valid = false: the group
+    // does not take part (it is not wholly inside the row's vectors)
+    __device__ __forceinline__ void take(float gsum, const float (&inv_e)[ND], int g, bool valid) {
+#pragma unroll
         for (int j = 0; j < ND; ++j) {
-            const float q = gsum * rcp_approx(exponential_fast(w[j]));
+            const float q = valid ? gsum * inv_e[j] : -1.f;
             // groups are met in ascending order: '>' keeps the lower g among equal ratios
             const bool up = q > best[j];
             runner[j] = fmaxf(runner[j], up ? best[j] : q);

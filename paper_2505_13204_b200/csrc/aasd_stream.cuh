@@ -224,6 +224,8 @@ __device__ __forceinline__ void row_vectors(const char* rowp, int vocab, int& he
     nvec = (vocab - head) / Elt<DT>::kVec;
 }
 
+__device__ __forceinline__ bool info_row_ok(unsigned int row, long long n_rows) { return (long long)row < n_rows; }
+
 __device__ __forceinline__ u64 make_vec_key(float vmax, int vec) {
     return ((u64)ordered_bits(vmax) << 32) | (u64)(0xFFFFFFFFu - (unsigned int)vec);
 }
@@ -302,6 +304,10 @@ struct TileAccumulator {
             S2[i] = __fadd2_rn(S2[i], e);
             A2[i] = __ffma2_rn(e, t, A2[i]);
         }
+        track(raw, vec_index);
+    }
+    // the vector joins the K best ones if its maximum says so
+    __device__ __forceinline__ void track(const uint4& raw, int vec_index) {
         float vmax = Clamp<DT>::vector_max(raw);
         int vi = vec_index;
 #pragma unroll
@@ -367,31 +373,46 @@ __device__ __forceinline__ void add_sums(TileAccumulator<DT, K>& acc, const uint
     }
 }
 
+// Where the finisher re-reads vectors of the item it finishes: the row in global memory, or,
+// when the item's tiles are all still resident (launches of one item per CTA with no more
+// tiles than ring stages), the shared-memory ring itself: tile t of the item sits in stage
+// t - tb.
+struct VectorSource {
+    const char* vbase;              // the row's first vector in global memory
+    const unsigned char* resident;  // the ring, or nullptr
+    int tb;                         // first tile of the item
+    __device__ __forceinline__ uint4 load(int v) const {
+        constexpr int kTileVecs = kTileBytes / 16;
+        if (resident) return lds16(resident + ((size_t)(v / kTileVecs - tb) * kTileVecs + (size_t)(v % kTileVecs)) * 16);
+        return __ldg(reinterpret_cast<const uint4*>(vbase) + v);
+    }
+};
+
 // First vector (lowest index) with maximum m among the vectors thread `tid` of the consumers
 // read in tile t: vectors t * 2048 + k * 256 + tid, or, in sampling kernels (GROUPED), the eight
 // neighbours t * 2048 + 8 * tid + k.  By a whole warp; -1 if none.
 template <int DT, bool GROUPED>
-__device__ int first_vector_in_tile(const char* rowp, int nvec, int t, int tid, float m) {
+__device__ int first_vector_in_tile(const VectorSource& src, int nvec, int t, int tid, float m) {
     constexpr int kTileVecs = kTileBytes / 16;
     constexpr int kPer = kTileVecs / kConsumers;
     const int lane = threadIdx.x & 31;
     const int step = GROUPED ? 1 : kConsumers, first = GROUPED ? kPer * tid : tid;
     const int v = t * kTileVecs + first + lane * step;
     bool hit = false;
-    if (lane < kPer && v < nvec) hit = Clamp<DT>::vector_max(__ldg(reinterpret_cast<const uint4*>(rowp) + v)) == m;
+    if (lane < kPer && v < nvec) hit = Clamp<DT>::vector_max(src.load(v)) == m;
     const unsigned int bal = __ballot_sync(0xFFFFFFFFu, hit);
     return bal ? t * kTileVecs + first + (__ffs(bal) - 1) * step : -1;
 }
 // The same over every vector of tiles [tb, te) (many lanes tie for the maximum).
 template <int DT>
-__device__ int first_vector_of_range(const char* rowp, int nvec, int tb, int te, float m) {
+__device__ int first_vector_of_range(const VectorSource& src, int nvec, int tb, int te, float m) {
     constexpr int kTileVecs = kTileBytes / 16;
     const int lane = threadIdx.x & 31;
     const int end = min(te * kTileVecs, nvec);
     for (int base = tb * kTileVecs; base < end; base += 32) {
         const int v = base + lane;
         bool hit = false;
-        if (v < end) hit = Clamp<DT>::vector_max(__ldg(reinterpret_cast<const uint4*>(rowp) + v)) == m;
+        if (v < end) hit = Clamp<DT>::vector_max(src.load(v)) == m;
         const unsigned int bal = __ballot_sync(0xFFFFFFFFu, hit);
         if (bal) return base + __ffs(bal) - 1;
     }
@@ -471,12 +492,13 @@ template <> struct AheadCounter<AASD_F32> {
     }
 };
 
-// The sums of one vector in a sampling kernel: the vector's weights are added to `gs`, the
-// running sum of the sampling group the vector belongs to (the caller adds a whole group's sum
-// to S at once, and needs it for the group's ratio).
+// The sums of one vector in a sampling kernel: the vector's weights are added to the running
+// sum of the sampling group the vector belongs to, kept in two halves (`ga` takes the even
+// pairs, `gb` the odd ones) so that consecutive additions do not wait for one another.  The
+// caller adds a whole group's sum to S at once, and needs it for the group's ratio.
 template <int DT, int K, bool FIN>
 __device__ __forceinline__ void add_to_group(TileAccumulator<DT, K>& acc, const uint4& raw, float c1, float neg_refc,
-                                             float2& gs) {
+                                             float2& ga, float2& gb) {
     constexpr int kVec = Elt<DT>::kVec;
     float x[kVec];
     Elt<DT>::unpack(FIN ? raw : Clamp<DT>::apply(raw), x);
@@ -486,7 +508,8 @@ __device__ __forceinline__ void add_to_group(TileAccumulator<DT, K>& acc, const 
     for (int i = 0; i < kVec / 2; ++i) {
         float2 t = __ffma2_rn(make_float2(x[2 * i], x[2 * i + 1]), cc, rr);
         float2 e = make_float2(ex2_approx(t.x), ex2_approx(t.y));
-        gs = __fadd2_rn(gs, e);
+        if (i & 1) gb = __fadd2_rn(gb, e);
+        else ga = __fadd2_rn(ga, e);
         acc.A2[i] = __ffma2_rn(e, t, acc.A2[i]);
     }
 }
@@ -610,6 +633,13 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
                 const unsigned char* base = tiles + (size_t)s * kTileBytes;
                 const int v0 = (tb + t) * kTileVecs;
                 const int nv = min(kTileVecs, nvec - v0);
+                // (checked build) the tile lies inside the ring and inside the row
+                if (!AASD_IN_RANGE(s >= 0 && s < kStages && nv >= 1 && v0 >= 0 && v0 + nv <= nvec &&
+                                   (long long)info_row_ok(row_ctr, rj.n_rows), rj.state)) {
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sh.empty[s]);   // the stage goes back unread
+                    continue;
+                }
                 if (kLazyMax) tilemax.init();
                 if (ND > 0) {
                     // A thread takes the eight neighbouring vectors 8 * tid .. 8 * tid + 7 of the
@@ -623,21 +653,45 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
                     constexpr int kGroupsPerThread = kPer / kVecsPerGroup; // 2 or 1
                     static_assert(kPer == 8 && kGroupsPerThread >= 1, "eight vectors per thread and tile");
                     const int hsel = (lane >> 2) & 1, rot = lane & 3;
+                    // the groups' random variates need their indices only: issued first, the
+                    // generator's long dependent chain runs beside the exponentials below
+                    const int g0 = (v0 + kPer * tid) * kVec / kGroup;
+                    float inv_e[kGroupsPerThread][ND > 0 ? ND : 1];
+#pragma unroll
+                    for (int gi = 0; gi < kGroupsPerThread; ++gi)
+                        GroupRace<(ND > 0 ? ND : 1)>::inverse_variates(g0 + gi, row_ctr, job.smp, inv_e[gi]);
                     uint4 q[kPer];
-                    bool ok[kPer];
+                    // running sums of the vectors read at k < 4 and at k >= 4, two halves each
+                    float2 first = make_float2(0.f, 0.f), second = make_float2(0.f, 0.f);
+                    float2 first_b = make_float2(0.f, 0.f), second_b = make_float2(0.f, 0.f);
+                    if (nv == kTileVecs) {
 #pragma unroll
-                    for (int k = 0; k < kPer; ++k) {
-                        const int v = kPer * tid + (((((k >> 2) ^ hsel) & 1) << 2) | ((k + rot) & 3));
-                        ok[k] = v < nv;
-                        if (ok[k]) q[k] = lds16(base + (size_t)v * 16);
-                    }
-                    float2 first = make_float2(0.f, 0.f), second = make_float2(0.f, 0.f);   // k < 4, k >= 4
+                        for (int k = 0; k < kPer; ++k)
+                            q[k] = lds16(base + (size_t)(kPer * tid + (((((k >> 2) ^ hsel) & 1) << 2) | ((k + rot) & 3))) * 16);
 #pragma unroll
-                    for (int k = 0; k < kPer; ++k)
-                        if (ok[k]) {
-                            add_to_group<DT, K, FIN>(acc, q[k], c1, neg_refc, k < 4 ? first : second);
-                            tilemax.update(q[k]);
+                        for (int k = 0; k < kPer; ++k) {
+                            add_to_group<DT, K, FIN>(acc, q[k], c1, neg_refc, k < 4 ? first : second, k < 4 ? first_b : second_b);
+                            if (kLazyMax) tilemax.update(q[k]);
+                            else acc.track(q[k], v0 + kPer * tid + (((((k >> 2) ^ hsel) & 1) << 2) | ((k + rot) & 3)));
                         }
+                    } else {
+                        bool ok[kPer];
+#pragma unroll
+                        for (int k = 0; k < kPer; ++k) {
+                            const int v = kPer * tid + (((((k >> 2) ^ hsel) & 1) << 2) | ((k + rot) & 3));
+                            ok[k] = v < nv;
+                            if (ok[k]) q[k] = lds16(base + (size_t)v * 16);
+                        }
+#pragma unroll
+                        for (int k = 0; k < kPer; ++k)
+                            if (ok[k]) {
+                                add_to_group<DT, K, FIN>(acc, q[k], c1, neg_refc, k < 4 ? first : second, k < 4 ? first_b : second_b);
+                                if (kLazyMax) tilemax.update(q[k]);
+                                else acc.track(q[k], v0 + kPer * tid + (((((k >> 2) ^ hsel) & 1) << 2) | ((k + rot) & 3)));
+                            }
+                    }
+                    first = __fadd2_rn(first, first_b);
+                    second = __fadd2_rn(second, second_b);
                     float2 gs[kGroupsPerThread];
                     if (kGroupsPerThread == 2) {
                         gs[0] = hsel ? second : first;    // vectors 0-3 of the thread's share
@@ -645,11 +699,10 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
                     } else {
                         gs[0] = __fadd2_rn(first, second);
                     }
-                    const int g0 = (v0 + kPer * tid) * kVec / kGroup;
 #pragma unroll
                     for (int gi = 0; gi < kGroupsPerThread; ++gi) {
                         acc.S2[0] = __fadd2_rn(acc.S2[0], gs[gi]);
-                        if (g0 + gi < job.full_groups) race.offer(gs[gi].x + gs[gi].y, g0 + gi, row_ctr, job.smp);
+                        race.take(gs[gi].x + gs[gi].y, inv_e[gi], g0 + gi, g0 + gi < job.full_groups);
                     }
                 } else if (nv == kTileVecs) {
                     uint4 q[kTileVecs / kConsumers];
@@ -811,6 +864,33 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
             int row, chunk;
             decode_item(job, item, row, chunk);
             const char* rowp = row_pointer<DT>(rj, row);
+            int head, nvec, tb, te;
+            row_vectors<DT>(rowp, rj.vocab, head, nvec);
+            const char* vbase = rowp + (size_t)head * Elt<DT>::kSize;
+            tile_range(job, row, chunk, nvec, tb, te);
+            // The item's first tile is sent off before anything else: the loads that give the
+            // row's reference (two dependent trips to memory) then run while the copy is under
+            // way.  The tile is announced (the producer's arrival on the stage's barrier, which
+            // the phase needs whatever bytes have landed) only after the item's record is written.
+            unsigned int first_bytes = 0;
+            int first_stage = 0;
+            if (lane == 0) {
+                first_stage = it % kStages;
+                if (!mbar_wait(&sh.empty[first_stage], ((it / kStages) & 1u) ^ 1u, abort_flag, job.wait_limit)) {
+                    alive = false;
+                } else if (!(item == job.withhold_item && job.withhold_tile == 0)) {   // (testing aid)
+                    const long long off = (long long)tb * kTileBytes;
+                    const long long left = (long long)nvec * 16 - off;
+                    first_bytes = (unsigned int)(left < kTileBytes ? left : kTileBytes);
+                    if (!AASD_IN_RANGE(row >= 0 && row < rj.n_rows && off >= 0 && left > 0 &&
+                                       (long long)head * Elt<DT>::kSize + (long long)nvec * 16 <= (long long)rj.vocab * Elt<DT>::kSize &&
+                                       ((uintptr_t)(vbase + off) & 15u) == 0 && (first_bytes & 15u) == 0, rj.state))
+                        first_bytes = 0;
+                    else
+                    bulk_copy_g2s(tiles + (size_t)first_stage * kTileBytes, vbase + off, first_bytes, &sh.full[first_stage]);
+                    armed |= 1u << first_stage;
+                }
+            }
             // reference of the row: its hinted logit and its first entries
             const int hint = __ldg(job.hint_ids + row);
             const bool hint_ok = hint >= 0 && hint < rj.vocab;
@@ -822,21 +902,18 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
             for (int o = 4; o > 0; o >>= 1) r = fmaxf(r, __shfl_xor_sync(0xFFFFFFFFu, r, o));
             r = __shfl_sync(0xFFFFFFFFu, r, 0);
             if (!(fabsf(r) <= 3.0e38f)) r = 0.f;
-            if (lane == 0) {
+            if (lane == 0 && alive) {
                 ItemInfo& info = sh.ring[seq % kRing];
                 info.neg_refc = -(r * c1);
                 info.hint = hint;
                 info.hint_logit = hint_logit;
                 info.row = row;
                 info.chunk = chunk;
-                int head, nvec;
-                row_vectors<DT>(rowp, rj.vocab, head, nvec);
                 info.head = head;
                 info.nvec = nvec;
-                const char* vbase = rowp + (size_t)head * Elt<DT>::kSize;
-                int tb, te;
-                tile_range(job, row, chunk, nvec, tb, te);
-                for (int t = tb; t < te; ++t, ++it) {
+                if (first_bytes) mbar_arrive_expect_tx(&sh.full[first_stage], first_bytes);
+                ++it;
+                for (int t = tb + 1; t < te; ++t, ++it) {
                     const int s = it % kStages;
                     if (!mbar_wait(&sh.empty[s], ((it / kStages) & 1u) ^ 1u, abort_flag, job.wait_limit)) {
                         alive = false;
@@ -846,6 +923,9 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
                     const long long off = (long long)t * kTileBytes;
                     const long long left = (long long)nvec * 16 - off;
                     const unsigned int bytes = (unsigned int)(left < kTileBytes ? left : kTileBytes);
+                    if (!AASD_IN_RANGE(off >= 0 && left > 0 && ((uintptr_t)(vbase + off) & 15u) == 0 && (bytes & 15u) == 0,
+                                       rj.state))
+                        continue;
                     mbar_arrive_expect_tx(&sh.full[s], bytes);
                     bulk_copy_g2s(tiles + (size_t)s * kTileBytes, vbase + off, bytes, &sh.full[s]);
                     armed |= 1u << s;
@@ -928,6 +1008,14 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
         A = warp_sum_f64(A);
         if (TK) n_ahead = warp_sum_i64(n_ahead);
         u64 mk[K];   // merged vector keys, identical in every lane
+        // One item per CTA whose tiles all fit the ring (the small launches whose rows are cut
+        // into one cluster each): the tiles are still in shared memory, so the finisher finds the
+        // maximum's place there and hands on the best token itself instead of its vector: no
+        // trip to global memory on its way.
+        int item_tb, item_te;
+        tile_range(job, info.row, info.chunk, nvec, item_tb, item_te);
+        const bool resident = K == 1 && job.cluster_pieces && (tiles_of(nvec) + chunks - 1) / chunks <= kStages;
+        const VectorSource vsrc{vbase, resident ? tiles : nullptr, item_tb};
         if (K == 1) {
             // the consumers reported (maximum, lanes holding it) per warp: find the first vector
             // of the item that attains the maximum
@@ -938,8 +1026,7 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
                 const float m = unordered_bits(best);
                 const unsigned int mine = (lane < kConsumerWarps && top == best) ? (unsigned int)vk[0] : 0u;
                 int n_holders = __reduce_add_sync(0xFFFFFFFFu, __popc(mine));
-                int tb, te;
-                tile_range(job, info.row, info.chunk, nvec, tb, te);
+                const int tb = item_tb, te = item_te;
                 int vfirst = 0x7FFFFFFF;
                 if (n_holders <= 16) {
 #pragma unroll
@@ -949,15 +1036,26 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
                             const int l = __ffs(lanes) - 1;
                             lanes &= lanes - 1;
                             const int t = tb + (int)__shfl_sync(0xFFFFFFFFu, (unsigned int)my_tiles[w], l);
-                            const int v = first_vector_in_tile<DT, (ND > 0)>(vbase, nvec, t, w * 32 + l, m);
+                            const int v = first_vector_in_tile<DT, (ND > 0)>(vsrc, nvec, t, w * 32 + l, m);
                             if (v >= 0 && v < vfirst) vfirst = v;
                         }
                     }
                 } else {
-                    const int v = first_vector_of_range<DT>(vbase, nvec, tb, te, m);
+                    const int v = first_vector_of_range<DT>(vsrc, nvec, tb, te, m);
                     if (v >= 0) vfirst = v;
                 }
-                if (vfirst != 0x7FFFFFFF) mk[0] = make_vec_key(m, vfirst);
+                if (vfirst != 0x7FFFFFFF) {
+                    mk[0] = make_vec_key(m, vfirst);
+                    if (resident) {
+                        // the best token of that vector: the lowest id that holds the maximum
+                        float x[kVec];
+                        Elt<DT>::unpack(vsrc.load(vfirst), x);
+                        int first_i = kVec - 1;
+#pragma unroll
+                        for (int i = kVec - 1; i >= 0; --i) first_i = (x[i] == m) ? i : first_i;
+                        mk[0] = make_key(m, head + vfirst * kVec + first_i);
+                    }
+                }
             }
         } else {
 #pragma unroll
@@ -976,7 +1074,7 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
             // write their records into the first CTA's shared memory and signal its barrier;
             // the first CTA waits for them and carries on.  No trip through global memory.
             if (chunk != 0) {
-                if (lane == 0) {
+                if (lane == 0 && AASD_IN_RANGE(chunk > 0 && chunk < kMaxCluster, rj.state)) {
                     const unsigned int dst = cluster_map(&sh.cluster_piece[chunk], 0);
                     cluster_store_u64(dst + (unsigned int)offsetof(RowPartial, S), (u64)__double_as_longlong(S));
                     cluster_store_u64(dst + (unsigned int)offsetof(RowPartial, A), (u64)__double_as_longlong(A));
@@ -1031,7 +1129,9 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
             // pieces of a row meet in global memory; the last one to arrive carries on
             RowPartial* slots = rj.partials + (row - job.whole_rows) * chunks;
             int last = 0;
-            if (lane == 0) {
+            if (lane == 0 && AASD_IN_RANGE((row - job.whole_rows) * chunks + chunk >= 0 &&
+                                           (row - job.whole_rows + 1) * chunks <= (ND > 0 ? kRaceSlots : kPartialSlots) &&
+                                           row < rj.n_rows, rj.state)) {
                 RowPartial mine;
                 mine.S = S;
                 mine.A = A;
@@ -1106,7 +1206,9 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
 #pragma unroll
             for (int j = 0; j < K; ++j)
                 if (lane == j) mine = mk[j];
-            if (lane < K && mine != 0) {
+            if (resident) {
+                if (lane == 0 && mine != 0) key_insert<K>(ek, mine);   // already the row's best token
+            } else if (lane < K && mine != 0 && AASD_IN_RANGE(key_id(mine) >= 0 && key_id(mine) < nvec, rj.state)) {
                 const int vec = key_id(mine);
                 const uint4 q = __ldg(reinterpret_cast<const uint4*>(vbase) + vec);
                 float x[kVec];

@@ -9,6 +9,8 @@ constexpr int kMaxCands = 64;   // candidates per sequence a draft call can emit
 constexpr int kExtScan = 32;    // depths per main whose extra counts are fetched in parallel
 constexpr int kDraftThreads = 1024;   // one CTA per sequence: long histories want many lanes
 constexpr int kDraftWarps = kDraftThreads / 32;
+constexpr int kHitWords = 128;        // places per window of the lookup = 32 * kHitWords
+constexpr int kMatchBytes = 32768;    // histories up to this many tokens keep their match lengths in shared memory
 
 struct DraftArgs {
     aasd_draft_in in;
@@ -17,15 +19,27 @@ struct DraftArgs {
     DeviceState* state;
 };
 
-// One CTA per sequence.  Every history position p (the index right after a possible key
-// occurrence) is scored by the length of the common suffix of hist[..p) and the key; the
-// positions that reach the best length are the lookup result of Algorithm 1's dictionary
-// for the longest key that has one (Sec. 3.1: longer keys first).  Warp ballots compact the
-// hits in descending position order.
+// A place of the external pool in the lists of places (history places are >= 1).
+__device__ __forceinline__ int pool_place(int p) { return -2 - p; }
+__device__ __forceinline__ bool is_pool_place(int code) { return code <= -2; }
+__device__ __forceinline__ int place_of(int code) { return code <= -2 ? -2 - code : code; }
+
+// One CTA per sequence.  Every place p of the sequence's token buffer (the index right after a
+// possible key occurrence, with a continuation behind it) is scored by the length of the common
+// suffix of the tokens in front of it and the key; the places that reach the best length are
+// the lookup result of Algorithm 1's dictionary for the longest key that has one (Sec. 3.1:
+// longer keys first).  An external pool (a second token buffer shared by all sequences, NONE
+// between its documents) is scored the same way and its places come after the sequence's own.
+// The places are found in two sweeps: the best length (block-wide maximum), then one bit per
+// place that reaches it, written by warp ballots into a bit field in shared memory (a window
+// of 4096 places at a time, from the top down, until enough places are found) from which one
+// warp reads the places off in descending order.
 __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs a) {
     __shared__ int s_rec[AASD_MAX_NGRAM];
-    __shared__ int s_pos[kMaxCands];
-    __shared__ int s_warp[kDraftWarps];
+    __shared__ int s_pos[kMaxCands];        // places of the mains (pool places encoded)
+    __shared__ int s_len[kMaxCands];        // and how many tokens follow them
+    __shared__ unsigned int s_hits[kHitWords];
+    __shared__ unsigned char s_m[kMatchBytes];   // match length of every place of the history (short histories)
     __shared__ int s_count;
     __shared__ int s_kstar;
     __shared__ unsigned char s_next[kMaxCands * kExtScan];
@@ -44,6 +58,9 @@ __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs a)
     const bool have_align = a.in.align_ids != nullptr && a.in.align_n != nullptr && K > 0;
     const bool match_align = have_align && (a.p.flags & AASD_DRAFT_MATCH_ALIGN);
     const int64_t arow0 = have_align ? (int64_t)a.in.align_row_offsets[b] : 0;
+    const int32_t* pool = a.in.pool_ids;
+    const int pool_len = pool != nullptr ? a.in.pool_len : 0;
+    const bool have_pool_align = pool_len > 0 && a.in.pool_align_ids != nullptr && a.in.pool_align_n != nullptr && K > 0;
 
     int rl;
     if (a.in.recent_ids) {
@@ -64,6 +81,11 @@ __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs a)
         return min(K, max(0, a.in.align_n[arow0 + q - 1]));
     };
     auto ext = [&](int q, int s) -> int { return a.in.align_ids[(arow0 + q - 1) * K + s]; };
+    auto n_pool_ext = [&](int q) -> int {
+        if (!have_pool_align || q < 1 || q >= pool_len) return 0;
+        return min(K, max(0, a.in.pool_align_n[q - 1]));
+    };
+    auto pool_ext = [&](int q, int s) -> int { return a.in.pool_align_ids[(int64_t)(q - 1) * K + s]; };
     auto match_len_at = [&](int p) -> int {
         const int lim = min(min(n, p), rl);
         int m = 0;
@@ -79,39 +101,98 @@ __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs a)
         }
         return m;
     };
+    // a place of the pool: NONE equals no key token (keys hold tokens, and a key slot that is
+    // NONE must not match a document boundary), and a place on a boundary has no continuation
+    auto pool_match_len_at = [&](int p) -> int {
+        if (pool[p] == AASD_NONE) return 0;
+        const int lim = min(min(n, p), rl);
+        int m = 0;
+        for (int j = 1; j <= lim; ++j) {
+            const int t = pool[p - j];
+            if (t == AASD_NONE || t != s_rec[rl - j]) break;
+            m = j;
+        }
+        return m;
+    };
 
-    // pass 1: the longest key that occurs at a place with a continuation (p < len)
+    // sweep 1: the longest key that occurs at a place with a continuation (the lengths are kept
+    // for sweep 2 when the history is short enough)
+    const bool cached = len <= kMatchBytes;
     int best = 0;
-    for (int p = 1 + tid; p < len; p += kDraftThreads) best = max(best, match_len_at(p));
+    {
+        // A place matches at all only if the token in front of it is the key's last one (or, with
+        // the table, one of that position's extras): the tokens of eight places are fetched
+        // together, so that their trips to memory overlap, and the full comparison runs for
+        // the few places that pass this test.
+        constexpr int kBatch = 8;
+        const int want_last = rl > 0 ? s_rec[rl - 1] : AASD_NONE;
+        for (int base = 1 + tid; base < len; base += kBatch * kDraftThreads) {
+            int front[kBatch];
+#pragma unroll
+            for (int u = 0; u < kBatch; ++u) {
+                const int p = base + u * kDraftThreads;
+                front[u] = p < len ? h[p - 1] : AASD_NONE;
+            }
+#pragma unroll
+            for (int u = 0; u < kBatch; ++u) {
+                const int p = base + u * kDraftThreads;
+                if (p >= len) break;
+                const int m = (rl > 0 && (front[u] == want_last || match_align)) ? match_len_at(p) : 0;
+                if (cached) s_m[p] = (unsigned char)m;
+                best = max(best, m);
+            }
+        }
+    }
+    for (int p = 1 + tid; p < pool_len; p += kDraftThreads) best = max(best, pool_match_len_at(p));
     best = __reduce_max_sync(0xFFFFFFFFu, best);
     if (lane == 0 && best > 0) atomicMax(&s_kstar, best);
     __syncthreads();
     const int kstar = s_kstar;
 
-    // pass 2: its places, most recent first
+    // sweep 2: its places, the sequence's own first, most recent first within a source, in
+    // windows of 32 * kHitWords places from the top down
     if (kstar > 0) {
-        for (int base = len - 1; base >= 1; base -= kDraftThreads) {
-            const int p = base - tid;
-            const bool hit = p >= 1 && match_len_at(p) == kstar;
-            const unsigned int bal = __ballot_sync(0xFFFFFFFFu, hit);
-            if (lane == 0) s_warp[warp] = __popc(bal);
-            __syncthreads();
-            // hits of the warps before this one: every warp scans the per-warp counts itself
-            const int mine = lane < kDraftWarps ? s_warp[lane] : 0;
-            int incl = mine;
+        for (int src = 0; src < 2; ++src) {
+            const int top = src == 0 ? len : pool_len;     // places 1 .. top - 1
+            for (int hi = top; hi > 1 && s_count < max_cands; hi -= 32 * kHitWords) {
+                const int lo = max(1, hi - 32 * kHitWords);   // window [lo, hi)
+                const int words = (hi - lo + 31) / 32;
+                for (int wd = warp; wd < words; wd += kDraftWarps) {
+                    const int p = lo + wd * 32 + lane;
+                    const bool hit = p < hi && (src == 0 ? (cached ? (int)s_m[p] : match_len_at(p)) : pool_match_len_at(p)) == kstar;
+                    const unsigned int bal = __ballot_sync(0xFFFFFFFFu, hit);
+                    if (lane == 0) s_hits[wd] = bal;
+                }
+                __syncthreads();
+                if (warp == 0) {
+                    int count = s_count;
+                    for (int base = words - 1; base >= 0 && count < max_cands; base -= 32) {
+                        const int wd = base - lane;              // lane 0 takes the highest word
+                        const unsigned int bits = wd >= 0 ? s_hits[wd] : 0u;
+                        const int mine = __popc(bits);
+                        int incl = mine;
 #pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const int up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-                if (lane >= o) incl += up;
+                        for (int o = 1; o < 32; o <<= 1) {
+                            const int up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                            if (lane >= o) incl += up;
+                        }
+                        int rank = count + incl - mine;          // places of higher words come first
+                        unsigned int left = bits;
+                        while (left && rank < max_cands) {
+                            const int bit = 31 - __clz(left);    // the highest place of the word first
+                            left &= ~(1u << bit);
+                            const int p = lo + wd * 32 + bit;
+                            if (!AASD_IN_RANGE(rank >= 0 && rank < kMaxCands && p >= 1 && p < top && wd >= 0 && wd < kHitWords,
+                                               a.state))
+                                break;
+                            s_pos[rank++] = src == 0 ? p : pool_place(p);
+                        }
+                        count += __shfl_sync(0xFFFFFFFFu, incl, 31);
+                    }
+                    if (lane == 0) s_count = min(count, max_cands);
+                }
+                __syncthreads();
             }
-            const int before = s_count + __shfl_sync(0xFFFFFFFFu, incl - mine, warp);
-            const int total = __shfl_sync(0xFFFFFFFFu, incl, 31);
-            const int rank = before + __popc(bal & ((1u << lane) - 1u));
-            if (hit && rank < max_cands) s_pos[rank] = p;
-            __syncthreads();
-            if (tid == 0) s_count += total;
-            __syncthreads();
-            if (s_count >= max_cands) break;
         }
     }
     const int n_main = min(s_count, max_cands);
@@ -120,32 +201,53 @@ __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs a)
     uint8_t* d_fl = a.out.draft_flags + (int64_t)b * max_cands * draft_len;
     int32_t* c_len = a.out.cand_len + (int64_t)b * max_cands;
     int32_t* c_pos = a.out.cand_pos + (int64_t)b * max_cands;
+    // how many tokens follow each main: up to draft_len, to the end of its buffer, and in the
+    // pool to the end of the document
+    for (int c = tid; c < n_main; c += kDraftThreads) {
+        const int code = s_pos[c], p = place_of(code);
+        int L;
+        if (!is_pool_place(code)) {
+            L = min(draft_len, len - p);
+        } else {
+            L = 0;
+            while (L < draft_len && p + L < pool_len && pool[p + L] != AASD_NONE) ++L;
+        }
+        s_len[c] = L;
+    }
+    __syncthreads();
     for (int i = tid; i < max_cands * draft_len; i += kDraftThreads) {
         const int c = i / draft_len, j = i % draft_len;
         int tok = AASD_NONE;
         unsigned int fl = 0;
-        if (c < n_main) {
-            const int q = s_pos[c] + j;
-            if (q < len) {
+        if (c < n_main && j < s_len[c]) {
+            const int code = s_pos[c], q = place_of(code) + j;
+            if (!AASD_IN_RANGE(q >= 0 && q < (is_pool_place(code) ? pool_len : len), a.state)) continue;
+            if (!is_pool_place(code)) {
                 tok = h[q];
                 fl = (q < plen) ? AASD_FLAG_CONDITIONAL : 0u;
+            } else {
+                tok = pool[q];      // not input context: verified strictly
             }
         }
         d_ids[i] = tok;
         d_fl[i] = (uint8_t)fl;
     }
     for (int c = tid; c < max_cands; c += kDraftThreads) {
-        c_len[c] = c < n_main ? min(draft_len, len - s_pos[c]) : 0;
+        c_len[c] = c < n_main ? s_len[c] : 0;
         c_pos[c] = c < n_main ? s_pos[c] : AASD_NONE;
     }
     // how many extras each (main, depth) has: fetched by all threads at once, so that the
     // serial walk below does not pay a trip to memory per step
+    const bool any_table = have_align || have_pool_align;
     const int scan = min(draft_len, kExtScan);
-    if (have_align && n_main < max_cands) {
+    auto extras_at = [&](int c, int depth) -> int {
+        const int code = s_pos[c], q = place_of(code) + depth;
+        return is_pool_place(code) ? n_pool_ext(q) : n_ext(q);
+    };
+    if (any_table && n_main < max_cands) {
         for (int i = tid; i < n_main * scan; i += kDraftThreads) {
             const int c = i / scan, depth = i % scan;
-            const int p = s_pos[c];
-            s_next[c * kExtScan + depth] = (unsigned char)(depth < min(draft_len, len - p) ? n_ext(p + depth) : 0);
+            s_next[c * kExtScan + depth] = (unsigned char)(depth < s_len[c] ? extras_at(c, depth) : 0);
         }
     }
     __syncthreads();
@@ -155,11 +257,10 @@ __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs a)
     // the counts in shared memory; all threads then write the tokens.
     if (tid == 0) {
         int total = n_main;
-        for (int c = 0; c < n_main && total < max_cands && have_align; ++c) {
-            const int p = s_pos[c];
-            const int L = min(draft_len, len - p);
+        for (int c = 0; c < n_main && total < max_cands && any_table; ++c) {
+            const int L = s_len[c];
             for (int i = 0; i < L && total < max_cands; ++i) {
-                const int ne = i < scan ? (int)s_next[c * kExtScan + i] : n_ext(p + i);
+                const int ne = i < scan ? (int)s_next[c * kExtScan + i] : extras_at(c, i);
                 for (int s = 0; s < ne && total < max_cands; ++s) {
                     s_alt[total] = (c << 16) | (s << 12) | 0;   // main and extra slot; the depth goes beside
                     s_alt_depth[total] = i;
@@ -176,15 +277,16 @@ __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs a)
     for (int i = tid; i < (total - n_main) * draft_len; i += kDraftThreads) {
         const int slot = n_main + i / draft_len, q = i % draft_len;
         const int c = s_alt[slot] >> 16, es = (s_alt[slot] >> 12) & 15, depth = s_alt_depth[slot];
-        const int p = s_pos[c];
+        const int code = s_pos[c], p = place_of(code);
+        const bool from_pool = is_pool_place(code);
         if (q < depth) {
-            d_ids[slot * draft_len + q] = h[p + q];
-            d_fl[slot * draft_len + q] = (uint8_t)((p + q < plen) ? AASD_FLAG_CONDITIONAL : 0u);
+            d_ids[slot * draft_len + q] = from_pool ? pool[p + q] : h[p + q];
+            d_fl[slot * draft_len + q] = (uint8_t)((!from_pool && p + q < plen) ? AASD_FLAG_CONDITIONAL : 0u);
         } else if (q == depth) {
-            d_ids[slot * draft_len + q] = ext(p + depth, es);
+            d_ids[slot * draft_len + q] = from_pool ? pool_ext(p + depth, es) : ext(p + depth, es);
             d_fl[slot * draft_len + q] = (uint8_t)(AASD_FLAG_CONDITIONAL | AASD_FLAG_EXTRA);
             c_len[slot] = depth + 1;
-            c_pos[slot] = p;
+            c_pos[slot] = code;
         }
     }
 }

@@ -17,6 +17,8 @@ int launch_tree_bf16(const LaunchEnv& env, const StreamJob* sj, const TreeArgs& 
     if (sj) {
         if (a.mode == AASD_VERIFY_STRICT_SAMPLED)
             return launch_stream<DT, 1, 1, false, false, TreeEpilogue<DT>>(env, *sj, a, grid, false);
+        if (a.mode == AASD_VERIFY_TOP_K)   // the consumers also count the tokens ahead of each row's first child
+            return launch_stream<DT, 1, 0, true, false, TreeEpilogue<DT>>(env, *sj, a, grid, false);
         return launch_stream<DT, 1, 0, false, false, TreeEpilogue<DT>>(env, *sj, a, grid, false);
     }
     launch(tree_kernel<DT>, grid, (unsigned int)kThreads, 0, env.stream, a);

@@ -104,6 +104,8 @@ struct TreeRowStat {
     float neg_refc, m;
     int own;     // the target's own token of the row (argmax or keyed draw), NONE on a bad row
     int flags;   // bit 0: bad row, bit 1: sums are max-centred
+    int ahead;   // top-k mode: tokens ahead of the row's hinted token (its first child's), -1: not counted
+    int pad;
 };
 
 struct TreeArgs {
@@ -115,6 +117,7 @@ struct TreeArgs {
     int n_trees;
     float alpha, beta;
     int mode;
+    int top_k;                    // TOP_K mode
     int emit_stride;
     SampleJob smp;
     int32_t* hint;                // scratch [n_rows]: token of each row's first child
@@ -167,9 +170,22 @@ __global__ void tree_empty_kernel(const TreeArgs a) {
 
 // Row epilogue, entered by a whole warp.  Phase one (lane 0): the row's statistics.  Phase
 // two (the warp that completes the tree): nodes, paths, result.
+// Tokens of a row that are ahead of token d (raw logit xd) in the order (logit descending, id
+// ascending), counted by a whole warp going over the row: the slow, exact way.
+template <int DT>
+__device__ int warp_count_ahead(const char* rowp, int V, int d, float xd) {
+    int n = 0;
+    for (int i = threadIdx.x & 31; i < V; i += 32) {
+        const float x = Elt<DT>::load(rowp, i);
+        n += (x > xd || (x == xd && i < d)) ? 1 : 0;
+    }
+    return __reduce_add_sync(0xFFFFFFFFu, n);
+}
+
+// ahead: the streaming pass's count for the row's hinted token (top-k mode), or -1.
 template <int DT>
 __device__ void tree_finish_warp(const TreeArgs& a, const RowJob& job, int64_t row, const RowPartial& merged,
-                                 float neg_refc, bool centered, int sampled, Tally& tally) {
+                                 float neg_refc, bool centered, int sampled, int ahead, Tally& tally) {
     const int lane = threadIdx.x & 31;
     int t = 0, last = 0;
     int64_t lo = 0, hi = 0;
@@ -184,6 +200,8 @@ __device__ void tree_finish_warp(const TreeArgs& a, const RowJob& job, int64_t r
         st.m = f.m;
         st.own = f.bad ? AASD_NONE : (a.mode == AASD_VERIFY_STRICT_SAMPLED ? sampled : f.top1);
         st.flags = (f.bad ? 1 : 0) | (centered ? 2 : 0);
+        st.ahead = ahead;
+        st.pad = 0;
         a.stats[row] = st;
         if (a.out.entropy) a.out.entropy[row] = (float)f.H;
         if (a.out.pmax) a.out.pmax[row] = (float)f.pmax;
@@ -216,21 +234,24 @@ __device__ void tree_finish_warp(const TreeArgs& a, const RowJob& job, int64_t r
     __threadfence();
     const int n = (int)(hi - lo);
 
-    // every node's own accept bit, judged with its parent's row (Eq. 3-6 / strict)
+    // every node's own accept bit, judged with its parent's row (Eq. 3-6 / top-k / strict)
     unsigned int n_near = 0, n_acc = 0, status = 0;
-    for (int v = lane; v < n; v += 32) {
+    for (int base = 0; base < n; base += 32) {
+        const int v = base + lane;
         const int64_t g = lo + v;
-        const int p = v == 0 ? AASD_NONE : a.node_parent[g];
+        const int p = (v == 0 || v >= n) ? AASD_NONE : a.node_parent[g];
         double pt = 0.0;
-        bool acc = false;
+        bool acc = false, rank_wanted = false;
+        int d = AASD_NONE, n_ahead = AASD_NONE;
+        float x = 0.f;
         if (p >= 0 && p < v) {
             const TreeRowStat* ps = a.stats + lo + p;
-            const int d = a.node_token[g];
+            d = a.node_token[g];
             const bool d_ok = d >= 0 && d < job.vocab;
             if (!d_ok && d != AASD_NONE) status |= AASD_STATUS_ID_RANGE;
             const int pflags = __ldcg(&ps->flags);
             if (d_ok && !(pflags & 1)) {
-                const float x = Elt<DT>::load(row_pointer<DT>(job, lo + p), d);
+                x = Elt<DT>::load(row_pointer<DT>(job, lo + p), d);
                 RowFinal f;
                 f.c1 = (double)job.c1;
                 f.neg_refc = (double)__ldcg(&ps->neg_refc);
@@ -243,15 +264,38 @@ __device__ void tree_finish_warp(const TreeArgs& a, const RowJob& job, int64_t r
                     const bool at_max = (x == __ldcg(&ps->m));
                     acc = at_max || (pt >= lin);
                     if (!at_max && fabs(pt - lin) <= 1.0e-6) n_near += 1;
+                } else if (a.mode == AASD_VERIFY_TOP_K && (flag & AASD_FLAG_CONDITIONAL)) {
+                    rank_wanted = x > -CUDART_INF_F;     // a masked token has no rank and never passes
                 } else {
                     acc = (d == __ldcg(&ps->own));
                 }
+                if (a.mode == AASD_VERIFY_TOP_K && x > -CUDART_INF_F) {
+                    // the streaming pass counted for the parent's first child; siblings are counted below
+                    const int counted = __ldcg(&ps->ahead);
+                    if (counted >= 0 && d == __ldcg(a.hint + lo + p)) n_ahead = counted;
+                    else n_ahead = -2;   // to be counted
+                }
             }
         }
-        if (a.out.p_token) a.out.p_token[g] = (float)pt;
-        if (a.out.accept) a.out.accept[g] = acc ? 1 : 0;
-        a.node_ok[g] = acc ? 1 : 0;
-        n_acc += acc ? 1 : 0;
+        if (a.mode == AASD_VERIFY_TOP_K) {
+            unsigned int todo = __ballot_sync(0xFFFFFFFFu, n_ahead == -2);
+            while (todo) {
+                const int l = __ffs(todo) - 1;
+                todo &= todo - 1;
+                const int pp = __shfl_sync(0xFFFFFFFFu, p, l), dd = __shfl_sync(0xFFFFFFFFu, d, l);
+                const float xx = __shfl_sync(0xFFFFFFFFu, x, l);
+                const int cnt = warp_count_ahead<DT>(row_pointer<DT>(job, lo + pp), job.vocab, dd, xx);
+                if (lane == l) n_ahead = cnt;
+            }
+            if (rank_wanted) acc = n_ahead >= 0 && n_ahead < a.top_k;
+        }
+        if (v < n) {
+            if (a.out.p_token) a.out.p_token[g] = (float)pt;
+            if (a.out.accept) a.out.accept[g] = acc ? 1 : 0;
+            if (a.out.n_greater) a.out.n_greater[g] = (a.mode == AASD_VERIFY_TOP_K && n_ahead >= 0) ? n_ahead : AASD_NONE;
+            a.node_ok[g] = acc ? 1 : 0;
+            n_acc += acc ? 1 : 0;
+        }
     }
     __syncwarp();
     n_near = __reduce_add_sync(0xFFFFFFFFu, n_near);
@@ -310,7 +354,12 @@ struct TreeEpilogue {
         if (ND > 0 && !partial_bad(fr.merged))
             sampled = warp_sample_decide<DT>(rowp, job.vocab, (unsigned int)row, 0, a.smp, races[0], tail_group,
                                              fr.centered, tally.recheck, tally.exhaustive);
-        tree_finish_warp<DT>(a, job, row, fr.merged, fr.neg_refc, fr.centered, sampled, tally);
+        // top-k mode: the streaming pass counted the tokens ahead of the hinted token (exact when
+        // the hint is a token of the vocabulary that is not masked)
+        const bool counted = a.mode == AASD_VERIFY_TOP_K && info.hint >= 0 && info.hint < job.vocab &&
+                             info.hint_logit > -CUDART_INF_F;
+        tree_finish_warp<DT>(a, job, row, fr.merged, fr.neg_refc, fr.centered, sampled,
+                             counted ? (int)fr.merged.ahead : -1, tally);
     }
 };
 
@@ -335,7 +384,7 @@ __global__ void __launch_bounds__(kThreads) tree_kernel(const TreeArgs a) {
         sampled = warp_sample_exhaustive<DT>(rowp, job.vocab, (unsigned int)row, 0, a.smp);
         tally.exhaustive += 1;
     }
-    tree_finish_warp<DT>(a, job, row, sc.merged, neg_refc, centered, sampled, tally);
+    tree_finish_warp<DT>(a, job, row, sc.merged, neg_refc, centered, sampled, -1, tally);
     if (threadIdx.x == 0) tally.flush(job.state);
 }
 

@@ -94,8 +94,8 @@ def test_host_side_errors_of_tree_and_top_k_calls(ctx):
     tok = torch.tensor([-1, 1, 2, 3], dtype=torch.int32, device="cuda")
     par = torch.tensor([-1, 0, 1, 1], dtype=torch.int32, device="cuda")
     with pytest.raises(binding.AasdError) as e:
-        ctx.verify_tree(x, tok, par, [0, 4], 3, mode=binding.VERIFY_TOP_K)
-    assert e.value.code == 7
+        ctx.verify_tree(x, tok, par, [0, 4], 3, mode=binding.VERIFY_TOP_K, top_k=0)
+    assert e.value.code == 1
     with pytest.raises(binding.AasdError) as e:
         ctx.verify_tree(x, tok, par, [0, 4], 0)
     assert e.value.code == 2

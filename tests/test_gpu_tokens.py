@@ -98,6 +98,80 @@ def test_draft_long_history_many_matches(ctx):
         assert ref["match_len"][0] >= 1
 
 
+def test_draft_histories_longer_than_one_window(ctx):
+    # the lookup reads the places off a bit field of 4096 places per window, from the top down:
+    # a 150k-token history with rare matches, some right at window edges, and caps that are
+    # reached after a few windows
+    rng = np.random.default_rng(8)
+    L = 150000
+    hist = rng.integers(0, 40, L).astype(np.int32)
+    key = np.array([41, 42, 43], np.int32)                 # occurs only where planted
+    planted = [70, 3000, 18925, 18928, 18931, 70000, L - 16 * 4096 - 3, L - 16 * 4096, L - 16 * 4096 + 3, 140000,
+               L - 30]   # three of them around a window edge
+    for p in planted:
+        hist[p - 3:p] = key
+    hist[L - 3:] = key
+    buf = np.full(L + 8, -1, np.int32)
+    buf[:L] = hist
+    offs = np.array([0, L + 8], np.int32)
+    for max_cands in (64, 5, 1):
+        ref = oracle.draft(buf, offs, [L], [L], key[None, :], [3], 3, 4, max_cands)
+        got = ctx.draft(_dev(buf), _dev(offs), _dev([L]), _dev([L]), 3, 4, max_cands, recent_ids=_dev(key[None, :]),
+                        recent_len=_dev([3]))
+        check_draft(got, ref)
+        assert ref["cand_pos"][0, :ref["n_cands"][0]].tolist() == sorted(planted, reverse=True)[:max_cands]
+
+
+def _pool_case(rng, B, alphabet, max_len, pool_len, K, tables, n):
+    c = _draft_case(rng, B, alphabet, max_len, K, tables, n, own_tail=bool(rng.integers(0, 2)))
+    pool = rng.integers(0, alphabet, pool_len).astype(np.int32)
+    pool[rng.random(pool_len) < 0.05] = -1                 # document boundaries
+    c["pool"] = pool
+    c["pool_align_ids"] = c["pool_align_n"] = None
+    if tables:
+        c["pool_align_ids"] = np.full((pool_len, K), -1, np.int32)
+        c["pool_align_n"] = np.zeros(pool_len, np.int32)
+        for r in range(pool_len):
+            k = int(rng.integers(0, K + 1))
+            c["pool_align_ids"][r, :k] = rng.choice(alphabet + 3, size=k, replace=False) + 100
+            c["pool_align_n"][r] = k
+    return c
+
+
+@pytest.mark.parametrize("alphabet,max_len,pool_len", [(3, 40, 1), (4, 200, 300), (30, 800, 70000), (6, 30, 5000)])
+@pytest.mark.parametrize("tables", [False, True])
+def test_draft_with_an_external_pool(ctx, alphabet, max_len, pool_len, tables):
+    """A second token buffer, shared by all sequences, looked up like the history (Limitations);
+    its places follow the history's, its tokens are verified strictly, its own table gives
+    alternatives."""
+    rng = np.random.default_rng(alphabet + max_len + pool_len + tables)
+    for trial in range(3):
+        B = int(rng.integers(1, 10))
+        n = int(rng.integers(1, 7))
+        draft_len = int(rng.integers(1, 10))
+        max_cands = int(rng.integers(1, 12))
+        K = 2
+        c = _pool_case(rng, B, alphabet, max_len, pool_len, K, tables, n)
+        ref = oracle.draft(c["hist"], c["offs"], c["lens"], c["plens"], c["recent"], c["rlen"], n, draft_len,
+                           max_cands, align_ids=c["align_ids"], align_n=c["align_n"],
+                           align_row_offsets=None if c["arow"] is None else c["arow"][:-1], k_extra=K if tables else 0,
+                           pool_ids=c["pool"], pool_align_ids=c["pool_align_ids"], pool_align_n=c["pool_align_n"])
+        kw = {}
+        if tables:
+            kw = dict(align_ids=_dev(c["align_ids"]), align_n=_dev(c["align_n"]), align_row_offsets=_dev(c["arow"][:-1]),
+                      pool_align_ids=_dev(c["pool_align_ids"]), pool_align_n=_dev(c["pool_align_n"]))
+        got = ctx.draft(_dev(c["hist"]), _dev(c["offs"]), _dev(c["lens"]), _dev(c["plens"]), n, draft_len, max_cands,
+                        recent_ids=_dev(c["recent"]), recent_len=_dev(c["rlen"]), pool_ids=_dev(c["pool"]), **kw)
+        check_draft(got, ref)
+        used = ref["cand_pos"][ref["cand_pos"] <= -2]
+        if pool_len >= 1000 and max_len <= 40:
+            assert used.size > 0                         # short histories: the pool did supply candidates
+        # pool tokens are never eligible for conditional verification unless they are extras
+        from_pool = np.repeat((ref["cand_pos"] <= -2)[:, :, None], draft_len, axis=2)
+        fl = ref["draft_flags"]
+        assert ((fl[from_pool] == 0) | (fl[from_pool] == 3)).all()
+
+
 def test_select_and_append_parity(ctx):
     rng = np.random.default_rng(9)
     B, L = 37, 6

@@ -79,7 +79,7 @@ TREE_CASES = [
 
 @pytest.mark.parametrize("V,dtype,stride,B,Cm,Ld", TREE_CASES)
 @pytest.mark.parametrize("mode", [binding.VERIFY_CONDITIONAL, binding.VERIFY_STRICT_GREEDY,
-                                  binding.VERIFY_STRICT_SAMPLED])
+                                  binding.VERIFY_STRICT_SAMPLED, binding.VERIFY_TOP_K])
 def test_verify_tree_parity(ctx, V, dtype, stride, B, Cm, Ld, mode):
     rng = np.random.default_rng(V + B + mode)
     d, f, clen, nc = _random_candidates(rng, B, Cm, Ld, 6)
@@ -99,6 +99,9 @@ def test_verify_tree_parity(ctx, V, dtype, stride, B, Cm, Ld, mode):
                 hints[lo + par[lo + v]] = tok[lo + v]
     recipe = synth.LogitRecipe(sigma=2.5, p_hint=0.8, p_random=0.1, spike_lo=9, spike_hi=16)
     x = synth.logits(R, V, dtype, recipe, torch.as_tensor(hints), 900 + V)
+    if mode == binding.VERIFY_TOP_K and R > 6:
+        x[2, :] = x[2, 0]                                        # every token equal: ids decide the ranks
+        x[4, int(tok[5]) if tok[5] >= 0 else 0] = -float("inf")  # a masked token somewhere
     if stride is not None:
         buf = torch.zeros((R, stride), dtype=dtype)
         buf[:, :V] = x
@@ -106,18 +109,23 @@ def test_verify_tree_parity(ctx, V, dtype, stride, B, Cm, Ld, mode):
     alpha, beta, seed, step = F32(0.1), F32(0.05), 77, 4
     E = Ld + 1
     ref = oracle.verify_tree(to_oracle(x), tok, par, offs, E, node_flags=fl, alpha=alpha, beta=beta, mode=mode,
-                             seed=seed, step=step)
+                             seed=seed, step=step, top_k=3)
     base = x._base if x._base is not None else x
     xd = base.cuda()[:, :V] if base.shape != x.shape else base.cuda()
     got = ctx.verify_tree(xd, _dev(tok), _dev(par), offs, E, node_flags=_dev(fl, torch.uint8), alpha=alpha,
-                          beta=beta, mode=mode, seed=seed, step=step)
+                          beta=beta, mode=mode, seed=seed, step=step, top_k=3)
     near = _check_tree(got, ref, dtype)
     assert near == 0
+    if mode == binding.VERIFY_TOP_K:
+        # the count is an integer and must be exact, for first children (counted while the row
+        # streams) and for their siblings (counted by a second pass over the row)
+        assert np.array_equal(cpu(got["n_greater"]), ref["n_greater"])
+        assert B == 1 or (ref["n_greater"] >= 0).sum() > 0
     if B >= 8:
         assert ref["n_accept"].max() >= 1
     assert ctx.poll_status() == 0
     again = ctx.verify_tree(xd, _dev(tok), _dev(par), offs, E, node_flags=_dev(fl, torch.uint8), alpha=alpha,
-                            beta=beta, mode=mode, seed=seed, step=step)
+                            beta=beta, mode=mode, seed=seed, step=step, top_k=3)
     for k in ("accept", "best_node", "emit_ids", "p_token", "entropy"):
         assert torch.equal(got[k], again[k]), k
 
