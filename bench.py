@@ -815,10 +815,10 @@ def run_micro(args):
                               finite_hint=FINITE_HINT)
         elif args.micro == "verify-sampled":
             outs = ctx.verify(bufs[j], ids[j], None, rows_per_cand=rpc, outputs=outs, seed=17, step=j,
-                              mode=binding.VERIFY_STRICT_SAMPLED)
+                              mode=binding.VERIFY_STRICT_SAMPLED, finite_hint=FINITE_HINT)
         elif args.micro == "align-gumbel":
             outs = ctx.align_sample(bufs[j], ids[j], offs, k_extra=K_EXTRA, outputs=outs, seed=17,
-                                    mode=binding.ALIGN_GUMBEL)
+                                    mode=binding.ALIGN_GUMBEL, finite_hint=FINITE_HINT)
         else:
             outs = ctx.align_sample(bufs[j], ids[j], offs, k_extra=K_EXTRA, outputs=outs, finite_hint=FINITE_HINT)
 

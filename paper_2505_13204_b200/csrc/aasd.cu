@@ -525,6 +525,7 @@ int aasd_step(aasd_ctx* ctx, const aasd_step_args* s, void* workspace, size_t wo
     // sequence's last candidate does both
     SeqTail tail{};
     tail.cands_per_seq = dp.max_cands;
+    tail.rows_per_seq = dp.max_cands * dp.draft_len;
     tail.emit_stride = dp.draft_len + 1;
     tail.best_cand = s->best_cand;
     tail.n_emit = s->n_emit;

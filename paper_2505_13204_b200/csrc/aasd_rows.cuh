@@ -337,6 +337,7 @@ __device__ inline RowFinal finish_row(const RowPartial& p, float c1, float neg_r
 struct SeqTail {
     int enabled;
     int cands_per_seq;
+    int rows_per_seq;            // cands_per_seq * rows per candidate
     int emit_stride;
     unsigned int* seq_tickets;   // [n_seqs], zero between launches
     int32_t* best_cand;
@@ -414,14 +415,14 @@ struct Tally {
 // its candidate) is taken right behind it, so that the stores of the row's outputs, which
 // nobody inside the launch reads, are under way while the ticket travels.  Returns the
 // ticket's value.
+// flag: the row's draft-token flag byte (AASD_FLAG_CONDITIONAL when the call has no flags).
 template <int DT>
 __device__ unsigned int verify_row(const VerifyArgs& a, const RowJob& job, int64_t row, const RowPartial& merged,
-                                   float neg_refc, bool centered, int d, float xd, int sampled, unsigned int* ticket,
-                                   Tally& tally) {
+                                   float neg_refc, bool centered, int d, float xd, unsigned int flag, int sampled,
+                                   unsigned int* ticket, Tally& tally) {
     const bool d_ok = d >= 0 && d < job.vocab;
     const RowFinal f = finish_row(merged, job.c1, neg_refc, centered);
     if (!AASD_IN_RANGE(row >= 0 && row < job.n_rows && (f.bad || (f.top1 >= 0 && f.top1 < job.vocab)), job.state)) return 0xFFFFFFFFu;
-    const unsigned int flag = a.draft_flags ? a.draft_flags[row] : AASD_FLAG_CONDITIONAL;
     const double lin = (double)a.alpha * f.H + (double)a.beta;
     const double thr = f.bad ? 0.0 : fmin(lin, f.pmax);
     const int own = a.mode == AASD_VERIFY_STRICT_SAMPLED ? sampled : f.top1;   // NONE on a bad row
@@ -507,20 +508,173 @@ __device__ inline int candidate_of_row(const VerifyArgs& a, int64_t n_rows, int6
     return c;
 }
 
-// Row epilogue of verification, run by a whole warp: lane 0 evaluates the row (Eq. 4-6), and
-// the warp that completes a candidate applies the prefix rule with one load per lane.
+// A row whose ticket has been taken but not looked at yet: what the warp needs to complete the
+// row's candidate once the ticket's value is in (lane 0's copy counts).
+struct PendingRow {
+    int valid;
+    int c;
+    int64_t lo, hi;
+    unsigned int ticket;
+    int whole_sequence;   // the ticket counts the rows of the candidate's whole sequence (see below)
+};
+
+// A launch that also selects and appends (SeqTail) with sequences of at most 32 rows counts
+// rows per sequence instead of rows per candidate: one ticket per row, and the warp that takes
+// a sequence's last one does everything for it with the rows' records in its lanes.
+__device__ __forceinline__ bool sequence_tickets(const VerifyArgs& a) {
+    return a.seq.enabled && a.seq.rows_per_seq <= 32;
+}
+
+// Row epilogue of verification, first half, run by a whole warp: lane 0 evaluates the row
+// (Eq. 4-6), writes its outputs and takes the ticket of its candidate.
+template <int DT>
+__device__ void verify_row_warp(const VerifyArgs& a, const RowJob& job, int64_t row, const RowPartial& merged,
+                                float neg_refc, bool centered, int d, float xd, unsigned int flag, int sampled,
+                                PendingRow& pending, Tally& tally) {
+    pending.valid = 1;
+    pending.c = 0;
+    pending.lo = pending.hi = 0;
+    pending.ticket = 0;
+    pending.whole_sequence = 0;
+    if ((threadIdx.x & 31) == 0) {
+        int64_t lo = 0, hi = 0;
+        int c = candidate_of_row(a, job.n_rows, row, lo, hi);
+        if (!AASD_IN_RANGE(c >= 0 && c < a.n_cands && lo >= 0 && lo <= row && row < hi && hi <= job.n_rows, job.state)) c = 0, hi = lo = 0;
+        pending.whole_sequence = sequence_tickets(a) ? 1 : 0;
+        unsigned int* ticket = pending.whole_sequence ? &a.seq.seq_tickets[c / a.seq.cands_per_seq] : &a.cand_tickets[c];
+        pending.ticket = verify_row<DT>(a, job, row, merged, neg_refc, centered, d, xd, flag, sampled, ticket, tally);
+        pending.c = c;
+        pending.lo = lo;
+        pending.hi = hi;
+    }
+}
+
+// Second half: the warp that took a candidate's last ticket applies the prefix rule with one
+// load per lane, and, when that completes a sequence, selects and appends.  The streaming
+// kernel runs it one row late, so that the ticket's trip to memory is hidden behind the next
+// row's work.
+__device__ inline void verify_complete_warp(const VerifyArgs& a, const RowJob& job, const PendingRow& pending, Tally& tally);
+
 template <int DT>
 __device__ void verify_finish_warp(const VerifyArgs& a, const RowJob& job, int64_t row, const RowPartial& merged,
-                                   float neg_refc, bool centered, int d, float xd, int sampled, Tally& tally) {
+                                   float neg_refc, bool centered, int d, float xd, unsigned int flag, int sampled,
+                                   Tally& tally) {
+    PendingRow pending;
+    verify_row_warp<DT>(a, job, row, merged, neg_refc, centered, d, xd, flag, sampled, pending, tally);
+    verify_complete_warp(a, job, pending, tally);
+}
+
+// Emission of a finished sequence b: the winning candidate's accepted draft tokens and the
+// target's own token go to emit_ids and to the history, their extras to the alignment table.
+// draft_token(i): token i of the winning candidate.
+template <class DraftToken>
+__device__ __forceinline__ void emit_and_append(const VerifyArgs& a, int b, int best, int best_a, int nt, int off, int cap,
+                                                int len, DraftToken draft_token, Tally& tally) {
     const int lane = threadIdx.x & 31;
-    int c = 0, last = 0;
-    int64_t lo = 0, hi = 0;
+    const int stride = a.seq.emit_stride;
+    int32_t* e = a.seq.emit_ids + (int64_t)b * stride;
+    int ne = 0;
+    if (best != AASD_NONE) {
+        ne = min(best_a, stride);
+        if (nt != AASD_NONE && ne < stride) ne += 1;
+    }
+    for (int base = 0; base < stride; base += 32) {
+        const int i = base + lane;
+        const int drafted = draft_token(i < best_a ? i : 0);     // (a shuffle: every lane takes part)
+        if (i < stride) {
+            int tok = AASD_NONE;
+            if (i < ne) tok = (i < best_a) ? drafted : nt;
+            e[i] = tok;
+            if (i < ne && len + i < cap) a.seq.hist_ids[off + len + i] = tok;
+        }
+    }
+    if (a.seq.table_ids) {
+        // table rows of the emitted tokens: position len + i has row (first row) + len + i - 1
+        const int64_t row0 = (int64_t)a.seq.table_row_offsets[b] + len - 1;
+        const int K = a.seq.table_k;
+        for (int i = lane; i < ne; i += 32) {
+            if (len + i >= cap || len + i < 1) continue;
+            int n = 0, ids[kMaxK];
+#pragma unroll
+            for (int j = 0; j < kMaxK; ++j) ids[j] = AASD_NONE;
+            if (i < best_a) {
+                const int32_t* x = a.row_extra + ((int64_t)best * a.rows_per_cand + i) * kRowExtraInts;
+                n = __ldcg(x);
+#pragma unroll
+                for (int j = 0; j < kMaxK; ++j) ids[j] = __ldcg(x + 1 + j);
+            }
+            a.seq.table_n[row0 + i] = n;
+#pragma unroll
+            for (int j = 0; j < kMaxK; ++j)
+                if (j < K) a.seq.table_ids[(row0 + i) * K + j] = ids[j];
+        }
+    }
+    __syncwarp();
     if (lane == 0) {
-        c = candidate_of_row(a, job.n_rows, row, lo, hi);
-        if (!AASD_IN_RANGE(c >= 0 && c < a.n_cands && lo >= 0 && lo <= row && row < hi && hi <= job.n_rows, job.state)) c = 0, hi = lo = 0;
-        const unsigned int t = verify_row<DT>(a, job, row, merged, neg_refc, centered, d, xd, sampled,
-                                              &a.cand_tickets[c], tally);
-        last = (t == (unsigned int)(hi - lo) - 1u);
+        a.seq.best_cand[b] = best;
+        a.seq.n_emit[b] = ne;
+        a.seq.hist_len[b] = min(len + ne, cap);
+        if (len + ne > cap) tally.status |= AASD_STATUS_HIST_OVERFLOW;
+    }
+}
+
+// Everything a finished sequence of at most 32 rows needs, with row i of the sequence in lane
+// i: the prefix rule per candidate (Sec. 2.1), the longest passing candidate (Sec. 3.3), the
+// emission and the history update (Algorithm 1).  One trip to memory for the rows' records.
+__device__ inline void verify_complete_sequence(const VerifyArgs& a, int b, Tally& tally) {
+    const int lane = threadIdx.x & 31;
+    const int cps = a.seq.cands_per_seq, rpc = a.rows_per_cand, rps = a.seq.rows_per_seq;
+    const int64_t row0 = (int64_t)b * rps;
+    const u64 st = lane < rps ? __ldcg(a.row_state + row0 + lane) : 1ull;
+    const int dtok = lane < rps ? __ldg(a.draft_ids + row0 + lane) : AASD_NONE;
+    const int off = a.seq.hist_offsets[b];
+    const int cap = a.seq.hist_offsets[b + 1] - off;
+    const int len = a.seq.hist_len[b];
+    const unsigned int rejected = __ballot_sync(0xFFFFFFFFu, lane < rps && (st & 1ull) == 0);
+    const int own = (int)(unsigned int)(st >> 32);
+    const unsigned int seg_mask = rpc >= 32 ? 0xFFFFFFFFu : ((1u << rpc) - 1u);
+    int best = AASD_NONE, best_a = -1, nt = AASD_NONE;
+    for (int j = 0; j < cps; ++j) {
+        const unsigned int seg = (rejected >> (j * rpc)) & seg_mask;
+        const int n = seg ? __ffs(seg) - 1 : rpc;              // leading accepted rows
+        int next = __shfl_sync(0xFFFFFFFFu, own, j * rpc + (seg ? n : 0));
+        next = seg ? next : AASD_NONE;                          // the own token of the first row that does not pass
+        if (lane == 0) {
+            if (a.out.accept_len) a.out.accept_len[b * cps + j] = n;
+            if (a.out.next_token) a.out.next_token[b * cps + j] = next;
+        }
+        if (n > best_a) {      // ties go to the lower candidate
+            best_a = n;
+            best = b * cps + j;
+            nt = next;
+        }
+    }
+    if (best == AASD_NONE) best_a = 0;
+    const int first_row = (best - b * cps) * rpc;
+    emit_and_append(a, b, best, best_a, nt, off, cap, len,
+                    [&](int i) { return __shfl_sync(0xFFFFFFFFu, dtok, best == AASD_NONE ? 0 : first_row + i); }, tally);
+}
+
+__device__ inline void verify_complete_warp(const VerifyArgs& a, const RowJob& job, const PendingRow& pending, Tally& tally) {
+    const int lane = threadIdx.x & 31;
+    int c = pending.c, last = 0;
+    int64_t lo = pending.lo, hi = pending.hi;
+    if (__shfl_sync(0xFFFFFFFFu, pending.whole_sequence, 0)) {
+        int b = 0;
+        if (lane == 0) {
+            b = c / a.seq.cands_per_seq;
+            last = (pending.ticket == (unsigned int)a.seq.rows_per_seq - 1u);
+            if (last) a.seq.seq_tickets[b] = 0;
+        }
+        last = __shfl_sync(0xFFFFFFFFu, last, 0);
+        if (!last) return;
+        b = __shfl_sync(0xFFFFFFFFu, b, 0);
+        __threadfence();
+        verify_complete_sequence(a, b, tally);
+        return;
+    }
+    if (lane == 0) {
+        last = (pending.ticket == (unsigned int)(hi - lo) - 1u);
         if (last) a.cand_tickets[c] = 0;
     }
     last = __shfl_sync(0xFFFFFFFFu, last, 0);
@@ -569,56 +723,17 @@ __device__ void verify_finish_warp(const VerifyArgs& a, const RowJob& job, int64
         key = k > key ? k : key;
     }
     key = warp_max_u64(key);
-    int best = AASD_NONE, best_a = 0, ne = 0;
+    int best = AASD_NONE, best_a = 0;
     if (key != 0) {
         best = (int)(0xFFFFFFFFu - (unsigned int)key);
         best_a = (int)(key >> 32) - 1;
     }
-    const int stride = a.seq.emit_stride;
-    int32_t* e = a.seq.emit_ids + (int64_t)b * stride;
     const int off = a.seq.hist_offsets[b];
     const int cap = a.seq.hist_offsets[b + 1] - off;
     const int len = a.seq.hist_len[b];
-    int nt = AASD_NONE;
-    if (best != AASD_NONE) {
-        nt = __ldcg(a.out.next_token + best);
-        ne = min(best_a, stride);
-        if (nt != AASD_NONE && ne < stride) ne += 1;
-    }
-    for (int i = lane; i < stride; i += 32) {
-        int tok = AASD_NONE;
-        if (i < ne) tok = (i < best_a) ? a.draft_ids[(int64_t)best * a.rows_per_cand + i] : nt;
-        e[i] = tok;
-        if (i < ne && len + i < cap) a.seq.hist_ids[off + len + i] = tok;
-    }
-    if (a.seq.table_ids) {
-        // table rows of the emitted tokens: position len + i has row (first row) + len + i - 1
-        const int64_t row0 = (int64_t)a.seq.table_row_offsets[b] + len - 1;
-        const int K = a.seq.table_k;
-        for (int i = lane; i < ne; i += 32) {
-            if (len + i >= cap || len + i < 1) continue;
-            int n = 0, ids[kMaxK];
-#pragma unroll
-            for (int j = 0; j < kMaxK; ++j) ids[j] = AASD_NONE;
-            if (i < best_a) {
-                const int32_t* x = a.row_extra + ((int64_t)best * a.rows_per_cand + i) * kRowExtraInts;
-                n = __ldcg(x);
-#pragma unroll
-                for (int j = 0; j < kMaxK; ++j) ids[j] = __ldcg(x + 1 + j);
-            }
-            a.seq.table_n[row0 + i] = n;
-#pragma unroll
-            for (int j = 0; j < kMaxK; ++j)
-                if (j < K) a.seq.table_ids[(row0 + i) * K + j] = ids[j];
-        }
-    }
-    __syncwarp();
-    if (lane == 0) {
-        a.seq.best_cand[b] = best;
-        a.seq.n_emit[b] = ne;
-        a.seq.hist_len[b] = min(len + ne, cap);
-        if (len + ne > cap) tally.status |= AASD_STATUS_HIST_OVERFLOW;
-    }
+    const int nt = best != AASD_NONE ? __ldcg(a.out.next_token + best) : AASD_NONE;
+    emit_and_append(a, b, best, best_a, nt, off, cap, len,
+                    [&](int i) { return best != AASD_NONE ? a.draft_ids[(int64_t)best * a.rows_per_cand + i] : AASD_NONE; }, tally);
 }
 
 // One CTA (or `chunks` CTAs) per row with plain vector / scalar loads: the path for logits
@@ -662,7 +777,8 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(const VerifyArgs a) {
         sc.merged.ahead = n;
         __syncwarp();
     }
-    verify_finish_warp<DT>(a, job, row, sc.merged, neg_refc, centered, d, xd, sampled, tally);
+    const unsigned int flag = a.draft_flags ? a.draft_flags[row] : AASD_FLAG_CONDITIONAL;
+    verify_finish_warp<DT>(a, job, row, sc.merged, neg_refc, centered, d, xd, flag, sampled, tally);
     if (threadIdx.x == 0) tally.flush(job.state);
 }
 

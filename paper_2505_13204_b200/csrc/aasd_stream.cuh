@@ -142,6 +142,7 @@ struct ItemInfo {
     int chunk;        // which piece of the row
     int head;         // tokens of the row in front of its first 16-byte boundary (0 for aligned rows)
     int nvec;         // whole 16-byte vectors of the row from that boundary on
+    int aux;          // a per-row word the epilogue wants fetched ahead of time (E::prefetch)
 };
 constexpr int kNoItem = -1;
 constexpr int kMaxCluster = 8;   // portable cluster size
@@ -551,6 +552,13 @@ struct FinishedRow {
 // Epilogue interface (static functions of a policy type E):
 //   E::finish<ND>(args, job, row, rowp, FinishedRow&, ItemInfo&, races, tail_group, Tally&)
 //   - entered by the whole finisher warp
+//   E::State, E::drain(args, job, State&, Tally&)
+//   - what an epilogue carries from one row to the next (verification looks at a row's ticket
+//     one row late); drain is called once when the finisher warp has seen its last item
+//   E::prefetch(args, row) -> int
+//   - a per-row input of the epilogue, loaded by the producer together with the row's reference
+//     and handed over in ItemInfo::aux, so that the finisher's serial path has no trip to
+//     memory for it
 //   ND: keyed draws per row the kernel prepares (0: no sampling)
 //   TK: count the tokens ahead of the hinted token (top-k verification)
 //   FIN: the logits are expected to hold no -inf: the clamp that makes masked tokens harmless
@@ -897,6 +905,9 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
             float r = -CUDART_INF_F;
             if (lane < 4 && lane < rj.vocab) r = Elt<DT>::load(rowp, lane);
             if (lane == 4 && hint_ok) r = Elt<DT>::load(rowp, hint);
+            int aux = 0;
+            if (lane == 5) aux = E::prefetch(args, row);
+            aux = __shfl_sync(0xFFFFFFFFu, aux, 5);
             const float hint_logit = __shfl_sync(0xFFFFFFFFu, r, 4);
 #pragma unroll
             for (int o = 4; o > 0; o >>= 1) r = fmaxf(r, __shfl_xor_sync(0xFFFFFFFFu, r, o));
@@ -911,6 +922,7 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
                 info.chunk = chunk;
                 info.head = head;
                 info.nvec = nvec;
+                info.aux = aux;
                 if (first_bytes) mbar_arrive_expect_tx(&sh.full[first_stage], first_bytes);
                 ++it;
                 for (int t = tb + 1; t < te; ++t, ++it) {
@@ -954,6 +966,8 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
     // the items go round the NF finisher warps
     Tally tally;   // lane 0's running counters, flushed when the warp leaves
     tally.clear();
+    typename E::State estate;
+    E::init(estate);
     for (unsigned int seq = (unsigned int)(warp - kConsumerWarps - 1);; seq += NF) {
         const int p = seq % kSlots;
         if (!mbar_wait(&sh.done[p], (seq / kSlots) & 1u, abort_flag, job.wait_limit)) {
@@ -1283,8 +1297,9 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
         // ids beyond the last complete group of the vector part were not raced (sampling
         // launches take aligned rows only: head == 0)
         const int tail_group = (ND > 0 && job.full_groups * kGroup < rj.vocab) ? job.full_groups : -1;
-        E::template finish<ND>(args, rj, row, rowp, fr, info, races, tail_group, tally);
+        E::template finish<ND>(args, rj, row, rowp, fr, info, races, tail_group, estate, tally);
     }
+    E::drain(args, rj, estate, tally);
     if (lane == 0) tally.flush(rj.state);
     if (job.cluster_pieces) cluster_exit_sync();
 }
@@ -1293,25 +1308,43 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
 template <int DT>
 struct VerifyEpilogue {
     using Args = VerifyArgs;
+    using State = PendingRow;
+    static __device__ __forceinline__ void init(State& st) { st.valid = 0; }
     template <int ND>
     static __device__ void finish(const VerifyArgs& a, const RowJob& job, int64_t row, const char* rowp,
                                   const FinishedRow& fr, const ItemInfo& info, const RaceSummary* races, int tail_group,
-                                  Tally& tally) {
+                                  State& previous, Tally& tally) {
         int sampled = AASD_NONE;
         if (ND > 0 && !partial_bad(fr.merged))
             sampled = warp_sample_decide<DT>(rowp, job.vocab, (unsigned int)row, 0, a.smp, races[0], tail_group,
                                              fr.centered, tally.recheck, tally.exhaustive);
-        verify_finish_warp<DT>(a, job, row, fr.merged, fr.neg_refc, fr.centered, info.hint, info.hint_logit, sampled,
-                               tally);
+        // this row's evaluation and ticket first, then the previous row's ticket, which has had
+        // a whole row's time to come back
+        PendingRow mine;
+        verify_row_warp<DT>(a, job, row, fr.merged, fr.neg_refc, fr.centered, info.hint, info.hint_logit,
+                            (unsigned int)info.aux, sampled, mine, tally);
+        if (previous.valid) verify_complete_warp(a, job, previous, tally);
+        previous = mine;
+    }
+    static __device__ void drain(const VerifyArgs& a, const RowJob& job, State& previous, Tally& tally) {
+        if (previous.valid) verify_complete_warp(a, job, previous, tally);
+        previous.valid = 0;
+    }
+    // the row's flag byte
+    static __device__ __forceinline__ int prefetch(const VerifyArgs& a, int64_t row) {
+        return a.draft_flags ? (int)__ldg(a.draft_flags + row) : (int)AASD_FLAG_CONDITIONAL;
     }
 };
 template <int DT>
 struct AlignEpilogue {
     using Args = AlignArgs;
+    struct State {};
+    static __device__ __forceinline__ void init(State&) {}
+    static __device__ __forceinline__ void drain(const AlignArgs&, const RowJob&, State&, Tally&) {}
     template <int ND>
     static __device__ void finish(const AlignArgs& a, const RowJob& job, int64_t row, const char* rowp,
                                   const FinishedRow& fr, const ItemInfo& info, const RaceSummary* races, int tail_group,
-                                  Tally& tally) {
+                                  State&, Tally& tally) {
         // next_ids holds validated tokens only, so the hint is the row's next token
         int draws[kMaxK];
 #pragma unroll
@@ -1326,6 +1359,7 @@ struct AlignEpilogue {
         align_finish_warp<DT>(a, job, row, rowp, fr.merged, fr.neg_refc, fr.centered, info.hint, info.hint_logit, draws,
                               tally);
     }
+    static __device__ __forceinline__ int prefetch(const AlignArgs&, int64_t) { return 0; }
 };
 
 }  // namespace aasd

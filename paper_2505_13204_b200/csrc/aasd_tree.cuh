@@ -346,10 +346,13 @@ __device__ void tree_finish_warp(const TreeArgs& a, const RowJob& job, int64_t r
 template <int DT>
 struct TreeEpilogue {
     using Args = TreeArgs;
+    struct State {};
+    static __device__ __forceinline__ void init(State&) {}
+    static __device__ __forceinline__ void drain(const TreeArgs&, const RowJob&, State&, Tally&) {}
     template <int ND>
     static __device__ void finish(const TreeArgs& a, const RowJob& job, int64_t row, const char* rowp,
                                   const FinishedRow& fr, const ItemInfo& info, const RaceSummary* races, int tail_group,
-                                  Tally& tally) {
+                                  State&, Tally& tally) {
         int sampled = AASD_NONE;
         if (ND > 0 && !partial_bad(fr.merged))
             sampled = warp_sample_decide<DT>(rowp, job.vocab, (unsigned int)row, 0, a.smp, races[0], tail_group,
@@ -361,6 +364,7 @@ struct TreeEpilogue {
         tree_finish_warp<DT>(a, job, row, fr.merged, fr.neg_refc, fr.centered, sampled,
                              counted ? (int)fr.merged.ahead : -1, tally);
     }
+    static __device__ __forceinline__ int prefetch(const TreeArgs&, int64_t) { return 0; }
 };
 
 // Plain-load kernel for layouts whose rows are not 16-byte aligned.
