@@ -202,6 +202,7 @@ SampleJob make_sample_job(uint64_t seed, uint32_t step, bool align, float inv_te
     s.dom_group = align ? kDomAlignGroup : kDomVerifyGroup;
     s.dom_elem = align ? kDomAlignElem : kDomVerifyElem;
     s.inv_t = inv_temperature;
+    fill_round_keys(s);
     return s;
 }
 

@@ -38,16 +38,28 @@ enum SampleDomain : unsigned int {
 };
 
 // What the kernels need to know to sample.
+constexpr unsigned int kPhiloxW0 = 0x9E3779B9u, kPhiloxW1 = 0xBB67AE85u;   // key increments per round
+
 struct SampleJob {
     unsigned int key0, key1;   // seed
     unsigned int step;         // decoding step / stream tag
     unsigned int dom_group, dom_elem;
     float inv_t;               // inv_temperature
+    // the generator's key schedule, key + round * increment, laid out by the host so that the
+    // streaming pass reads its round keys as launch constants instead of adding them up
+    unsigned int rk0[10], rk1[10];
 };
+
+inline void fill_round_keys(SampleJob& s) {
+    for (int r = 0; r < 10; ++r) {
+        s.rk0[r] = s.key0 + (unsigned int)r * kPhiloxW0;
+        s.rk1[r] = s.key1 + (unsigned int)r * kPhiloxW1;
+    }
+}
 
 __device__ __forceinline__ void philox4x32_10(unsigned int c0, unsigned int c1, unsigned int c2, unsigned int c3,
                                               unsigned int k0, unsigned int k1, unsigned int (&out)[4]) {
-    constexpr unsigned int M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+    constexpr unsigned int M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = kPhiloxW0, W1 = kPhiloxW1;
 #pragma unroll
     for (int round = 0; round < 10; ++round) {
         const u64 p0 = (u64)M0 * c0, p1 = (u64)M1 * c2;   // one wide multiply each
@@ -60,6 +72,27 @@ __device__ __forceinline__ void philox4x32_10(unsigned int c0, unsigned int c1, 
         c3 = lo0;
         k0 += W0;
         k1 += W1;
+    }
+    out[0] = c0;
+    out[1] = c1;
+    out[2] = c2;
+    out[3] = c3;
+}
+
+// The same generator with the round keys taken from the job (see SampleJob::rk0).
+__device__ __forceinline__ void philox4x32_10_scheduled(unsigned int c0, unsigned int c1, unsigned int c2, unsigned int c3,
+                                                        const SampleJob& sj, unsigned int (&out)[4]) {
+    constexpr unsigned int M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;
+#pragma unroll
+    for (int round = 0; round < 10; ++round) {
+        const u64 p0 = (u64)M0 * c0, p1 = (u64)M1 * c2;
+        const unsigned int hi0 = (unsigned int)(p0 >> 32), lo0 = (unsigned int)p0;
+        const unsigned int hi1 = (unsigned int)(p1 >> 32), lo1 = (unsigned int)p1;
+        const unsigned int n0 = hi1 ^ c1 ^ sj.rk0[round], n2 = hi0 ^ c3 ^ sj.rk1[round];
+        c0 = n0;
+        c1 = lo1;
+        c2 = n2;
+        c3 = lo0;
     }
     out[0] = c0;
     out[1] = c1;
@@ -123,7 +156,7 @@ struct GroupRace {
     // a caller can have it computed while the logits are still on their way through the pipes
     static __device__ __forceinline__ void inverse_variates(int g, unsigned int row, const SampleJob& sj, float (&inv_e)[ND]) {
         unsigned int w[4];
-        philox4x32_10((unsigned int)g, row, sj.step, sj.dom_group, sj.key0, sj.key1, w);
+        philox4x32_10_scheduled((unsigned int)g, row, sj.step, sj.dom_group, sj, w);
 #pragma unroll
         for (int j = 0; j < ND; ++j) inv_e[j] = rcp_approx(exponential_fast(w[j]));
     }
