@@ -93,6 +93,13 @@ __device__ __forceinline__ double warp_sum_f64(double v) {
     return v;
 }
 
+// Sum of the values held by lanes 0..7 (the other lanes' values are ignored), in every lane.
+__device__ __forceinline__ double octet_sum_f64(double v) {
+#pragma unroll
+    for (int o = 4; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return __shfl_sync(0xFFFFFFFFu, v, 0);
+}
+
 __device__ __forceinline__ long long warp_sum_i64(long long v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);

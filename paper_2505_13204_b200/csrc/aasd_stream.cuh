@@ -189,21 +189,23 @@ struct StreamJob {
 };
 constexpr int kRaceSlots = 1024;  // cut-row pieces a sampling launch may have
 
-// Work item -> (row, piece); pieces of a row are balanced ranges of its tiles.
+// Work item -> (row, piece); pieces of a row are balanced ranges of its tiles.  (Item, row and
+// tile counts fit 32 bits - the host refuses launches beyond that - and 32-bit divisions are
+// several times cheaper than 64-bit ones on a path every item walks.)
 __device__ __forceinline__ void decode_item(const StreamJob& job, long long item, int& row, int& chunk) {
     if (item < job.whole_rows) {
         row = (int)item;
         chunk = 0;
     } else {
-        const long long j = item - job.whole_rows;
-        row = job.whole_rows + (int)(j / job.tail_chunks);
-        chunk = (int)(j % job.tail_chunks);
+        const unsigned int j = (unsigned int)(item - job.whole_rows), c = (unsigned int)job.tail_chunks;
+        row = job.whole_rows + (int)(j / c);
+        chunk = (int)(j % c);
     }
 }
 __device__ __forceinline__ int chunks_of(const StreamJob& job, int row) {
     return row < job.whole_rows ? 1 : job.tail_chunks;
 }
-__device__ __forceinline__ int tiles_of(int nvec) { return (int)(((long long)nvec * 16 + kTileBytes - 1) / kTileBytes); }
+__device__ __forceinline__ int tiles_of(int nvec) { return (int)(((unsigned int)nvec + (kTileBytes / 16 - 1)) / (kTileBytes / 16)); }
 // nvec: the row's own vector count (rows that do not start on a 16-byte boundary differ by one)
 __device__ __forceinline__ void tile_range(const StreamJob& job, int row, int chunk, int nvec, int& tb, int& te) {
     const int tiles = tiles_of(nvec);
@@ -211,8 +213,10 @@ __device__ __forceinline__ void tile_range(const StreamJob& job, int row, int ch
         tb = 0;
         te = tiles;
     } else {
-        tb = (int)(((long long)chunk * tiles) / job.tail_chunks);
-        te = (int)(((long long)(chunk + 1) * tiles) / job.tail_chunks);
+        // chunk < tail_chunks <= 32 and tiles < 2^20: the products stay far inside 32 bits
+        const unsigned int c = (unsigned int)job.tail_chunks;
+        tb = (int)(((unsigned int)chunk * (unsigned int)tiles) / c);
+        te = (int)(((unsigned int)(chunk + 1) * (unsigned int)tiles) / c);
     }
 }
 // Where a row's vectors begin: rows are streamed from their first 16-byte boundary, the few
@@ -856,10 +860,12 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
                         for (int j = 0; j < NF; ++j) sh.ring[(seq + j) % kRing].row = kNoItem;
                         mbar_arrive(&sh.full[s]);
                         // the last CTA to get here leaves the counters ready for the next launch
-                        __threadfence();
-                        if (atomicAdd(job.sched + 1, 1u) == gridDim.x - 1) {
-                            job.sched[0] = 0;
-                            job.sched[1] = 0;
+                        if (!job.cluster_pieces) {
+                            __threadfence();
+                            if (atomicAdd(job.sched + 1, 1u) == gridDim.x - 1) {
+                                job.sched[0] = 0;
+                                job.sched[1] = 0;
+                            }
                         }
                     } else {
                         alive = false;
@@ -868,7 +874,6 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
                 alive = __shfl_sync(0xFFFFFFFFu, alive ? 1 : 0, 0) != 0;
                 break;
             }
-            if (lane == 0) next = (long long)gridDim.x + (long long)atomicAdd(job.sched, 1u);
             int row, chunk;
             decode_item(job, item, row, chunk);
             const char* rowp = row_pointer<DT>(rj, row);
@@ -898,6 +903,9 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
                     bulk_copy_g2s(tiles + (size_t)first_stage * kTileBytes, vbase + off, first_bytes, &sh.full[first_stage]);
                     armed |= 1u << first_stage;
                 }
+                // the next item: claimed one ahead, behind this item's first copy (launches of one
+                // item per CTA have nothing to claim)
+                next = job.cluster_pieces ? job.n_items : (long long)gridDim.x + (long long)atomicAdd(job.sched, 1u);
             }
             // reference of the row: its hinted logit and its first entries
             const int hint = __ldg(job.hint_ids + row);
@@ -1018,8 +1026,9 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&sh.freeb[p]);
-        S = warp_sum_f64(S);
-        A = warp_sum_f64(A);
+        static_assert(kConsumerWarps == 8, "the eight warp partials sit in lanes 0-7");
+        S = octet_sum_f64(S);
+        A = octet_sum_f64(A);
         if (TK) n_ahead = warp_sum_i64(n_ahead);
         u64 mk[K];   // merged vector keys, identical in every lane
         // One item per CTA whose tiles all fit the ring (the small launches whose rows are cut
@@ -1126,8 +1135,9 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
 #pragma unroll
                 for (int j = 0; j < K; ++j) key_insert<K>(vk, q.key[j]);
             }
-            S = warp_sum_f64(S);
-            A = warp_sum_f64(A);
+            static_assert(kMaxCluster <= 8, "a cluster's pieces sit in lanes 0-7");
+            S = octet_sum_f64(S);
+            A = octet_sum_f64(A);
             if (TK) n_ahead = warp_sum_i64(n_ahead);
 #pragma unroll
             for (int r = 0; r < K; ++r) {
@@ -1243,8 +1253,10 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
                 if (x > -CUDART_INF_F) key_insert<K>(ek, make_key(x, i));
             }
         }
-        S += warp_sum_f64((double)ts);
-        A += warp_sum_f64((double)ta);
+        if (head > 0 || nvec * kVec < rj.vocab) {     // (no token outside the vectors: nothing to add)
+            S += warp_sum_f64((double)ts);
+            A += warp_sum_f64((double)ta);
+        }
         FinishedRow fr;
 #pragma unroll
         for (int r = 0; r < kMaxK; ++r) fr.merged.key[r] = 0;
