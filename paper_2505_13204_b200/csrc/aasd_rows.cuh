@@ -328,6 +328,49 @@ __device__ inline RowFinal finish_row(const RowPartial& p, float c1, float neg_r
     return f;
 }
 
+// The same by a whole warp, with the probabilities of up to 31 tokens of the row alongside:
+// lane l < 31 hands in the raw logit of a token (`my_x`; anything where it has none) and
+// gets the token's probability back in `my_prob`.  All the fp64 work of a row - the logarithm
+// of Eq. 5 and the exponentials of the probabilities - is one exponential per lane, evaluated
+// by all lanes at once instead of one after the other by one lane: lane 31 evaluates
+// 2^-y0 for y0 = lg2.approx(S), which turns log2(S) = y0 + log2(S * 2^-y0) into a three-term
+// series in S * 2^-y0 - 1 (|.| < 2^-21, truncation below 1e-27); the divisions by S are
+// multiplications by one reciprocal.  Results differ from finish_row's by a few fp64 ulps.
+__device__ inline RowFinal finish_row_warp(const RowPartial& p, float c1, float neg_refc, bool centered, float my_x,
+                                           double& my_prob) {
+    RowFinal f;
+    f.c1 = (double)c1;
+    f.neg_refc = (double)neg_refc;
+    f.centered = centered;
+    f.m = key_value(p.key[0]);
+    f.top1 = key_id(p.key[0]);
+    f.S = p.S;
+    f.bad = partial_bad(p);     // the same in every lane: p is
+    my_prob = 0.0;
+    if (f.bad) {
+        f.top1 = AASD_NONE;
+        f.H = 0.0;
+        f.pmax = 0.0;
+        f.S = 1.0;
+        return f;
+    }
+    const int lane = threadIdx.x & 31;
+    float y0;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y0) : "f"((float)p.S));
+    if (!(fabsf(y0) <= 1.0e30f)) y0 = 0.f;      // S outside float's range: the series would not hold ...
+    const double t = lane == 31 ? -(double)y0
+                                : (centered ? ((double)my_x + f.neg_refc) * f.c1 : (double)my_x * f.c1 + f.neg_refc);
+    const double e = exp2(t);
+    const double inv_s = 1.0 / p.S;
+    my_prob = e * inv_s;
+    const double u = __shfl_sync(0xFFFFFFFFu, e, 31) * p.S - 1.0;
+    constexpr double kInvLn2 = 1.4426950408889634;
+    double log2_s = (double)y0 + u * (kInvLn2 + u * (-0.5 * kInvLn2 + u * (kInvLn2 / 3.0)));
+    if (!(fabs(u) <= 1.0e-3)) log2_s = log2(p.S);   // ... so take the library's logarithm there
+    f.H = kLn2 * (log2_s - p.A * inv_s);
+    return f;
+}
+
 // ---- conditional verification -----------------------------------------------------------------
 
 // Optional tail of a verification launch: once the last candidate of a sequence is done,
@@ -416,12 +459,12 @@ struct Tally {
 // nobody inside the launch reads, are under way while the ticket travels.  Returns the
 // ticket's value.
 // flag: the row's draft-token flag byte (AASD_FLAG_CONDITIONAL when the call has no flags).
+// f: the row's scalars (finish_row_warp), pd_in: the draft token's probability from the same call.
 template <int DT>
 __device__ unsigned int verify_row(const VerifyArgs& a, const RowJob& job, int64_t row, const RowPartial& merged,
-                                   float neg_refc, bool centered, int d, float xd, unsigned int flag, int sampled,
+                                   const RowFinal& f, double pd_in, int d, float xd, unsigned int flag, int sampled,
                                    unsigned int* ticket, Tally& tally) {
     const bool d_ok = d >= 0 && d < job.vocab;
-    const RowFinal f = finish_row(merged, job.c1, neg_refc, centered);
     if (!AASD_IN_RANGE(row >= 0 && row < job.n_rows && (f.bad || (f.top1 >= 0 && f.top1 < job.vocab)), job.state)) return 0xFFFFFFFFu;
     const double lin = (double)a.alpha * f.H + (double)a.beta;
     const double thr = f.bad ? 0.0 : fmin(lin, f.pmax);
@@ -431,7 +474,7 @@ __device__ unsigned int verify_row(const VerifyArgs& a, const RowJob& job, int64
     if (f.bad) tally.status |= AASD_STATUS_BAD_ROW;
     if (!d_ok && d != AASD_NONE) tally.status |= AASD_STATUS_ID_RANGE;
     if (d_ok && !f.bad) {
-        pd = f.prob(xd);
+        pd = pd_in;
         if (a.mode == AASD_VERIFY_CONDITIONAL && (flag & AASD_FLAG_CONDITIONAL)) {
             const bool at_max = (xd == f.m);
             acc = at_max || (pd >= lin);
@@ -536,13 +579,20 @@ __device__ void verify_row_warp(const VerifyArgs& a, const RowJob& job, int64_t 
     pending.lo = pending.hi = 0;
     pending.ticket = 0;
     pending.whole_sequence = 0;
-    if ((threadIdx.x & 31) == 0) {
+    // the row's scalars by the whole warp: lane 0 asks for the best token's probability
+    // (Delta of Eq. 6), lane 1 for the draft token's (Eq. 4)
+    const int lane_id = threadIdx.x & 31;
+    double my_prob;
+    RowFinal f = finish_row_warp(merged, job.c1, neg_refc, centered, lane_id == 1 ? xd : key_value(merged.key[0]), my_prob);
+    f.pmax = __shfl_sync(0xFFFFFFFFu, my_prob, 0);
+    const double pd = __shfl_sync(0xFFFFFFFFu, my_prob, 1);
+    if (lane_id == 0) {
         int64_t lo = 0, hi = 0;
         int c = candidate_of_row(a, job.n_rows, row, lo, hi);
         if (!AASD_IN_RANGE(c >= 0 && c < a.n_cands && lo >= 0 && lo <= row && row < hi && hi <= job.n_rows, job.state)) c = 0, hi = lo = 0;
         pending.whole_sequence = sequence_tickets(a) ? 1 : 0;
         unsigned int* ticket = pending.whole_sequence ? &a.seq.seq_tickets[c / a.seq.cands_per_seq] : &a.cand_tickets[c];
-        pending.ticket = verify_row<DT>(a, job, row, merged, neg_refc, centered, d, xd, flag, sampled, ticket, tally);
+        pending.ticket = verify_row<DT>(a, job, row, merged, f, pd, d, xd, flag, sampled, ticket, tally);
         pending.c = c;
         pending.lo = lo;
         pending.hi = hi;
@@ -834,13 +884,30 @@ __device__ inline bool align_wants_draws(const AlignArgs& a, const RowPartial& m
     return !(next != AASD_NONE && next == key_id(merged.key[0]));
 }
 
-// Row epilogue of alignment sampling (Sec. 2.3 alignment test, Fig. 2 extras), one thread.
+// Row epilogue of alignment sampling (Sec. 2.3 alignment test, Fig. 2 extras): entered by a whole
+// warp for the row's fp64 scalars, finished by lane 0.
 // next is the prompt's next token of the row (validated, or NONE), xn its raw logit.  In
 // GUMBEL mode draws[j] / draw_logits[j] are the row's keyed draws (NONE where not drawn).
 __device__ inline void align_row(const AlignArgs& a, const RowJob& job, int64_t row, const RowPartial& merged,
                                  float neg_refc, bool centered, int next, float xn_in, const int* draws,
                                  const float* draw_logits, Tally& tally) {
-    const RowFinal f = finish_row(merged, job.c1, neg_refc, centered);
+    // the row's scalars and every probability the row may report, by the whole warp: lane 0 the
+    // best token's, lane 1 the next token's, lanes 2 .. 2+K-1 the listed tokens' (TOPK) or the
+    // draws' (GUMBEL)
+    const int lane_id = threadIdx.x & 31;
+    float my_x = key_value(merged.key[0]);
+    if (lane_id == 1) my_x = xn_in;
+#pragma unroll
+    for (int j = 0; j < kMaxK; ++j)
+        if (lane_id == 2 + j) my_x = a.mode == AASD_ALIGN_GUMBEL ? draw_logits[j] : key_value(merged.key[j]);
+    double my_prob;
+    RowFinal f = finish_row_warp(merged, job.c1, neg_refc, centered, my_x, my_prob);
+    f.pmax = __shfl_sync(0xFFFFFFFFu, my_prob, 0);
+    const double p_next = __shfl_sync(0xFFFFFFFFu, my_prob, 1);
+    double p_listed[kMaxK];
+#pragma unroll
+    for (int j = 0; j < kMaxK; ++j) p_listed[j] = __shfl_sync(0xFFFFFFFFu, my_prob, 2 + j);
+    if (lane_id != 0) return;
     const int KE = a.k_extra;
     int ids[kMaxK];
     float ps[kMaxK];
@@ -855,7 +922,7 @@ __device__ inline void align_row(const AlignArgs& a, const RowJob& job, int64_t 
         float xn = 0.f;
         if (next != AASD_NONE) {
             xn = xn_in;
-            pn = f.prob(xn);
+            pn = p_next;
             aligned = (next == f.top1);
         }
         if (a.mode == AASD_ALIGN_GUMBEL) {
@@ -867,7 +934,7 @@ __device__ inline void align_row(const AlignArgs& a, const RowJob& job, int64_t 
                 for (int q = 0; q < n; ++q) dup |= (ids[q] == tok);
                 if (dup) continue;
                 ids[n] = tok;
-                ps[n] = (float)f.prob(draw_logits[j]);
+                ps[n] = (float)p_listed[j];
                 ++n;
             }
         } else {
@@ -879,7 +946,7 @@ __device__ inline void align_row(const AlignArgs& a, const RowJob& job, int64_t 
                 const int id = key_id(k);
                 if (next == AASD_NONE || xv > xn || (xv == xn && id < next)) {
                     ids[n] = id;
-                    ps[n] = (float)f.prob(xv);
+                    ps[n] = (float)p_listed[j];
                     ++n;
                 }
             }
@@ -907,7 +974,6 @@ template <int DT>
 __device__ void align_finish_warp(const AlignArgs& a, const RowJob& job, int64_t row, const char* rowp,
                                   const RowPartial& merged, float neg_refc, bool centered, int next, float xn,
                                   const int (&draws)[kMaxK], Tally& tally) {
-    if ((threadIdx.x & 31) != 0) return;
     float dx[kMaxK];
     for (int j = 0; j < kMaxK; ++j)
         dx[j] = (a.mode == AASD_ALIGN_GUMBEL && j < a.k_extra && draws[j] >= 0) ? Elt<DT>::load(rowp, draws[j]) : 0.f;

@@ -189,8 +189,10 @@ __device__ void tree_finish_warp(const TreeArgs& a, const RowJob& job, int64_t r
     const int lane = threadIdx.x & 31;
     int t = 0, last = 0;
     int64_t lo = 0, hi = 0;
+    double my_prob;
+    RowFinal f = finish_row_warp(merged, job.c1, neg_refc, centered, key_value(merged.key[0]), my_prob);
+    f.pmax = __shfl_sync(0xFFFFFFFFu, my_prob, 0);
     if (lane == 0) {
-        const RowFinal f = finish_row(merged, job.c1, neg_refc, centered);
         const double lin = (double)a.alpha * f.H + (double)a.beta;
         TreeRowStat st;
         st.S = f.S;
