@@ -719,7 +719,10 @@ __device__ inline void verify_complete_warp(const VerifyArgs& a, const RowJob& j
         last = __shfl_sync(0xFFFFFFFFu, last, 0);
         if (!last) return;
         b = __shfl_sync(0xFFFFFFFFu, b, 0);
-        __threadfence();
+        // lane 0's ticket acquired what the other rows' warps released; the warp barrier hands
+        // that on to the other lanes, whose loads go to L2 (no fence, which would also wait for
+        // this warp's own stores)
+        __syncwarp();
         verify_complete_sequence(a, b, tally);
         return;
     }
@@ -732,7 +735,7 @@ __device__ inline void verify_complete_warp(const VerifyArgs& a, const RowJob& j
     c = __shfl_sync(0xFFFFFFFFu, c, 0);
     lo = __shfl_sync(0xFFFFFFFFu, lo, 0);
     hi = __shfl_sync(0xFFFFFFFFu, hi, 0);
-    __threadfence();
+    __syncwarp();   // (as above: lane 0's ticket acquired the other rows' records)
     int64_t n = hi - lo;   // leading accepted rows
     int next = AASD_NONE;  // the own token of the first row that does not pass
     for (int64_t base = lo; base < hi; base += 32) {
@@ -763,7 +766,7 @@ __device__ inline void verify_complete_warp(const VerifyArgs& a, const RowJob& j
         }
         last = __shfl_sync(0xFFFFFFFFu, last, 0);
         if (!last) return;
-        __threadfence();
+        __syncwarp();
     }
     // longest accepted prefix, ties to the lowest candidate: key = (length + 1, ~candidate)
     u64 key = 0;
