@@ -597,6 +597,18 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
         mbar_init(&sh.cluster_bar, job.cluster_pieces ? (unsigned int)job.tail_chunks - 1u : 1u);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    // Where the producer's first item lies: launch constants only, so worked out on this side
+    // of the wait for the preceding kernel (and again, for the next item, at the end of each
+    // of the producer's iterations).
+    int g_row = 0, g_chunk = 0, g_head = 0, g_nvec = 0, g_tb = 0, g_te = 0;
+    const char* g_rowp = nullptr;
+    auto locate = [&](long long item) {
+        decode_item(job, item, g_row, g_chunk);
+        g_rowp = row_pointer<DT>(rj, g_row);
+        row_vectors<DT>(g_rowp, rj.vocab, g_head, g_nvec);
+        tile_range(job, g_row, g_chunk, g_nvec, g_tb, g_te);
+    };
+    if (warp == kConsumerWarps) locate(blockIdx.x);
     // nobody may signal a barrier of another CTA before that CTA has set it up
     if (job.cluster_pieces) cluster_sync_all();
     pdl_launch_dependents();
@@ -874,13 +886,9 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
                 alive = __shfl_sync(0xFFFFFFFFu, alive ? 1 : 0, 0) != 0;
                 break;
             }
-            int row, chunk;
-            decode_item(job, item, row, chunk);
-            const char* rowp = row_pointer<DT>(rj, row);
-            int head, nvec, tb, te;
-            row_vectors<DT>(rowp, rj.vocab, head, nvec);
+            const int row = g_row, chunk = g_chunk, head = g_head, nvec = g_nvec, tb = g_tb, te = g_te;
+            const char* rowp = g_rowp;
             const char* vbase = rowp + (size_t)head * Elt<DT>::kSize;
-            tile_range(job, row, chunk, nvec, tb, te);
             // The item's first tile is sent off before anything else: the loads that give the
             // row's reference (two dependent trips to memory) then run while the copy is under
             // way.  The tile is announced (the producer's arrival on the stage's barrier, which
@@ -953,6 +961,7 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
             }
             alive = __shfl_sync(0xFFFFFFFFu, alive ? 1 : 0, 0) != 0;
             next = __shfl_sync(0xFFFFFFFFu, next, 0);
+            if (next < job.n_items) locate(next);
         }
         if (!alive && lane == 0) {
             // give the copies still in flight a bounded time to land before the CTA leaves
