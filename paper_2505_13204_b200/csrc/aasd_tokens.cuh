@@ -33,13 +33,15 @@ __device__ __forceinline__ int place_of(int code) { return code <= -2 ? -2 - cod
 // The places are found in two sweeps: the best length (block-wide maximum), then one bit per
 // place that reaches it, written by warp ballots into a bit field in shared memory (a window
 // of 4096 places at a time, from the top down, until enough places are found) from which one
-// warp reads the places off in descending order.
+// warp reads the places off in descending order.  A history of more than one window whose
+// lengths are all kept in shared memory takes one pass instead: a word of hit bits per thread,
+// a block-wide count from the top down, and every thread writes its own places.
 __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs a) {
     __shared__ int s_rec[AASD_MAX_NGRAM];
     __shared__ int s_pos[kMaxCands];        // places of the mains (pool places encoded)
     __shared__ int s_len[kMaxCands];        // and how many tokens follow them
     __shared__ unsigned int s_hits[kHitWords];
-    __shared__ unsigned char s_m[kMatchBytes];   // match length of every place of the history (short histories)
+    __shared__ __align__(16) unsigned char s_m[kMatchBytes];   // match length of every place of the history (short histories)
     __shared__ int s_count;
     __shared__ int s_kstar;
     __shared__ unsigned char s_next[kMaxCands * kExtScan];
@@ -62,10 +64,21 @@ __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs a)
     const int pool_len = pool != nullptr ? a.in.pool_len : 0;
     const bool have_pool_align = pool_len > 0 && a.in.pool_align_ids != nullptr && a.in.pool_align_n != nullptr && K > 0;
 
+    // The tokens in front of the first places each thread looks at do not depend on the key:
+    // they are asked for together with it, so that both cross the memory system at once.
+    constexpr int kBatch = 8;
+    int front[kBatch];
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u) {
+        const int p = 1 + tid + u * kDraftThreads;
+        front[u] = p < len ? h[p - 1] : AASD_NONE;
+    }
     int rl;
     if (a.in.recent_ids) {
+        // (slot tid of the key is read whether it counts or not: one trip instead of two)
+        const int slot = tid < n ? a.in.recent_ids[(int64_t)b * n + tid] : AASD_NONE;
         rl = max(0, min(n, a.in.recent_len[b]));
-        if (tid < rl) s_rec[tid] = a.in.recent_ids[(int64_t)b * n + tid];
+        if (tid < rl) s_rec[tid] = slot;
     } else {
         rl = min(n, len);
         if (tid < rl) s_rec[tid] = h[len - rl + tid];
@@ -73,6 +86,7 @@ __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs a)
     if (tid == 0) {
         s_count = 0;
         s_kstar = 0;
+        s_m[0] = 0;   // no place 0: the bit field below reads whole words
     }
     __syncthreads();
 
@@ -124,14 +138,14 @@ __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs a)
         // the table, one of that position's extras): the tokens of eight places are fetched
         // together, so that their trips to memory overlap, and the full comparison runs for
         // the few places that pass this test.
-        constexpr int kBatch = 8;
         const int want_last = rl > 0 ? s_rec[rl - 1] : AASD_NONE;
         for (int base = 1 + tid; base < len; base += kBatch * kDraftThreads) {
-            int front[kBatch];
+            if (base != 1 + tid) {
 #pragma unroll
-            for (int u = 0; u < kBatch; ++u) {
-                const int p = base + u * kDraftThreads;
-                front[u] = p < len ? h[p - 1] : AASD_NONE;
+                for (int u = 0; u < kBatch; ++u) {
+                    const int p = base + u * kDraftThreads;
+                    front[u] = p < len ? h[p - 1] : AASD_NONE;
+                }
             }
 #pragma unroll
             for (int u = 0; u < kBatch; ++u) {
@@ -153,6 +167,53 @@ __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs a)
     // windows of 32 * kHitWords places from the top down
     if (kstar > 0) {
         for (int src = 0; src < 2; ++src) {
+            if (src == 0 && cached && len > 32 * kHitWords) {
+                // (a history of a single window measured no slower by the windows below)
+                // Every place's length is in shared memory: thread t turns places 32 t .. 32 t + 31
+                // into a word of hit bits (byte compares, four at a time), a block-wide count
+                // from the top down gives each word the rank of its highest place, and the
+                // threads whose places rank among the first max_cands write them: one barrier,
+                // whatever the history's length.
+                const int lo = 32 * tid;
+                unsigned int bits = 0;
+                if (lo < len) {
+                    const uint4* src16 = reinterpret_cast<const uint4*>(s_m + lo);
+                    const uint4 q0 = src16[0], q1 = src16[1];
+                    const unsigned int w[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
+                    const unsigned int want = 0x01010101u * (unsigned int)kstar;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const unsigned int eq = (__vcmpeq4(w[i], want) >> 7) & 0x01010101u;   // bit 0 of each equal byte
+                        bits |= ((eq * 0x01020408u) >> 24 & 0xFu) << (4 * i);
+                    }
+                    const int valid = min(32, len - lo);
+                    if (valid < 32) bits &= (1u << valid) - 1u;
+                    if (tid == 0) bits &= ~1u;
+                }
+                const int mine = __popc(bits);
+                int incl = mine;   // hits of this lane and of the lanes above it
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int dn = __shfl_down_sync(0xFFFFFFFFu, incl, o);
+                    if (lane + o < 32) incl += dn;
+                }
+                if (lane == 0) s_hits[warp] = (unsigned int)incl;   // the warp's hits
+                __syncthreads();
+                const int others = (int)s_hits[lane];
+                const int above = __reduce_add_sync(0xFFFFFFFFu, lane > warp ? others : 0);
+                const int all = __reduce_add_sync(0xFFFFFFFFu, others);
+                int rank = above + incl - mine;
+                unsigned int left = bits;
+                while (left && rank < max_cands) {
+                    const int bit = 31 - __clz(left);    // the highest place of the word first
+                    left &= ~(1u << bit);
+                    if (!AASD_IN_RANGE(rank >= 0 && rank < kMaxCands && lo + bit >= 1 && lo + bit < len, a.state)) break;
+                    s_pos[rank++] = lo + bit;
+                }
+                if (tid == 0) s_count = min(all, max_cands);
+                __syncthreads();
+                continue;
+            }
             const int top = src == 0 ? len : pool_len;     // places 1 .. top - 1
             for (int hi = top; hi > 1 && s_count < max_cands; hi -= 32 * kHitWords) {
                 const int lo = max(1, hi - 32 * kHitWords);   // window [lo, hi)
