@@ -17,7 +17,8 @@ emitted tokens are appended as always; the state is replayed (restored every 8 s
 small device copy inside the timed region).
 
 After the K timed steps the same step runs for a few seconds more (the `sustained` leg,
-clocks sampled inside it), the sampling variants of the two streaming kernels are timed on
+clocks sampled inside it, followed by the copy that defines the bandwidth peak run for as
+long), the sampling variants of the two streaming kernels are timed on
 the same buffers, and alignment sampling runs over one whole long-context prefill block
 (16384 x 128256 bf16, 4.2 GB).
 
@@ -489,6 +490,38 @@ def run_ours(args, rank, world, local_rank):
                      "sm_mhz_median": sclk["sm_mhz"], "sm_mhz_min": sclk.get("sm_min_mhz"),
                      "power_w_max": sclk.get("power_w_max"), "reasons": sclk["reasons"],
                      "clock_samples": sclk["samples"], "events": "every %dth step" % every}
+        # the operation the copy peak is defined by (torch copy_ of 1 Gi bf16 elements, read +
+        # write), run for as long: what the memory system itself sustains under the same cap
+        if world == 1:
+            n_el = 1 << 30
+            src = torch.empty(n_el, dtype=torch.bfloat16, device=dev).normal_()
+            dst = torch.empty_like(src)
+            for _ in range(3):
+                dst.copy_(src)
+            c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            c0.record()
+            dst.copy_(src)
+            c1.record()
+            torch.cuda.synchronize()
+            n_copy = max(8, int(s_ms / c0.elapsed_time(c1)))
+            cclocks = ClockSampler(local_rank, period_s=0.005)
+            cmark = cclocks.mark()
+            c0.record()
+            for _ in range(n_copy):
+                dst.copy_(src)
+            c1.record()
+            torch.cuda.synchronize()
+            cclk = cclocks.stop(since=cmark)
+            copy_gbs = 2.0 * n_el * 2 * n_copy / (c0.elapsed_time(c1) * 1e-3) / 1e9
+            sustained["copy_reference"] = {
+                "what": "torch copy_ of 1 Gi bf16 elements (read + write), %d copies back to back" % n_copy,
+                "seconds": c0.elapsed_time(c1) * 1e-3, "gbs": copy_gbs, "sm_mhz_median": cclk["sm_mhz"],
+                "power_w_max": cclk.get("power_w_max"), "reasons": cclk["reasons"]}
+            sustained["verify_frac_of_sustained_copy"] = sustained["verify_gbs"] / copy_gbs
+            sustained["align_frac_of_sustained_copy"] = sustained["align_gbs"] / copy_gbs
+            del src, dst
+            torch.cuda.empty_cache()
 
     # what a read-only stream with no arithmetic reaches on this device, same buffers, same run
     sink = torch.zeros(1, dtype=torch.int32, device=dev)
