@@ -381,7 +381,10 @@ int aasd_draft(aasd_ctx* ctx, const aasd_draft_in* in, const aasd_draft_params* 
         return AASD_ERR_INVALID_ARG;
     DraftArgs a{*in, *p, *out, ctx->state};
     AASD_CUDA(cudaSetDevice(ctx->device));
-    launch(draft_kernel, (unsigned int)p->n_seqs, (unsigned int)kDraftThreads, 0, ctx->stream, a);
+    if (p->n_seqs > ctx->sm_count)
+        launch(draft_kernel<kDraftThreadsBatch>, (unsigned int)p->n_seqs, (unsigned int)kDraftThreadsBatch, 0, ctx->stream, a);
+    else
+        launch(draft_kernel<kDraftThreads>, (unsigned int)p->n_seqs, (unsigned int)kDraftThreads, 0, ctx->stream, a);
     return after_launch(ctx, 1);
 }
 

@@ -8,7 +8,8 @@ namespace aasd {
 constexpr int kMaxCands = 64;   // candidates per sequence a draft call can emit
 constexpr int kExtScan = 32;    // depths per main whose extra counts are fetched in parallel
 constexpr int kDraftThreads = 1024;   // one CTA per sequence: long histories want many lanes
-constexpr int kDraftWarps = kDraftThreads / 32;
+constexpr int kDraftThreadsBatch = 256;   // batches with more sequences than SMs: CTAs share an SM, and the
+                                          // step is made of instructions every warp issues, so fewer warps each
 constexpr int kHitWords = 128;        // places per window of the lookup = 32 * kHitWords
 constexpr int kMatchBytes = 32768;    // histories up to this many tokens keep their match lengths in shared memory
 
@@ -36,7 +37,9 @@ __device__ __forceinline__ int place_of(int code) { return code <= -2 ? -2 - cod
 // warp reads the places off in descending order.  A history of more than one window whose
 // lengths are all kept in shared memory takes one pass instead: a word of hit bits per thread,
 // a block-wide count from the top down, and every thread writes its own places.
-__global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs a) {
+template <int NT>
+__global__ void __launch_bounds__(NT) draft_kernel(const DraftArgs a) {
+    constexpr int kWarps = NT / 32;
     __shared__ int s_rec[AASD_MAX_NGRAM];
     __shared__ int s_pos[kMaxCands];        // places of the mains (pool places encoded)
     __shared__ int s_len[kMaxCands];        // and how many tokens follow them
@@ -70,7 +73,7 @@ __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs a)
     int front[kBatch];
 #pragma unroll
     for (int u = 0; u < kBatch; ++u) {
-        const int p = 1 + tid + u * kDraftThreads;
+        const int p = 1 + tid + u * NT;
         front[u] = p < len ? h[p - 1] : AASD_NONE;
     }
     int rl;
@@ -139,17 +142,17 @@ __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs a)
         // together, so that their trips to memory overlap, and the full comparison runs for
         // the few places that pass this test.
         const int want_last = rl > 0 ? s_rec[rl - 1] : AASD_NONE;
-        for (int base = 1 + tid; base < len; base += kBatch * kDraftThreads) {
+        for (int base = 1 + tid; base < len; base += kBatch * NT) {
             if (base != 1 + tid) {
 #pragma unroll
                 for (int u = 0; u < kBatch; ++u) {
-                    const int p = base + u * kDraftThreads;
+                    const int p = base + u * NT;
                     front[u] = p < len ? h[p - 1] : AASD_NONE;
                 }
             }
 #pragma unroll
             for (int u = 0; u < kBatch; ++u) {
-                const int p = base + u * kDraftThreads;
+                const int p = base + u * NT;
                 if (p >= len) break;
                 const int m = (rl > 0 && (front[u] == want_last || match_align)) ? match_len_at(p) : 0;
                 if (cached) s_m[p] = (unsigned char)m;
@@ -157,7 +160,7 @@ __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs a)
             }
         }
     }
-    for (int p = 1 + tid; p < pool_len; p += kDraftThreads) best = max(best, pool_match_len_at(p));
+    for (int p = 1 + tid; p < pool_len; p += NT) best = max(best, pool_match_len_at(p));
     best = __reduce_max_sync(0xFFFFFFFFu, best);
     if (lane == 0 && best > 0) atomicMax(&s_kstar, best);
     __syncthreads();
@@ -167,7 +170,7 @@ __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs a)
     // windows of 32 * kHitWords places from the top down
     if (kstar > 0) {
         for (int src = 0; src < 2; ++src) {
-            if (src == 0 && cached && len > 32 * kHitWords) {
+            if (src == 0 && cached && len > 32 * kHitWords && len <= 32 * NT) {
                 // (a history of a single window measured no slower by the windows below)
                 // Every place's length is in shared memory: thread t turns places 32 t .. 32 t + 31
                 // into a word of hit bits (byte compares, four at a time), a block-wide count
@@ -199,7 +202,7 @@ __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs a)
                 }
                 if (lane == 0) s_hits[warp] = (unsigned int)incl;   // the warp's hits
                 __syncthreads();
-                const int others = (int)s_hits[lane];
+                const int others = lane < kWarps ? (int)s_hits[lane] : 0;
                 const int above = __reduce_add_sync(0xFFFFFFFFu, lane > warp ? others : 0);
                 const int all = __reduce_add_sync(0xFFFFFFFFu, others);
                 int rank = above + incl - mine;
@@ -218,7 +221,7 @@ __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs a)
             for (int hi = top; hi > 1 && s_count < max_cands; hi -= 32 * kHitWords) {
                 const int lo = max(1, hi - 32 * kHitWords);   // window [lo, hi)
                 const int words = (hi - lo + 31) / 32;
-                for (int wd = warp; wd < words; wd += kDraftWarps) {
+                for (int wd = warp; wd < words; wd += kWarps) {
                     const int p = lo + wd * 32 + lane;
                     const bool hit = p < hi && (src == 0 ? (cached ? (int)s_m[p] : match_len_at(p)) : pool_match_len_at(p)) == kstar;
                     const unsigned int bal = __ballot_sync(0xFFFFFFFFu, hit);
@@ -264,7 +267,7 @@ __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs a)
     int32_t* c_pos = a.out.cand_pos + (int64_t)b * max_cands;
     // how many tokens follow each main: up to draft_len, to the end of its buffer, and in the
     // pool to the end of the document
-    for (int c = tid; c < n_main; c += kDraftThreads) {
+    for (int c = tid; c < n_main; c += NT) {
         const int code = s_pos[c], p = place_of(code);
         int L;
         if (!is_pool_place(code)) {
@@ -276,7 +279,7 @@ __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs a)
         s_len[c] = L;
     }
     __syncthreads();
-    for (int i = tid; i < max_cands * draft_len; i += kDraftThreads) {
+    for (int i = tid; i < max_cands * draft_len; i += NT) {
         const int c = i / draft_len, j = i % draft_len;
         int tok = AASD_NONE;
         unsigned int fl = 0;
@@ -293,7 +296,7 @@ __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs a)
         d_ids[i] = tok;
         d_fl[i] = (uint8_t)fl;
     }
-    for (int c = tid; c < max_cands; c += kDraftThreads) {
+    for (int c = tid; c < max_cands; c += NT) {
         c_len[c] = c < n_main ? s_len[c] : 0;
         c_pos[c] = c < n_main ? s_pos[c] : AASD_NONE;
     }
@@ -306,7 +309,7 @@ __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs a)
         return is_pool_place(code) ? n_pool_ext(q) : n_ext(q);
     };
     if (any_table && n_main < max_cands) {
-        for (int i = tid; i < n_main * scan; i += kDraftThreads) {
+        for (int i = tid; i < n_main * scan; i += NT) {
             const int c = i / scan, depth = i % scan;
             s_next[c * kExtScan + depth] = (unsigned char)(depth < s_len[c] ? extras_at(c, depth) : 0);
         }
@@ -335,7 +338,7 @@ __global__ void __launch_bounds__(kDraftThreads) draft_kernel(const DraftArgs a)
     }
     __syncthreads();
     const int total = s_total;
-    for (int i = tid; i < (total - n_main) * draft_len; i += kDraftThreads) {
+    for (int i = tid; i < (total - n_main) * draft_len; i += NT) {
         const int slot = n_main + i / draft_len, q = i % draft_len;
         const int c = s_alt[slot] >> 16, es = (s_alt[slot] >> 12) & 15, depth = s_alt_depth[slot];
         const int code = s_pos[c], p = place_of(code);

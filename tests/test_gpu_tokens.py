@@ -122,6 +122,46 @@ def test_draft_histories_longer_than_one_window(ctx):
         assert ref["cand_pos"][0, :ref["n_cands"][0]].tolist() == sorted(planted, reverse=True)[:max_cands]
 
 
+@pytest.mark.parametrize("with_align", [False, True])
+def test_draft_batches_with_more_sequences_than_sms(ctx, with_align):
+    # such batches run narrower CTAs (several share an SM); histories of a few tokens, of one
+    # window, of several windows whose match lengths still fit shared memory, and beyond that
+    rng = np.random.default_rng(77 + with_align)
+    B, n, K = 200, 5, 2
+    c = _draft_case(rng, B, 4, 900, K, with_align, n, own_tail=True)
+    # four long sequences in front, binary alphabet so that matches abound
+    long_lens = [5000, 8192, 9000, 40000]
+    lens = np.concatenate([long_lens, c["lens"][4:]]).astype(np.int32)
+    caps = lens + 3
+    offs = np.concatenate([[0], np.cumsum(caps)]).astype(np.int32)
+    hist = np.full(offs[-1], -1, np.int32)
+    for b in range(B):
+        src = rng.integers(0, 2, lens[b]) if b < 4 else c["hist"][c["offs"][b]:c["offs"][b] + lens[b]]
+        hist[offs[b]:offs[b] + lens[b]] = src
+    plens = np.minimum(c["plens"], lens).astype(np.int32)
+    plens[:4] = [4000, 8192, 100, 30000]
+    align = {}
+    ref_kw = {}
+    if with_align:
+        arow = np.concatenate([[0], np.cumsum(plens)]).astype(np.int32)
+        align_ids = np.full((arow[-1], K), -1, np.int32)
+        align_n = rng.integers(0, K + 1, arow[-1]).astype(np.int32)
+        for k in range(K):
+            align_ids[:, k] = np.where(align_n > k, rng.integers(0, 6, arow[-1]) + 10 * k, -1)
+        ref_kw = dict(align_ids=align_ids, align_n=align_n, align_row_offsets=arow[:-1], k_extra=K)
+        align = dict(align_ids=_dev(align_ids), align_n=_dev(align_n), align_row_offsets=_dev(arow[:-1]))
+    recent = np.full((B, n), -1, np.int32)
+    for b in range(B):
+        rl = min(n, lens[b])
+        recent[b, :rl] = hist[offs[b] + lens[b] - rl: offs[b] + lens[b]]
+    rlen = np.minimum(n, lens).astype(np.int32)
+    for max_cands, draft_len in ((6, 7), (64, 3)):
+        ref = oracle.draft(hist, offs, lens, plens, recent, rlen, n, draft_len, max_cands, **ref_kw)
+        got = ctx.draft(_dev(hist), _dev(offs), _dev(lens), _dev(plens), n, draft_len, max_cands, **align)
+        check_draft(got, ref)
+    assert ref["match_len"][:4].min() >= 1
+
+
 def _pool_case(rng, B, alphabet, max_len, pool_len, K, tables, n):
     c = _draft_case(rng, B, alphabet, max_len, K, tables, n, own_tail=bool(rng.integers(0, 2)))
     pool = rng.integers(0, alphabet, pool_len).astype(np.int32)
