@@ -23,22 +23,30 @@ ALIGN_TOPK, ALIGN_GUMBEL = 0, 1
 VERIFY_CONDITIONAL, VERIFY_STRICT_GREEDY, VERIFY_STRICT_SAMPLED, VERIFY_TOP_K = 0, 1, 2, 3
 
 
-def build(force: bool = False) -> str:
-    """Compile the oracle with g++ (no-op when the library is newer than the source)."""
-    if (not force and os.path.exists(_LIB)
-            and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC)):
-        return _LIB
-    tmp = _LIB + ".tmp.%d" % os.getpid()
-    subprocess.check_call(["g++", "-O2", "-std=c++17", "-fopenmp", "-shared", "-fPIC",
-                           _SRC, "-o", tmp])
-    os.replace(tmp, _LIB)
-    return _LIB
+_LIB_SAN = os.path.join(_HERE, "liboracle_san.so")
+_SAN_FLAGS = ["-O1", "-g", "-fno-omit-frame-pointer", "-fsanitize=address,undefined", "-fno-sanitize-recover=all"]
+
+
+def build(force: bool = False, sanitized: bool = False) -> str:
+    """Compile the oracle with g++ (no-op when the library is newer than the source).
+
+    sanitized: the same source with AddressSanitizer and UndefinedBehaviorSanitizer, as a second
+    library; a process loads it by setting AASD_ORACLE_SANITIZED=1 and preloading libasan."""
+    out = _LIB_SAN if sanitized else _LIB
+    if (not force and os.path.exists(out)
+            and os.path.getmtime(out) >= os.path.getmtime(_SRC)):
+        return out
+    tmp = out + ".tmp.%d" % os.getpid()
+    subprocess.check_call(["g++"] + (_SAN_FLAGS if sanitized else ["-O2"]) +
+                          ["-std=c++17", "-fopenmp", "-shared", "-fPIC", _SRC, "-o", tmp])
+    os.replace(tmp, out)
+    return out
 
 
 def lib():
     global _lib
     if _lib is None:
-        _lib = C.CDLL(build())
+        _lib = C.CDLL(build(sanitized=os.environ.get("AASD_ORACLE_SANITIZED") == "1"))
         _lib.oracle_gumbel_of.restype = C.c_double
         _lib.oracle_gumbel_of.argtypes = [C.c_uint32]
         _lib.oracle_sample_row.restype = C.c_int32
