@@ -262,6 +262,18 @@ def test_config5_serving_batch256():
     assert r["open"]["below_delta"] > 0 and r["closed"]["below_delta"] > 0
 
 
+def test_config5_sampling_and_top_k_modes():
+    # the serving batch at full size through the kernels with the keyed sampler (GUMBEL extras in
+    # prefill, STRICT_SAMPLED verification: the launches the benchmark times as `roofline_sampled`)
+    # and through top-k verification; draws and counts are compared bit for bit on the followed
+    # sequences, every other sequence by the properties
+    r = _run_config(4, 2, align_mode=binding.ALIGN_GUMBEL, verify_mode=binding.VERIFY_STRICT_SAMPLED,
+                    loops=("open",))
+    assert min(r["open"]["real_rows"]) == 1.0 and r["counters"]["rows"] >= 64 * 4096
+    r = _run_config(4, 2, verify_mode=binding.VERIFY_TOP_K, loops=("open",))
+    assert min(r["open"]["real_rows"]) == 1.0 and r["open"]["tokens_per_step"] >= 1.5
+
+
 def test_config5_with_table_extension():
     # the serving batch with alignment sampling on generated context switched on
     r = _run_config(4, 4, extend=True, loops=("closed",))
