@@ -118,10 +118,8 @@ __device__ __forceinline__ float exponential_fast(unsigned int r) {
     const float two_m32 = 2.3283064365386963e-10f;
     const float w = fmaf((float)(~r), two_m32, 0.5f * two_m32);
     const float u = fmaf((float)r, two_m32, 0.5f * two_m32);
-    // w + w^2/2 + ... + w^6/6: truncation below 2^-30 relative for w < 2^-5
-    float p = fmaf(w, 1.0f / 6.0f, 0.2f);
-    p = fmaf(w, p, 0.25f);
-    p = fmaf(w, p, 1.0f / 3.0f);
+    // w + w^2/2 + w^3/3 + w^4/4: truncation below w^4/5 < 2e-7 relative for w < 2^-5
+    float p = fmaf(w, 0.25f, 1.0f / 3.0f);
     p = fmaf(w, p, 0.5f);
     p = fmaf(w, p, 1.0f);
     const float near_one = w * p;

@@ -669,14 +669,15 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
                     // A thread takes the eight neighbouring vectors 8 * tid .. 8 * tid + 7 of the
                     // tile: two sampling groups of bf16 ids (vectors 0-3 and 4-7), one group of
                     // fp32 ids.  So that a quarter-warp covers all shared-memory banks with every
-                    // load, a lane reads the two halves in an order given by bit 2 of its index
-                    // and rotates inside a half by its two low bits; which half a register holds
-                    // is then known at compile time up to one swap at the end.
+                    // load, load k of a lane takes vector k ^ (lane & 7): bit 2 of the lane index
+                    // swaps the two halves, its two low bits permute inside a half, and the
+                    // address is one logic operation away from the thread's base; which half a
+                    // register holds is known at compile time up to one swap at the end.
                     constexpr int kPer = kTileVecs / kConsumers;
                     constexpr int kVecsPerGroup = kGroup / kVec;           // 4 (bf16) or 8 (fp32)
                     constexpr int kGroupsPerThread = kPer / kVecsPerGroup; // 2 or 1
                     static_assert(kPer == 8 && kGroupsPerThread >= 1, "eight vectors per thread and tile");
-                    const int hsel = (lane >> 2) & 1, rot = lane & 3;
+                    const int hsel = (lane >> 2) & 1, l7 = lane & 7;
                     // the groups' random variates need their indices only: issued first, the
                     // generator's long dependent chain runs beside the exponentials below
                     const int g0 = (v0 + kPer * tid) * kVec / kGroup;
@@ -691,18 +692,18 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
                     if (nv == kTileVecs) {
 #pragma unroll
                         for (int k = 0; k < kPer; ++k)
-                            q[k] = lds16(base + (size_t)(kPer * tid + (((((k >> 2) ^ hsel) & 1) << 2) | ((k + rot) & 3))) * 16);
+                            q[k] = lds16(base + (size_t)(kPer * tid + (k ^ l7)) * 16);
 #pragma unroll
                         for (int k = 0; k < kPer; ++k) {
                             add_to_group<DT, K, FIN>(acc, q[k], c1, neg_refc, k < 4 ? first : second, k < 4 ? first_b : second_b);
                             if (kLazyMax) tilemax.update(q[k]);
-                            else acc.track(q[k], v0 + kPer * tid + (((((k >> 2) ^ hsel) & 1) << 2) | ((k + rot) & 3)));
+                            else acc.track(q[k], v0 + kPer * tid + (k ^ l7));
                         }
                     } else {
                         bool ok[kPer];
 #pragma unroll
                         for (int k = 0; k < kPer; ++k) {
-                            const int v = kPer * tid + (((((k >> 2) ^ hsel) & 1) << 2) | ((k + rot) & 3));
+                            const int v = kPer * tid + (k ^ l7);
                             ok[k] = v < nv;
                             if (ok[k]) q[k] = lds16(base + (size_t)v * 16);
                         }
@@ -711,7 +712,7 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
                             if (ok[k]) {
                                 add_to_group<DT, K, FIN>(acc, q[k], c1, neg_refc, k < 4 ? first : second, k < 4 ? first_b : second_b);
                                 if (kLazyMax) tilemax.update(q[k]);
-                                else acc.track(q[k], v0 + kPer * tid + (((((k >> 2) ^ hsel) & 1) << 2) | ((k + rot) & 3)));
+                                else acc.track(q[k], v0 + kPer * tid + (k ^ l7));
                             }
                     }
                     first = __fadd2_rn(first, first_b);
