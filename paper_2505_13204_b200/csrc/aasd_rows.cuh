@@ -297,7 +297,7 @@ struct RowFinal {
     // probability of a token from its raw logit, with the exponent the streaming pass used
     __device__ double prob(float x) const {
         const double t = centered ? ((double)x + neg_refc) * c1 : (double)x * c1 + neg_refc;
-        return exp2(t) / S;
+        return fmin(exp2(t) / S, 1.0);   // (S comes from fp32 sums: a lone spike may land a hair above 1)
     }
 };
 
@@ -323,7 +323,7 @@ __device__ inline RowFinal finish_row(const RowPartial& p, float c1, float neg_r
         f.S = 1.0;
         return f;
     }
-    f.H = log(p.S) - kLn2 * (p.A / p.S);
+    f.H = fmax(log(p.S) - kLn2 * (p.A / p.S), 0.0);   // (and its entropy a hair below 0)
     f.pmax = f.prob(f.m);
     return f;
 }
@@ -362,12 +362,12 @@ __device__ inline RowFinal finish_row_warp(const RowPartial& p, float c1, float 
                                 : (centered ? ((double)my_x + f.neg_refc) * f.c1 : (double)my_x * f.c1 + f.neg_refc);
     const double e = exp2(t);
     const double inv_s = 1.0 / p.S;
-    my_prob = e * inv_s;
+    my_prob = fmin(e * inv_s, 1.0);   // a probability (Eq. 4, 6): the fp32 sums may put a lone spike a hair above 1
     const double u = __shfl_sync(0xFFFFFFFFu, e, 31) * p.S - 1.0;
     constexpr double kInvLn2 = 1.4426950408889634;
     double log2_s = (double)y0 + u * (kInvLn2 + u * (-0.5 * kInvLn2 + u * (kInvLn2 / 3.0)));
     if (!(fabs(u) <= 1.0e-3)) log2_s = log2(p.S);   // ... so take the library's logarithm there
-    f.H = kLn2 * (log2_s - p.A * inv_s);
+    f.H = fmax(kLn2 * (log2_s - p.A * inv_s), 0.0);   // an entropy: likewise never below 0
     return f;
 }
 

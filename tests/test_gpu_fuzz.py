@@ -115,7 +115,7 @@ def test_random_case(ctx, case):
                          finite_hint=finite and mode != binding.VERIFY_STRICT_SAMPLED, **kw)
         if mode != binding.VERIFY_STRICT_SAMPLED:
             got = dict(got, sampled=None)
-        check_verify(got, ref, offs_np, dtype)
+        check_verify(got, ref, offs_np, dtype, alpha=alpha)
         if mode == binding.VERIFY_TOP_K:
             assert np.array_equal(cpu(got["n_greater"]), ref["n_greater"])
     else:

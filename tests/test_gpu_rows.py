@@ -81,7 +81,7 @@ def test_verify_parity(ctx, V, dtype, stride, rows, mode):
     xd = _to_dev(x)
     got = ctx.verify(xd, torch.as_tensor(d).cuda(), torch.as_tensor(offs).cuda(),
                      draft_flags=torch.as_tensor(flags).cuda(), alpha=alpha, beta=beta, mode=mode)
-    check_verify(got, ref, offs, dtype)
+    check_verify(got, ref, offs, dtype, alpha=alpha)
     st = ctx.poll_status()
     assert bool(st & binding.STATUS_ID_RANGE) == (rows > 10)
     assert not (st & binding.STATUS_BAD_ROW)
@@ -276,7 +276,7 @@ def test_finite_hint_gives_the_same_results(ctx, V, dtype, stride, rows):
     ctx.reset_counters()
     got = ctx.verify(_to_dev(x), torch.as_tensor(d).cuda(), torch.as_tensor(offs).cuda(), alpha=alpha, beta=beta,
                      finite_hint=True)
-    check_verify(got, ref, offs, dtype)
+    check_verify(got, ref, offs, dtype, alpha=alpha)
     prompt = rng.integers(0, V, rows).astype(np.int32)
     refa = oracle.align_sample(to_oracle(x), prompt, [0, rows], k_extra=2)
     gota = ctx.align_sample(_to_dev(x), torch.as_tensor(prompt).cuda(), [0, rows], k_extra=2, finite_hint=True)
@@ -310,7 +310,7 @@ def test_temperature_and_thresholds(ctx):
         ref = oracle.verify(to_oracle(x), d, offs, alpha=alpha, beta=beta, inv_temperature=invT)
         got = ctx.verify(x.cuda(), torch.as_tensor(d).cuda(), torch.as_tensor(offs).cuda(),
                          alpha=alpha, beta=beta, inv_temperature=invT)
-        check_verify(got, ref, offs, torch.bfloat16)
+        check_verify(got, ref, offs, torch.bfloat16, alpha=alpha)
         gr = ctx.verify(x.cuda(), torch.as_tensor(d).cuda(), None, alpha=alpha, beta=beta,
                         inv_temperature=invT, rows_per_cand=8)
         assert torch.equal(gr["accept_len"], got["accept_len"])
@@ -392,7 +392,7 @@ def test_cluster_and_global_combine_agree(V, dtype, rows, monkeypatch):
         results.append({**{"v_" + k: w.clone() for k, w in v.items() if w is not None},
                         "t_n_greater": t["n_greater"].clone(), "t_accept": t["accept"].clone(),
                         **{"a_" + k: w.clone() for k, w in a.items() if w is not None}})
-        check_verify(v, oracle.verify(to_oracle(x), d, offs, alpha=alpha, beta=beta), offs, dtype)
+        check_verify(v, oracle.verify(to_oracle(x), d, offs, alpha=alpha, beta=beta), offs, dtype, alpha=alpha)
         rt = oracle.verify(to_oracle(x), d, offs, mode=binding.VERIFY_TOP_K, top_k=3)
         assert np.array_equal(cpu(t["n_greater"]), rt["n_greater"])
         check_align(a, oracle.align_sample(to_oracle(x), d, seq, k_extra=2), dtype)
