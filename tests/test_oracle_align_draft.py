@@ -280,7 +280,7 @@ def test_draft_lookup_is_algorithm_1s_dictionary():
         L = int(rng.integers(3, 120))
         h = rng.integers(0, 3 + trial % 4, L)
         n = int(rng.integers(1, 8))
-        rl = int(rng.integers(1, n + 1))
+        rl = min(int(rng.integers(1, n + 1)), L)          # (a key taken from the history is no longer than it)
         rec = h[L - rl:] if trial % 3 else rng.integers(0, 4, rl)
         k, places = _dictionary_lookup(list(h), list(rec), n)
         recent = np.full(n, -1, np.int32)
