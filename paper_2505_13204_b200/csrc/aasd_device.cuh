@@ -224,9 +224,13 @@ struct RowAccumulator {
             for (int i = 1; i < kVec; ++i) vmax = fmaxf(vmax, x[i]);
             int vi = vec_index;
 #pragma unroll
+            bool up = false;
             for (int j = 0; j < K; ++j) {
-                // strict '>' keeps the earlier (lower id) vector ahead among equals
-                bool up = vmax > best[j];
+                // A thread meets its vectors in ascending order, so a new one goes ahead of a kept
+                // one only if it is larger ('>' keeps the lower id ahead among equals); what a
+                // slot hands down was ranked above everything below it and stays so, whatever
+                // the comparison of the values alone says (equal values: it is the earlier one).
+                up = up || vmax > best[j];
                 float hi = fmaxf(best[j], vmax);
                 float lo = fminf(best[j], vmax);
                 int hi_i = up ? vi : best_vec[j];

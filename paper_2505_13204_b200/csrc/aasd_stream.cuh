@@ -311,14 +311,21 @@ struct TileAccumulator {
         }
         track(raw, vec_index);
     }
-    // the vector joins the K best ones if its maximum says so
+    // The vector joins the K best ones if its maximum says so.  ASCENDING: the thread meets its
+    // vectors in ascending order, so a new one goes ahead of a kept one only if it is larger
+    // ('>' keeps the lower id ahead among equals), and what a slot hands down was ranked above
+    // everything below it and stays so whatever the values alone say (equal values: it is the
+    // earlier one).  Otherwise (the sampling kernels read a tile's vectors in an order of their
+    // own) value and index are compared at every slot.
+    template <bool ASCENDING = true>
     __device__ __forceinline__ void track(const uint4& raw, int vec_index) {
         float vmax = Clamp<DT>::vector_max(raw);
         int vi = vec_index;
+        bool up = false;
 #pragma unroll
         for (int j = 0; j < K; ++j) {
-            // strict '>' keeps the earlier (lower id) vector ahead among equals
-            const bool up = vmax > best[j];
+            if (ASCENDING) up = up || vmax > best[j];
+            else up = vmax > best[j] || (vmax == best[j] && vmax > -CUDART_INF_F && vi < best_vec[j]);
             const float hi = fmaxf(best[j], vmax);
             const float lo = fminf(best[j], vmax);
             const int hi_i = up ? vi : best_vec[j];
@@ -697,7 +704,7 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
                         for (int k = 0; k < kPer; ++k) {
                             add_to_group<DT, K, FIN>(acc, q[k], c1, neg_refc, k < 4 ? first : second, k < 4 ? first_b : second_b);
                             if (kLazyMax) tilemax.update(q[k]);
-                            else acc.track(q[k], v0 + kPer * tid + (k ^ l7));
+                            else acc.template track<false>(q[k], v0 + kPer * tid + (k ^ l7));
                         }
                     } else {
                         bool ok[kPer];
@@ -712,7 +719,7 @@ __global__ void __launch_bounds__(stream_threads(NF), 2) stream_kernel(const Str
                             if (ok[k]) {
                                 add_to_group<DT, K, FIN>(acc, q[k], c1, neg_refc, k < 4 ? first : second, k < 4 ? first_b : second_b);
                                 if (kLazyMax) tilemax.update(q[k]);
-                                else acc.track(q[k], v0 + kPer * tid + (k ^ l7));
+                                else acc.template track<false>(q[k], v0 + kPer * tid + (k ^ l7));
                             }
                     }
                     first = __fadd2_rn(first, first_b);

@@ -114,6 +114,33 @@ def test_align_parity(ctx, V, dtype, stride, rows, K):
     assert ctx.poll_status() == 0
 
 
+@pytest.mark.parametrize("V,dtype,stride", [(8192, torch.bfloat16, None), (40000, torch.bfloat16, None),
+                                            (20000, torch.float32, None), (9001, torch.bfloat16, 9001),
+                                            (152064, torch.bfloat16, None)])
+@pytest.mark.parametrize("K", [1, 2, 4])
+def test_best_tokens_on_rows_of_a_few_levels(ctx, V, dtype, stride, K):
+    """Rows whose logits take a handful of values, the higher the rarer: every rank is a tie
+    of many tokens, to be resolved by the lower id (Fig. 2), and a thread of the streaming pass
+    typically meets several vectors of one level before it meets one of the next level up.
+    The first row is that case spelt out: three vectors of one thread's share, the first two
+    at one level, the third above them."""
+    rows = 310 if V == 8192 else 24          # whole rows per CTA, or rows cut into pieces
+    rng = np.random.default_rng(V + K)
+    level = rng.choice(6, size=(rows, V), p=[0.55, 0.3, 0.1, 0.04, 0.009, 0.001]).astype(np.float32)
+    level[0, :] = 0.0
+    per = 8 if dtype == torch.bfloat16 else 4
+    for vec, val in ((5, 8.5), (5 + 256, 8.5), (5 + 512, 8.75)):
+        level[0, vec * per + 3] = val
+    x = torch.zeros((rows, stride or V), dtype=dtype)[:, :V]
+    x.copy_(torch.as_tensor(level))
+    prompt = rng.integers(0, V, rows).astype(np.int32)
+    cut = [0, 7, rows]
+    ref = oracle.align_sample(to_oracle(x), prompt, cut, k_extra=K)
+    got = ctx.align_sample(_to_dev(x), torch.as_tensor(prompt).cuda(), cut, k_extra=K)
+    check_align(got, ref, dtype)
+    assert ctx.poll_status() == 0
+
+
 SAMPLED_CASES = CASES + [
     (152064, torch.bfloat16, None, 300),   # more rows than CTA slots: whole-row items
     (32000, torch.float32, None, 310),
