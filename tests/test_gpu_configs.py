@@ -58,7 +58,7 @@ def _check_rows_against_oracle(x, ids, L, rows, got, dtype, mode, seed, tag, row
 
 
 def _run_config(index, n_follow, align_mode=binding.ALIGN_TOPK, verify_mode=binding.VERIFY_CONDITIONAL,
-                sample_rows=6, extend=False, loops=("closed", "open")):
+                sample_rows=32, extend=False, loops=("closed", "open")):
     w = synth.workload(index)
     dev = torch.device("cuda", 0)
     ctx = binding.Context()

@@ -5,7 +5,7 @@ import torch
 
 import oracle
 from paper_2505_13204_b200 import binding, synth
-from parity import F32, TOL, assert_entropy, assert_rel, cpu, to_oracle
+from parity import F32, TOL, assert_entropy, assert_rel, assert_threshold, cpu, to_oracle
 
 pytestmark = pytest.mark.gpu
 
@@ -61,7 +61,7 @@ def _check_tree(got, ref, dtype):
     assert np.array_equal(cpu(got["accept"])[~near], ref["accept"][~near])
     assert_rel(cpu(got["p_token"]), ref["p_token"], tol, "p_token")
     assert_rel(cpu(got["pmax"]), ref["pmax"], tol, "pmax")
-    assert_rel(cpu(got["threshold"]), ref["threshold"], tol, "threshold")
+    assert_threshold(cpu(got["threshold"]), ref["threshold"], ref["entropy"], tol, 0.1)
     assert_entropy(cpu(got["entropy"]), ref["entropy"], tol)
     return int(near.sum())
 
@@ -121,8 +121,8 @@ def test_verify_tree_parity(ctx, V, dtype, stride, B, Cm, Ld, mode):
         # streams) and for their siblings (counted by a second pass over the row)
         assert np.array_equal(cpu(got["n_greater"]), ref["n_greater"])
         assert B == 1 or (ref["n_greater"] >= 0).sum() > 0
-    if B >= 8:
-        assert ref["n_accept"].max() >= 1
+    if B >= 8 and mode in (binding.VERIFY_CONDITIONAL, binding.VERIFY_STRICT_GREEDY):
+        assert ref["n_accept"].max() >= 1       # (a sampled own token or a rank need not favour any child)
     assert ctx.poll_status() == 0
     again = ctx.verify_tree(xd, _dev(tok), _dev(par), offs, E, node_flags=_dev(fl, torch.uint8), alpha=alpha,
                             beta=beta, mode=mode, seed=seed, step=step, top_k=3)
