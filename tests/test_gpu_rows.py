@@ -226,7 +226,7 @@ def test_verify_top_k_parity(ctx, V, dtype, stride, rows):
                          draft_flags=torch.as_tensor(flags).cuda(), mode=binding.VERIFY_TOP_K, top_k=k)
         assert np.array_equal(cpu(got["n_greater"]), ref["n_greater"])
         check_verify(got, ref, offs, dtype)
-    assert ref["accept"].sum() > 0
+    assert rows <= 12 or ref["accept"].sum() > 0     # (a dozen rows may draw no draft among the first five)
     ctx.poll_status()
 
 

@@ -120,7 +120,7 @@ def test_verify_tree_parity(ctx, V, dtype, stride, B, Cm, Ld, mode):
         # the count is an integer and must be exact, for first children (counted while the row
         # streams) and for their siblings (counted by a second pass over the row)
         assert np.array_equal(cpu(got["n_greater"]), ref["n_greater"])
-        assert B == 1 or (ref["n_greater"] >= 0).sum() > 0
+        assert B <= 3 or (ref["n_greater"] >= 0).sum() > 0     # (a few small trees may hold no such node)
     if B >= 8 and mode in (binding.VERIFY_CONDITIONAL, binding.VERIFY_STRICT_GREEDY):
         assert ref["n_accept"].max() >= 1       # (a sampled own token or a rank need not favour any child)
     assert ctx.poll_status() == 0
