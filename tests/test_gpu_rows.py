@@ -138,6 +138,17 @@ def test_best_tokens_on_rows_of_a_few_levels(ctx, V, dtype, stride, K):
     ref = oracle.align_sample(to_oracle(x), prompt, cut, k_extra=K)
     got = ctx.align_sample(_to_dev(x), torch.as_tensor(prompt).cuda(), cut, k_extra=K)
     check_align(got, ref, dtype)
+    # the same rows through verification: the best token is the lowest id of a many-way tie
+    # (hundreds of lanes hold the maximum), and the rank of a draft token counts its ties
+    d = np.where(rng.random(rows) < 0.5, np.argmax(level, axis=1), prompt).astype(np.int32)
+    offs = np.arange(0, rows + 1, 2 if rows % 2 == 0 else 1, dtype=np.int32)
+    for mode in (binding.VERIFY_CONDITIONAL, binding.VERIFY_TOP_K, binding.VERIFY_STRICT_SAMPLED):
+        kw = dict(mode=mode, top_k=K + 1, seed=5, step=K)
+        vref = oracle.verify(to_oracle(x), d, offs, **kw)
+        vgot = ctx.verify(_to_dev(x), torch.as_tensor(d).cuda(), torch.as_tensor(offs).cuda(), **kw)
+        check_verify(vgot, vref, offs, dtype)
+        if mode == binding.VERIFY_TOP_K:
+            assert np.array_equal(cpu(vgot["n_greater"]), vref["n_greater"])
     assert ctx.poll_status() == 0
 
 
