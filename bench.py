@@ -61,8 +61,8 @@ EXTEND_TABLE = False
 # captures summarised under profiles/: (workload, kernel) -> (rows captured, bytes).  Traffic
 # is proportional to rows (each row is read once), so it is scaled to the launch's rows.
 # An entry is set to None whenever the kernel has changed since its capture.
-NCU_TRAFFIC = {("cfg5-serving-256", "verify"): (2048, 623.500032e6 + 5.597440e6),
-               ("cfg5-serving-256", "align"): (2048, 623.246592e6 + 6.961920e6)}
+NCU_TRAFFIC = {("cfg5-serving-256", "verify"): (2048, 623.521536e6 + 4.385024e6),
+               ("cfg5-serving-256", "align"): (2048, 623.264768e6 + 7.283712e6)}
 
 
 def ncu_traffic(workload: str, kernel: str, rows: int):
